@@ -1,0 +1,263 @@
+/*
+ * svip_oracle.c -- plain fp64 CPU oracle for the SVIP speculative-decoding epilogues.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, scalar, one-row-at-a-time
+ * definition that the CUDA library is checked against.  It shares no code,
+ * header, table or helper with the CUDA path, and nothing in the product
+ * (the CUDA library or its Python binding) may include, link or call it.
+ *
+ * What it follows (paper: "SVIP: Towards Training-free Dynamic Draft Length
+ * Policy for Speculative Decoding", arXiv 2411.18462):
+ *   - draft sampling and entropy stop test: Algorithm 1 (inner loop), Eq. 7
+ *   - acceptance test:   Algorithm 2 (sampling), Algorithm 3 (greedy)
+ *   - correction token:  Algorithm 4 (sampling), Algorithm 5 (greedy)
+ *   - verify loop, bonus token: Algorithm 1 (outer loop body) / Algorithm 6
+ *   - expected acceptance beta, TVD, KL: Eq. 1 - Eq. 4
+ *
+ * Readings of the paper that this file fixes (each is pinned by a CPU test):
+ *   - Algorithm 4 prints the residual with draft minus target.  Only
+ *     max(0, p - q) (target minus draft) makes the emitted token follow the
+ *     target distribution, which is the premise of speculative decoding, so
+ *     that sign is used.
+ *   - entropy is in nats (Pinsker's inequality in Eq. 3 is stated for nats).
+ *   - the stop test is exactly sqrt(H) > h, strict.
+ *   - the accept test is exactly r < p(x)/q(x), strict, r in [0,1).
+ *   - T > 0: every distribution is softmax(logits / T), and H is taken on it.
+ *     T == 0 (greedy): tokens are lowest-index argmax of the raw logits and
+ *     H is the entropy of softmax(logits) at temperature 1.
+ *   - argmax ties: lowest index among the maxima of the raw logits.
+ *   - inverse CDF: running sum in index order; the first index whose
+ *     cumulative weight EXCEEDS u * total; if rounding leaves none, the last
+ *     index with positive weight.
+ *
+ * Every function is pinned (closed forms, brute force on tiny vocabularies,
+ * chi-square tests of the emitted-token law); none is "parity unpinned".
+ *
+ * Logit rows come as raw memory: dtype 0 = IEEE fp32, dtype 1 = bfloat16 bits
+ * (uint16).  Both convert exactly to fp64.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+enum { SVIP_ORACLE_F32 = 0, SVIP_ORACLE_BF16 = 1 };
+
+static double logit_at(const void *row, int dtype, long i)
+{
+    if (dtype == SVIP_ORACLE_F32)
+        return (double)((const float *)row)[i];
+    uint32_t bits = (uint32_t)((const uint16_t *)row)[i] << 16;
+    float f;
+    memcpy(&f, &bits, sizeof f);
+    return (double)f;
+}
+
+/* Lowest index among the maxima of the raw logits. */
+long svip_oracle_argmax(const void *row, int dtype, long V)
+{
+    long best = 0;
+    double bv = logit_at(row, dtype, 0);
+    for (long i = 1; i < V; ++i) {
+        double v = logit_at(row, dtype, i);
+        if (v > bv) { bv = v; best = i; }
+    }
+    return best;
+}
+
+/* prob[i] = exp(l_i/T - M) / sum_j exp(l_j/T - M),  M = max_j l_j/T.  T > 0. */
+void svip_oracle_softmax(const void *row, int dtype, long V, double T, double *prob)
+{
+    double M = -INFINITY;
+    for (long i = 0; i < V; ++i) {
+        double s = logit_at(row, dtype, i) / T;
+        if (s > M) M = s;
+    }
+    double Z = 0.0;
+    for (long i = 0; i < V; ++i) {
+        double s = logit_at(row, dtype, i) / T;
+        double e = (s == -INFINITY) ? 0.0 : exp(s - M);
+        prob[i] = e;
+        Z += e;
+    }
+    for (long i = 0; i < V; ++i)
+        prob[i] /= Z;
+}
+
+/* H(p) = -sum p_i ln p_i, with 0 ln 0 = 0 (nats). */
+double svip_oracle_entropy(const double *prob, long V)
+{
+    double H = 0.0;
+    for (long i = 0; i < V; ++i)
+        if (prob[i] > 0.0)
+            H -= prob[i] * log(prob[i]);
+    return H;
+}
+
+/* First index whose cumulative weight exceeds u * total (index order). */
+long svip_oracle_invcdf(const double *w, long V, double u)
+{
+    double total = 0.0;
+    for (long i = 0; i < V; ++i)
+        total += w[i];
+    double target = u * total;
+    double c = 0.0;
+    long last_pos = -1;
+    for (long i = 0; i < V; ++i) {
+        c += w[i];
+        if (w[i] > 0.0) last_pos = i;
+        if (c > target) return i;
+    }
+    return last_pos;
+}
+
+/*
+ * One draft token (Algorithm 1, inner loop; Eq. 7).
+ *   T > 0 : q = softmax(l/T); token ~ q by inverse CDF at u; H = H(q)
+ *   T == 0: token = argmax l;  H = H(softmax(l))
+ *   stop  = sqrt(H) > h
+ * Returns 0, or -1 if scratch memory could not be obtained.
+ */
+int svip_oracle_draft_step(const void *row, int dtype, long V, double T, double h,
+                           double u, long *token, double *entropy, int *stop)
+{
+    double *q = (double *)malloc((size_t)V * sizeof(double));
+    if (!q) return -1;
+    if (T > 0.0) {
+        svip_oracle_softmax(row, dtype, V, T, q);
+        *token = svip_oracle_invcdf(q, V, u);
+    } else {
+        svip_oracle_softmax(row, dtype, V, 1.0, q);
+        *token = svip_oracle_argmax(row, dtype, V);
+    }
+    double H = svip_oracle_entropy(q, V);
+    *entropy = H;
+    *stop = sqrt(H) > h ? 1 : 0;
+    free(q);
+    return 0;
+}
+
+/* Acceptance probability min(1, p(x)/q(x)) of Algorithm 2; q(x) == 0 accepts iff p(x) > 0. */
+static double accept_probability(const double *p, const double *q, long x)
+{
+    if (q[x] > 0.0) {
+        double ratio = p[x] / q[x];
+        return ratio < 1.0 ? ratio : 1.0;
+    }
+    return p[x] > 0.0 ? 1.0 : 0.0;
+}
+
+/*
+ * One verification round of one sequence (Algorithm 1 outer-loop body with
+ * Algorithms 2-5).
+ *   K               draft length of this sequence (>= 1)
+ *   draft_tokens    K draft tokens x_0..x_{K-1}
+ *   q_rows          draft logits; row j starts q_stride elements after row j-1
+ *   t_rows          K+1 target logit rows, same convention with t_stride
+ *   r               K+1 uniforms in [0,1): r[0..K-1] accept draws, r[K] the
+ *                   draw for the correction or the bonus token
+ *   accept_prob     optional, K entries: min(1, p/q) at every position
+ *                   (filled for all K positions, also past the rejection)
+ * Outputs n_accepted in [0,K] and next_token (correction at position
+ * n_accepted when n_accepted < K, else the bonus token from row K).
+ * T == 0 selects the greedy variants; r is then unused and accept_prob is
+ * filled with 1.0 / 0.0.
+ */
+int svip_oracle_verify(long K, const int32_t *draft_tokens,
+                       const void *q_rows, long q_stride,
+                       const void *t_rows, long t_stride,
+                       int dtype, long V, double T, const double *r,
+                       long *n_accepted, long *next_token, double *accept_prob)
+{
+    size_t esz = dtype == SVIP_ORACLE_F32 ? 4 : 2;
+    const char *qb = (const char *)q_rows;
+    const char *tb = (const char *)t_rows;
+
+    if (!(T > 0.0)) {
+        long n_acc = K;
+        for (long j = 0; j < K; ++j) {
+            long am = svip_oracle_argmax(tb + (size_t)j * t_stride * esz, dtype, V);
+            int ok = am == (long)draft_tokens[j];
+            if (accept_prob) accept_prob[j] = ok ? 1.0 : 0.0;
+            if (!ok && n_acc == K) n_acc = j;
+        }
+        *n_accepted = n_acc;
+        *next_token = svip_oracle_argmax(tb + (size_t)n_acc * t_stride * esz, dtype, V);
+        return 0;
+    }
+
+    double *p = (double *)malloc((size_t)V * sizeof(double));
+    double *q = (double *)malloc((size_t)V * sizeof(double));
+    if (!p || !q) { free(p); free(q); return -1; }
+
+    long n_acc = K;
+    long next = -1;
+    for (long j = 0; j < K; ++j) {
+        if (n_acc < K && !accept_prob) break;
+        svip_oracle_softmax(tb + (size_t)j * t_stride * esz, dtype, V, T, p);
+        svip_oracle_softmax(qb + (size_t)j * q_stride * esz, dtype, V, T, q);
+        double a = accept_probability(p, q, (long)draft_tokens[j]);
+        if (accept_prob) accept_prob[j] = a;
+        if (n_acc < K) continue;           /* already rejected: only recording a_j */
+        if (!(r[j] < a)) {
+            n_acc = j;
+            double S = 0.0;
+            for (long i = 0; i < V; ++i) {
+                double w = p[i] - q[i];
+                q[i] = w > 0.0 ? w : 0.0;  /* q now holds the residual weights */
+                S += q[i];
+            }
+            next = S > 0.0 ? svip_oracle_invcdf(q, V, r[K])
+                           : svip_oracle_invcdf(p, V, r[K]);
+        }
+    }
+    if (n_acc == K) {
+        svip_oracle_softmax(tb + (size_t)K * t_stride * esz, dtype, V, T, p);
+        next = svip_oracle_invcdf(p, V, r[K]);
+    }
+    *n_accepted = n_acc;
+    *next_token = next;
+    free(p);
+    free(q);
+    return 0;
+}
+
+/* Eq. 1: beta = sum_x min(p(x), q(x)). */
+double svip_oracle_beta(const double *p, const double *q, long V)
+{
+    double b = 0.0;
+    for (long i = 0; i < V; ++i)
+        b += p[i] < q[i] ? p[i] : q[i];
+    return b;
+}
+
+/* Total variation distance, (1/2) sum |p - q| (Eq. 2). */
+double svip_oracle_tvd(const double *p, const double *q, long V)
+{
+    double s = 0.0;
+    for (long i = 0; i < V; ++i)
+        s += fabs(p[i] - q[i]);
+    return 0.5 * s;
+}
+
+/* Cross entropy H_{q,p} = -sum q ln p (Eq. 4); +inf if q > 0 where p == 0. */
+double svip_oracle_cross_entropy(const double *q, const double *p, long V)
+{
+    double s = 0.0;
+    for (long i = 0; i < V; ++i)
+        if (q[i] > 0.0)
+            s -= q[i] * log(p[i]);
+    return s;
+}
+
+/* Residual weights max(0, p - q) of Algorithm 4 (sign as fixed above); returns their sum. */
+double svip_oracle_residual(const double *p, const double *q, long V, double *w)
+{
+    double S = 0.0;
+    for (long i = 0; i < V; ++i) {
+        double d = p[i] - q[i];
+        w[i] = d > 0.0 ? d : 0.0;
+        S += w[i];
+    }
+    return S;
+}

@@ -1,0 +1,232 @@
+"""ctypes front end of the plain-C fp64 oracle (``svip_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
+CPU-baseline timing of the benchmark.  The product (the CUDA library and its
+binding) never imports this module.
+
+Logit arrays are numpy: ``float32`` for fp32 logits, ``uint16`` for bfloat16
+bit patterns.  All arithmetic happens in the C file; this module only
+marshals arguments, loops over rows / sequences (optionally on several host
+threads -- ctypes releases the GIL) and builds the shared object with gcc.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "svip_oracle.c")
+_LIB = os.path.join(_HERE, "libsvip_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile svip_oracle.c with gcc (strict IEEE fp64: no -ffast-math)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".%d.tmp" % os.getpid()
+        subprocess.check_call(
+            ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-Wall", "-Wextra",
+             "-ffp-contract=off", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(build())
+        dp = C.POINTER(C.c_double)
+        L.svip_oracle_argmax.restype = C.c_long
+        L.svip_oracle_argmax.argtypes = [C.c_void_p, C.c_int, C.c_long]
+        L.svip_oracle_softmax.restype = None
+        L.svip_oracle_softmax.argtypes = [C.c_void_p, C.c_int, C.c_long, C.c_double, dp]
+        L.svip_oracle_entropy.restype = C.c_double
+        L.svip_oracle_entropy.argtypes = [dp, C.c_long]
+        L.svip_oracle_invcdf.restype = C.c_long
+        L.svip_oracle_invcdf.argtypes = [dp, C.c_long, C.c_double]
+        L.svip_oracle_draft_step.restype = C.c_int
+        L.svip_oracle_draft_step.argtypes = [
+            C.c_void_p, C.c_int, C.c_long, C.c_double, C.c_double, C.c_double,
+            C.POINTER(C.c_long), dp, C.POINTER(C.c_int)]
+        L.svip_oracle_verify.restype = C.c_int
+        L.svip_oracle_verify.argtypes = [
+            C.c_long, C.c_void_p, C.c_void_p, C.c_long, C.c_void_p, C.c_long,
+            C.c_int, C.c_long, C.c_double, dp,
+            C.POINTER(C.c_long), C.POINTER(C.c_long), dp]
+        for name in ("svip_oracle_beta", "svip_oracle_tvd", "svip_oracle_cross_entropy"):
+            f = getattr(L, name)
+            f.restype = C.c_double
+            f.argtypes = [dp, dp, C.c_long]
+        L.svip_oracle_residual.restype = C.c_double
+        L.svip_oracle_residual.argtypes = [dp, dp, C.c_long, dp]
+        _lib = L
+    return _lib
+
+
+def _dtype_code(a: np.ndarray) -> int:
+    if a.dtype == np.float32:
+        return 0
+    if a.dtype == np.uint16:
+        return 1
+    raise TypeError("logits must be float32 or uint16 (bfloat16 bits), got %s" % a.dtype)
+
+
+def _dptr(a: np.ndarray):
+    return a.ctypes.data_as(C.POINTER(C.c_double))
+
+
+def _rows2d(a: np.ndarray) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    if a.ndim == 1:
+        a = a[None, :]
+    assert a.ndim == 2
+    return a
+
+
+def softmax(row: np.ndarray, T: float = 1.0) -> np.ndarray:
+    row = np.ascontiguousarray(row)
+    out = np.empty(row.shape[-1], dtype=np.float64)
+    lib().svip_oracle_softmax(row.ctypes.data, _dtype_code(row), row.shape[-1], float(T), _dptr(out))
+    return out
+
+
+def entropy(prob: np.ndarray) -> float:
+    prob = np.ascontiguousarray(prob, dtype=np.float64)
+    return float(lib().svip_oracle_entropy(_dptr(prob), prob.size))
+
+
+def invcdf(w: np.ndarray, u: float) -> int:
+    w = np.ascontiguousarray(w, dtype=np.float64)
+    return int(lib().svip_oracle_invcdf(_dptr(w), w.size, float(u)))
+
+
+def argmax(row: np.ndarray) -> int:
+    row = np.ascontiguousarray(row)
+    return int(lib().svip_oracle_argmax(row.ctypes.data, _dtype_code(row), row.shape[-1]))
+
+
+def beta(p, q) -> float:
+    p = np.ascontiguousarray(p, dtype=np.float64); q = np.ascontiguousarray(q, dtype=np.float64)
+    return float(lib().svip_oracle_beta(_dptr(p), _dptr(q), p.size))
+
+
+def tvd(p, q) -> float:
+    p = np.ascontiguousarray(p, dtype=np.float64); q = np.ascontiguousarray(q, dtype=np.float64)
+    return float(lib().svip_oracle_tvd(_dptr(p), _dptr(q), p.size))
+
+
+def cross_entropy(q, p) -> float:
+    p = np.ascontiguousarray(p, dtype=np.float64); q = np.ascontiguousarray(q, dtype=np.float64)
+    return float(lib().svip_oracle_cross_entropy(_dptr(q), _dptr(p), p.size))
+
+
+def residual(p, q):
+    p = np.ascontiguousarray(p, dtype=np.float64); q = np.ascontiguousarray(q, dtype=np.float64)
+    w = np.empty_like(p)
+    S = float(lib().svip_oracle_residual(_dptr(p), _dptr(q), p.size, _dptr(w)))
+    return w, S
+
+
+def _pmap(fn, n, threads):
+    if threads <= 1 or n <= 1:
+        for i in range(n):
+            fn(i)
+        return
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        list(ex.map(fn, range(n)))
+
+
+def draft_step(logits: np.ndarray, T: float, h: float, uniforms: np.ndarray, threads: int = 1):
+    """Rows of ``logits`` [B,V] -> (token int64[B], entropy float64[B], stop uint8[B])."""
+    logits = _rows2d(logits)
+    B, V = logits.shape
+    code = _dtype_code(logits)
+    u = np.ascontiguousarray(uniforms, dtype=np.float64).reshape(B)
+    token = np.empty(B, dtype=np.int64)
+    H = np.empty(B, dtype=np.float64)
+    stop = np.empty(B, dtype=np.uint8)
+    L = lib()
+    base = logits.ctypes.data
+    rowbytes = logits.strides[0]
+
+    def one(b):
+        tok = C.c_long(); ent = C.c_double(); st = C.c_int()
+        rc = L.svip_oracle_draft_step(base + b * rowbytes, code, V, float(T), float(h), float(u[b]),
+                                      C.byref(tok), C.byref(ent), C.byref(st))
+        if rc != 0:
+            raise MemoryError("oracle draft_step")
+        token[b] = tok.value; H[b] = ent.value; stop[b] = st.value
+
+    _pmap(one, B, threads)
+    return token, H, stop
+
+
+def verify(draft_tokens: np.ndarray, q_logits: np.ndarray, target_logits: np.ndarray,
+           cu_rows: np.ndarray, T: float, uniforms: np.ndarray,
+           q_row_of=None, want_accept_prob: bool = False, threads: int = 1):
+    """One verification round for a batch.
+
+    ``cu_rows`` int[B+1] is the exclusive prefix of (K_i+1): target row of
+    (i,j) is ``cu_rows[i]+j``; ``uniforms`` is indexed like target rows.
+    Draft-side arrays (``draft_tokens``, rows of ``q_logits``) are indexed by
+    ``q_row_of(i, j)``; the default is the packed layout ``cu_rows[i]-i+j``.
+    Returns (n_accepted int64[B], next_token int64[B], accept_prob list | None).
+    """
+    q_logits = _rows2d(q_logits)
+    target_logits = _rows2d(target_logits)
+    V = target_logits.shape[1]
+    code = _dtype_code(target_logits)
+    assert _dtype_code(q_logits) == code and q_logits.shape[1] == V
+    cu = np.asarray(cu_rows, dtype=np.int64)
+    B = cu.size - 1
+    toks = np.ascontiguousarray(draft_tokens, dtype=np.int32)
+    u = np.ascontiguousarray(uniforms, dtype=np.float64)
+    n_acc = np.empty(B, dtype=np.int64)
+    nxt = np.empty(B, dtype=np.int64)
+    aprob = [None] * B
+    L = lib()
+    esz = target_logits.itemsize
+
+    def one(i):
+        K = int(cu[i + 1] - cu[i] - 1)
+        if q_row_of is None:
+            rows = np.arange(K, dtype=np.int64) + (cu[i] - i)
+        else:
+            rows = np.array([q_row_of(i, j) for j in range(K)], dtype=np.int64)
+        # the C routine wants one stride between consecutive draft rows
+        qstride_rows = int(rows[1] - rows[0]) if K > 1 else 1
+        assert K == 1 or np.all(np.diff(rows) == qstride_rows)
+        xi = np.ascontiguousarray(toks[rows])
+        ri = np.ascontiguousarray(u[cu[i]:cu[i] + K + 1])
+        a = np.empty(K, dtype=np.float64) if want_accept_prob else None
+        na = C.c_long(); nx = C.c_long()
+        rc = L.svip_oracle_verify(
+            K, xi.ctypes.data,
+            q_logits.ctypes.data + int(rows[0]) * q_logits.strides[0], qstride_rows * V,
+            target_logits.ctypes.data + int(cu[i]) * target_logits.strides[0], V,
+            code, V, float(T), _dptr(ri), C.byref(na), C.byref(nx),
+            _dptr(a) if a is not None else None)
+        if rc != 0:
+            raise MemoryError("oracle verify")
+        assert esz in (2, 4)
+        n_acc[i] = na.value; nxt[i] = nx.value; aprob[i] = a
+
+    _pmap(one, B, threads)
+    return n_acc, nxt, (aprob if want_accept_prob else None)
+
+
+def pack_ragged(draft_len):
+    """Exclusive prefix of (K_i+1) and the row -> (sequence, position) maps, by plain loops."""
+    cu = [0]
+    row_seq, row_pos = [], []
+    for i, K in enumerate(draft_len):
+        for j in range(int(K) + 1):
+            row_seq.append(i)
+            row_pos.append(j)
+        cu.append(cu[-1] + int(K) + 1)
+    return (np.array(cu, dtype=np.int64), np.array(row_seq, dtype=np.int64),
+            np.array(row_pos, dtype=np.int64))
