@@ -1,0 +1,199 @@
+/*
+ * svip.h -- C ABI of the SVIP speculative-decoding epilogue library (sm_100a).
+ *
+ * The library computes, on the GPU, the vocabulary-wide per-step work of
+ * self-verification speculative decoding (SVIP, arXiv 2411.18462):
+ *   draft side : temperature softmax, entropy, sample, entropy stop test
+ *                (Algorithm 1 inner loop, Eq. 7)
+ *   target side: softmax of the K+1 target rows, accept test min(1, p/q),
+ *                first rejection, correction token from the normalised
+ *                residual max(0, p - q) or bonus token
+ *                (Algorithm 1 outer-loop body, Algorithms 2-5)
+ * Model forwards are not part of it: callers hand over logits.
+ *
+ * Conventions for every call
+ *   - Pointers marked DEVICE point to memory of the context's GPU, owned by
+ *     the caller.  Logit rows must be aligned to their element size; any row
+ *     start, any row stride and any V are accepted.  Pointers marked HOST are
+ *     ordinary host memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Calls enqueue work on it and return; they never synchronise
+ *     and never allocate (only svip_create and svip_graph_end allocate,
+ *     only svip_read_status synchronises).
+ *   - Return value: SVIP_OK (0) or a negative svip_status.  Argument errors
+ *     are found on the host before anything is launched.  Data-dependent
+ *     trouble (a row whose maximum is not finite, a draft length outside
+ *     [1, K_max]) never traps: it sets bits in a device status word that
+ *     svip_read_status returns.
+ *   - Logits: SVIP_F32 = IEEE binary32, SVIP_BF16 = bfloat16.  Arithmetic is
+ *     fp32.  -inf logits carry zero mass; NaN logits are treated as -inf.
+ *   - Temperature T > 0 selects sampling; T == 0 selects the greedy variants
+ *     (lowest-index argmax of the raw logits).
+ *   - Uniform random numbers are inputs (fp32 in [0,1)); the library draws
+ *     none itself.
+ *   - Inverse-CDF sampling: the token is the first index whose cumulative
+ *     weight, in index order, exceeds u * total.
+ *   - A context is bound to one device and may be used by one host thread at
+ *     a time; calls that share a context must not overlap on the GPU (they
+ *     share its workspace).
+ */
+#ifndef SVIP_H
+#define SVIP_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct svip_ctx svip_ctx;
+typedef struct svip_graph svip_graph;
+
+typedef enum { SVIP_F32 = 0, SVIP_BF16 = 1 } svip_dtype;
+
+typedef enum {
+    SVIP_OK = 0,
+    SVIP_ERR_INVALID_ARG = -1, /* null pointer, size <= 0, T < 0, NaN threshold, misaligned pointer */
+    SVIP_ERR_UNSUPPORTED = -2, /* unknown dtype, device that is not compute capability 10.x */
+    SVIP_ERR_WORKSPACE = -3,   /* more rows than the context was created for */
+    SVIP_ERR_CUDA = -4,        /* a CUDA runtime call failed; svip_last_cuda_error() has its code */
+    SVIP_ERR_STATE = -5        /* graph capture begun twice, ended without begin, ... */
+} svip_status;
+
+/* bits of the device status word */
+#define SVIP_STATUS_NONFINITE_ROW 1u /* some row's maximum was +inf, or every logit was -inf / NaN */
+#define SVIP_STATUS_BAD_DRAFT_LEN 2u /* svip_pack_ragged saw K_i outside [1, K_max] (it was clamped) */
+
+/* draft-side layout selector for svip_verify: rows packed sequence after sequence */
+#define SVIP_Q_PACKED (-1L)
+
+/* Text for a status code (static storage). */
+const char* svip_strerror(int status);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int svip_version(void);
+
+/* CUDA error code of the last call that returned SVIP_ERR_CUDA on this context (0 if none). */
+int svip_last_cuda_error(const svip_ctx* ctx);
+
+/*
+ * Creates a context on `device` with a workspace for up to `max_rows` target
+ * rows (and as many draft rows) per svip_verify call.  Allocates device
+ * memory (about 32 bytes per row); makes `device` current while it runs and
+ * restores the previous device.  *ctx is written only on success.
+ */
+int svip_create(svip_ctx** ctx, int device, int max_rows);
+
+/* Frees the workspace.  The caller must have drained all streams that used the context. */
+int svip_destroy(svip_ctx* ctx);
+
+/*
+ * Launch-shape override, for tests and tuning: `cluster_size` in {0,1,2,4,8}
+ * is the number of thread blocks (one cluster) that share one logits row;
+ * 0 restores the automatic choice from (rows, V, dtype).  Every choice gives
+ * the same integers, and entropies equal to within fp32 summation order.
+ */
+int svip_set_cluster_size(svip_ctx* ctx, int cluster_size);
+
+/* Number of kernels this context has launched (or recorded into a graph) so far. */
+long svip_launch_count(const svip_ctx* ctx);
+
+/* Copies the device status word to *flags (HOST) and clears it.  Synchronises `stream`. */
+int svip_read_status(svip_ctx* ctx, unsigned* flags, void* stream);
+
+/*
+ * One draft token for each of B sequences (Algorithm 1, inner loop: the
+ * sampling line and the entropy test; Eq. 7).
+ *
+ *   logits      DEVICE, row b starts at element b*row_stride and has V logits
+ *   T           temperature; T > 0: q = softmax(logits/T), token ~ q by inverse
+ *               CDF at uniforms[b], entropy = H(q).  T == 0: token = argmax,
+ *               entropy = H(softmax(logits)) (temperature 1).
+ *   thresh      h of Eq. 7
+ *   uniforms    DEVICE [B] fp32 in [0,1); may be NULL when T == 0
+ *   token       DEVICE [B] int32 out
+ *   entropy     DEVICE [B] fp32 out, nats, >= 0
+ *   stop        DEVICE [B] uint8 out: 1 iff sqrt(entropy) > thresh (strict)
+ *   row_stats   DEVICE [B][2] fp32 out or NULL: (m, Z) with m the largest logit
+ *               and Z = sum_i exp((l_i - m)/T') where T' = T (or 1 when T == 0);
+ *               svip_verify takes these as q_stats and then need not re-read
+ *               the draft rows whose tokens it accepts
+ */
+int svip_draft_step(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, int V,
+                    long row_stride, float T, float thresh, const float* uniforms,
+                    int32_t* token, float* entropy, uint8_t* stop, float* row_stats,
+                    void* stream);
+
+/*
+ * Ragged packing of per-sequence draft lengths (the per-sequence gamma that
+ * Algorithm 1 sets when the stop test fires; batching sequences of different
+ * gamma is an addition of this library -- the paper's algorithms handle one
+ * sequence).
+ *
+ *   draft_len   DEVICE [B] int32, K_i in [1, K_max] (else clamped + status bit)
+ *   cu_rows     DEVICE [B+1] int32 out: exclusive prefix of (K_i + 1); target row
+ *               of (sequence i, position j) is cu_rows[i] + j, draft row of the
+ *               packed layout is cu_rows[i] - i + j
+ *   row_seq     DEVICE [B*(K_max+1)] int32 out or NULL: sequence of each target row
+ *   row_pos     DEVICE [B*(K_max+1)] int32 out or NULL: position of each target row
+ *               (entries past the last target row are left untouched)
+ * 1 <= B <= 65536, 1 <= K_max, B*(K_max+1) < 2^31.
+ */
+int svip_pack_ragged(svip_ctx* ctx, const int32_t* draft_len, int B, int K_max,
+                     int32_t* cu_rows, int32_t* row_seq, int32_t* row_pos, void* stream);
+
+/*
+ * One verification round for B sequences (Algorithm 1, outer-loop body).
+ *
+ * For sequence i with K_i draft tokens, T > 0: for j = 0..K_i-1 in order,
+ * accept while uniforms[cu_rows[i]+j] < p_j(x_j)/q_j(x_j) (Algorithm 2); at
+ * the first failure n_accepted[i] = j and next_token[i] is drawn from
+ * max(0, p_j - q_j)/sum (Algorithm 4, with the sign that keeps the target
+ * distribution) by inverse CDF at uniforms[cu_rows[i]+K_i]; if nothing fails,
+ * n_accepted[i] = K_i and next_token[i] ~ p_{K_i} with that same uniform.
+ * T == 0: accept while argmax p_j == x_j (Algorithm 3); next_token is the
+ * argmax of target row n_accepted (Algorithm 5); uniforms unused (may be NULL).
+ * p_j = softmax(target row j / T), q_j = softmax(draft row j / T).
+ *
+ *   draft_tokens   DEVICE int32, indexed by draft row
+ *   q_logits       DEVICE draft logits, draft row r starts at element r*q_row_stride
+ *                  (may be NULL when T == 0)
+ *   q_stats        DEVICE [draft rows][2] fp32 as written by svip_draft_step with
+ *                  the same T, or NULL (then recomputed from q_logits)
+ *   q_seq_stride,  draft row of (i, j) = i*q_seq_stride + j*q_pos_stride; or, with
+ *   q_pos_stride   q_seq_stride == SVIP_Q_PACKED, cu_rows[i] - i + j (which is
+ *                  i*K + j when cu_rows == NULL)
+ *   target_logits  DEVICE, target row r starts at element r*t_row_stride
+ *   cu_rows        DEVICE [B+1] from svip_pack_ragged, or NULL: every sequence
+ *                  has the fixed draft length K
+ *   K              the fixed draft length (cu_rows == NULL), else K_max
+ *   n_target_rows  total target rows, sum (K_i + 1); the host knows it from the
+ *                  target forward.  Must be B*(K+1) when cu_rows == NULL.
+ *   uniforms       DEVICE [n_target_rows] fp32 in [0,1), indexed like target rows
+ *   n_accepted     DEVICE [B] int32 out, in [0, K_i]
+ *   next_token     DEVICE [B] int32 out
+ * Needs n_target_rows <= max_rows of svip_create (else SVIP_ERR_WORKSPACE).
+ */
+int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits,
+                long q_row_stride, const float* q_stats, long q_seq_stride, long q_pos_stride,
+                const void* target_logits, long t_row_stride, svip_dtype dtype,
+                const int32_t* cu_rows, int B, int K, int n_target_rows, int V, float T,
+                const float* uniforms, int32_t* n_accepted, int32_t* next_token, void* stream);
+
+/*
+ * CUDA-graph replay for latency-bound use (small B).  Between begin and end
+ * every svip_* call on `stream` is recorded instead of run; svip_graph_end
+ * returns an executable graph that svip_graph_launch replays.  All pointers
+ * passed while recording must stay valid and are re-read at every replay
+ * (refill the logits / uniforms buffers in place between replays).
+ * The paper has no counterpart; this serves the B = 1 step latency.
+ */
+int svip_graph_begin(svip_ctx* ctx, void* stream);
+int svip_graph_end(svip_ctx* ctx, void* stream, svip_graph** graph);
+int svip_graph_launch(svip_graph* graph, void* stream);
+int svip_graph_destroy(svip_graph* graph);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SVIP_H */

@@ -1,0 +1,172 @@
+"""ctypes binding of the C ABI in ``include/svip.h``: argument marshalling only.
+
+Every method of :class:`Context` has the name and the argument order of the C
+function it calls.  Device buffers may be given as ``torch`` CUDA tensors (their
+``data_ptr()`` is passed) or as integer device addresses; ``stream`` may be a
+``torch.cuda.Stream``, an integer ``cudaStream_t`` or ``None`` (the legacy
+default stream).  Nothing here computes: if the compiled library is missing the
+import of a symbol fails with :class:`SvipError`.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+SVIP_F32 = 0
+SVIP_BF16 = 1
+SVIP_Q_PACKED = -1
+SVIP_STATUS_NONFINITE_ROW = 1
+SVIP_STATUS_BAD_DRAFT_LEN = 2
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "csrc", "libsvip.so")
+_lib = None
+
+
+class SvipError(RuntimeError):
+    def __init__(self, code: int, text: str):
+        super().__init__("svip: %s (status %d)" % (text, code))
+        self.code = code
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def library():
+    """Loads csrc/libsvip.so (built by ``python -m paper_2411_18462_b200.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise SvipError(-100, "CUDA library %s is not built; run python -m paper_2411_18462_b200.build"
+                        % _LIB_PATH)
+    L = C.CDLL(_LIB_PATH)
+    vp, i32, lng, f32 = C.c_void_p, C.c_int, C.c_long, C.c_float
+    L.svip_strerror.restype = C.c_char_p
+    L.svip_strerror.argtypes = [i32]
+    L.svip_version.restype = i32
+    L.svip_version.argtypes = []
+    L.svip_last_cuda_error.restype = i32
+    L.svip_last_cuda_error.argtypes = [vp]
+    L.svip_create.restype = i32
+    L.svip_create.argtypes = [C.POINTER(vp), i32, i32]
+    L.svip_destroy.restype = i32
+    L.svip_destroy.argtypes = [vp]
+    L.svip_set_cluster_size.restype = i32
+    L.svip_set_cluster_size.argtypes = [vp, i32]
+    L.svip_launch_count.restype = lng
+    L.svip_launch_count.argtypes = [vp]
+    L.svip_read_status.restype = i32
+    L.svip_read_status.argtypes = [vp, C.POINTER(C.c_uint), vp]
+    L.svip_draft_step.restype = i32
+    L.svip_draft_step.argtypes = [vp, vp, i32, i32, i32, lng, f32, f32, vp, vp, vp, vp, vp, vp]
+    L.svip_pack_ragged.restype = i32
+    L.svip_pack_ragged.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
+    L.svip_verify.restype = i32
+    L.svip_verify.argtypes = [vp, vp, vp, lng, vp, lng, lng, vp, lng, i32, vp, i32, i32, i32, i32, f32,
+                              vp, vp, vp, vp]
+    L.svip_graph_begin.restype = i32
+    L.svip_graph_begin.argtypes = [vp, vp]
+    L.svip_graph_end.restype = i32
+    L.svip_graph_end.argtypes = [vp, vp, C.POINTER(vp)]
+    L.svip_graph_launch.restype = i32
+    L.svip_graph_launch.argtypes = [vp, vp]
+    L.svip_graph_destroy.restype = i32
+    L.svip_graph_destroy.argtypes = [vp]
+    _lib = L
+    return L
+
+
+def _ptr(x):
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    return x.data_ptr()
+
+
+def _stream(s):
+    if s is None:
+        return None
+    if isinstance(s, int):
+        return s
+    return s.cuda_stream
+
+
+def _check(code: int, ctx=None):
+    if code != 0:
+        text = library().svip_strerror(code).decode()
+        if code == -4 and ctx is not None:
+            text += " (cudaError %d)" % library().svip_last_cuda_error(ctx)
+        raise SvipError(code, text)
+
+
+class Graph:
+    def __init__(self, handle):
+        self._h = handle
+
+    def launch(self, stream=None):
+        _check(library().svip_graph_launch(self._h, _stream(stream)))
+
+    def destroy(self):
+        if self._h:
+            library().svip_graph_destroy(self._h)
+            self._h = None
+
+
+class Context:
+    """Owns an ``svip_ctx``; methods mirror the C functions one to one."""
+
+    def __init__(self, device: int = 0, max_rows: int = 1 << 15):
+        self._h = C.c_void_p()
+        _check(library().svip_create(C.byref(self._h), int(device), int(max_rows)))
+
+    def destroy(self):
+        if self._h:
+            library().svip_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def set_cluster_size(self, cluster_size: int):
+        _check(library().svip_set_cluster_size(self._h, int(cluster_size)))
+
+    def launch_count(self) -> int:
+        return int(library().svip_launch_count(self._h))
+
+    def read_status(self, stream=None) -> int:
+        flags = C.c_uint(0)
+        _check(library().svip_read_status(self._h, C.byref(flags), _stream(stream)), self._h)
+        return int(flags.value)
+
+    def draft_step(self, logits, dtype, B, V, row_stride, T, thresh, uniforms, token, entropy, stop,
+                   row_stats=None, stream=None):
+        _check(library().svip_draft_step(self._h, _ptr(logits), int(dtype), int(B), int(V), int(row_stride),
+                                         float(T), float(thresh), _ptr(uniforms), _ptr(token), _ptr(entropy),
+                                         _ptr(stop), _ptr(row_stats), _stream(stream)), self._h)
+
+    def pack_ragged(self, draft_len, B, K_max, cu_rows, row_seq=None, row_pos=None, stream=None):
+        _check(library().svip_pack_ragged(self._h, _ptr(draft_len), int(B), int(K_max), _ptr(cu_rows),
+                                          _ptr(row_seq), _ptr(row_pos), _stream(stream)), self._h)
+
+    def verify(self, draft_tokens, q_logits, q_row_stride, q_stats, q_seq_stride, q_pos_stride,
+               target_logits, t_row_stride, dtype, cu_rows, B, K, n_target_rows, V, T, uniforms,
+               n_accepted, next_token, stream=None):
+        _check(library().svip_verify(self._h, _ptr(draft_tokens), _ptr(q_logits), int(q_row_stride),
+                                     _ptr(q_stats), int(q_seq_stride), int(q_pos_stride),
+                                     _ptr(target_logits), int(t_row_stride), int(dtype), _ptr(cu_rows),
+                                     int(B), int(K), int(n_target_rows), int(V), float(T), _ptr(uniforms),
+                                     _ptr(n_accepted), _ptr(next_token), _stream(stream)), self._h)
+
+    def graph_begin(self, stream):
+        _check(library().svip_graph_begin(self._h, _stream(stream)), self._h)
+
+    def graph_end(self, stream) -> Graph:
+        g = C.c_void_p()
+        _check(library().svip_graph_end(self._h, _stream(stream), C.byref(g)), self._h)
+        return Graph(g)

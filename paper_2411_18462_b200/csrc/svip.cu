@@ -1,0 +1,840 @@
+// SVIP speculative-decoding epilogues for sm_100a: kernels and the C ABI (see include/svip.h).
+//
+// Kernels
+//   draft_step_kernel    Algorithm 1 inner loop + Eq. 7: one pass over a logits row gives
+//                        max / mass / entropy term / argmax; the sampled token is then found by
+//                        re-reading one warp segment.  A row is shared by a thread-block
+//                        cluster (1..8 blocks) whose partials meet in distributed shared memory.
+//   row_stats_kernel     softmax normalisers (or argmax, greedy) of target rows, and of draft
+//                        rows when the caller has no q_stats.
+//   verify_finish_kernel Algorithms 2 and 4 + the loop of Algorithm 1: ratio tests by one warp
+//                        (ballot + first set bit = first rejection), then the residual
+//                        max(0, p - q) or the bonus row is sampled by inverse CDF.
+//   verify_greedy_kernel Algorithms 3 and 5 on the per-row argmax.
+//   pack_ragged_kernel   exclusive scan of (K_i + 1) and the row -> (sequence, position) maps.
+#include "svip_device.cuh"
+
+#include <cmath>
+#include <cstdio>
+#include <new>
+
+#include "svip.h"
+
+namespace svip {
+
+struct SegEntry {
+    float m;
+    int idx;
+    float Z;
+    float A;
+};
+
+// Reads every segment entry of the cluster (warp-collective, run by warp 0 of each block), merges
+// them into the row's partial and selects the segment holding the mass u * Z.
+template <int kMode>
+__device__ __forceinline__ void combine_segments(cg::cluster_group& cluster, SegEntry* seg, int S,
+                                                 float c, float u, int lane, Partial& row,
+                                                 SegPick& pick) {
+    const int nseg = S * kWarps;
+    const int per = (nseg + 31) / 32;
+    Partial e[kSegPerLane];
+    float m = neg_inf();
+#pragma unroll
+    for (int k = 0; k < kSegPerLane; ++k) {
+        e[k].m = neg_inf(); e[k].idx = kIntMax; e[k].Z = 0.f; e[k].A = 0.f;
+        int s = lane * per + k;
+        if (k < per && s < nseg) {
+            const SegEntry* remote = cluster.map_shared_rank(seg, s / kWarps);
+            SegEntry v = remote[s % kWarps];
+            e[k].m = v.m; e[k].idx = v.idx; e[k].Z = v.Z; e[k].A = v.A;
+        }
+        m = fmaxf(m, e[k].m);
+    }
+    m = warp_max(m);
+    int idx = kIntMax;
+    float mass[kSegPerLane];
+    float asum = 0.f;
+#pragma unroll
+    for (int k = 0; k < kSegPerLane; ++k) {
+        if (e[k].m == m) idx = min(idx, e[k].idx);
+        rescale_to<kMode>(e[k], m, c);
+        mass[k] = e[k].Z;
+        asum += e[k].A;
+    }
+    row.m = m;
+    row.idx = warp_min_int(idx);
+    row.A = warp_sum(asum);
+    pick = pick_segment(mass, per, nseg, u, lane);
+    row.Z = pick.total;
+}
+
+// Fine scan of one segment by the whole block.  `wf(vi, w)` yields the weights of the elements
+// of vector vi.  Returns the virtual element index (vector * EPV + lane element) of the first
+// element whose cumulative weight exceeds `target`, else the last element with positive weight,
+// else -1.
+template <int EPV, class WF>
+__device__ __forceinline__ int fine_scan(WF& wf, int v_lo, int v_hi, float prefix, float target,
+                                         ScanShared& sh, int tid, int lane, int warp) {
+    if (tid == 0) { sh.hit = kIntMax; sh.lastpos = -1; }
+    __syncthreads();
+    float running = prefix;
+    for (int cb = v_lo; cb < v_hi; cb += kThreads) {
+        int vi = cb + tid;
+        float w[EPV];
+        float ls = 0.f;
+        if (vi < v_hi) {
+            wf(vi, w);
+#pragma unroll
+            for (int j = 0; j < EPV; ++j) ls += w[j];
+        } else {
+#pragma unroll
+            for (int j = 0; j < EPV; ++j) w[j] = 0.f;
+        }
+        float total;
+        float ex = block_scan_excl(ls, sh.wsum, lane, warp, total);
+        float cum = running + ex;
+        int myhit = kIntMax, mylast = -1;
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) {
+            cum += w[j];
+            if (w[j] > 0.f) {
+                mylast = vi * EPV + j;
+                if (cum > target && myhit == kIntMax) myhit = vi * EPV + j;
+            }
+        }
+        if (myhit != kIntMax) atomicMin(&sh.hit, myhit);
+        if (mylast >= 0) atomicMax(&sh.lastpos, mylast);
+        __syncthreads();
+        if (sh.hit != kIntMax) break;
+        running += total;
+    }
+    return sh.hit != kIntMax ? sh.hit : sh.lastpos;
+}
+
+// ------------------------------------------------------------------ draft step
+
+struct DraftArgs {
+    const void* logits;
+    long row_stride;
+    int V;
+    float c;          // log2(e) / T   (T = 1 when greedy)
+    float thresh;
+    int greedy;
+    const float* uniforms;
+    int32_t* token;
+    float* entropy;
+    uint8_t* stop;
+    float* row_stats;
+    unsigned* status;
+};
+
+template <int DT>
+struct SoftmaxWeights {
+    RowGeom g;
+    float c, M;
+    __device__ __forceinline__ void operator()(int vi, float (&w)[ElemTraits<DT>::kEPV]) const {
+        constexpr int EPV = ElemTraits<DT>::kEPV;
+        float x[EPV];
+        unpack_masked<DT>(g.base[vi], vi, g, x);
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) w[j] = ex2_approx(fmaxf(__fmaf_rn(x[j], c, -M), kArgFloor));
+    }
+};
+
+struct RowShared {
+    Partial row;
+    SegPick pick;
+};
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads) draft_step_kernel(DraftArgs a) {
+    constexpr int EPV = ElemTraits<DT>::kEPV;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int S = cluster.dim_blocks().x;
+    const int rank = cluster.block_rank();
+    const int row = blockIdx.x / S;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __shared__ SegEntry seg[kWarps];
+    __shared__ ScanShared scan;
+    __shared__ RowShared res;
+
+    const char* rp = static_cast<const char*>(a.logits) +
+                     static_cast<size_t>(row) * a.row_stride * ElemTraits<DT>::kBytes;
+    const RowGeom g = make_geom<DT>(rp, a.V, S * kWarps);
+    Partial t = reduce_segment<DT, 2>(g, rank * kWarps + warp, a.c, lane);
+    t = warp_merge<2>(t, a.c);
+    if (lane == 0) { seg[warp].m = t.m; seg[warp].idx = t.idx; seg[warp].Z = t.Z; seg[warp].A = t.A; }
+    cluster.sync();
+    if (warp == 0) {
+        float u = a.greedy ? 0.f : a.uniforms[row];
+        Partial r; SegPick p;
+        combine_segments<2>(cluster, seg, S, a.c, u, lane, r, p);
+        if (lane == 0) { res.row = r; res.pick = p; }
+    }
+    cluster.sync();   // remote reads are done (blocks may now exit); res is visible block-wide
+    const Partial R = res.row;
+    const SegPick P = res.pick;
+    const bool ok = (R.Z > 0.f) && (fabsf(R.m) <= 3.0e38f);
+    if (rank == 0 && tid == 0) {
+        float H = 0.f;
+        if (ok) H = fmaxf(kLn2 * (log2f(R.Z) - R.A / R.Z), 0.f);
+        else atomicOr(a.status, SVIP_STATUS_NONFINITE_ROW);
+        a.entropy[row] = H;
+        a.stop[row] = __fsqrt_rn(H) > a.thresh ? 1 : 0;
+        if (a.row_stats) { a.row_stats[2 * row] = R.m; a.row_stats[2 * row + 1] = R.Z; }
+        if (a.greedy || !ok) a.token[row] = (R.idx >= 0 && R.idx < a.V) ? R.idx : 0;
+    }
+    if (!a.greedy && ok && P.seg / kWarps == rank) {
+        SoftmaxWeights<DT> wf;
+        wf.g = g; wf.c = a.c; wf.M = __fmul_rn(R.m, a.c);
+        int v_lo, v_hi;
+        seg_range(g, P.seg, v_lo, v_hi);
+        int virt = fine_scan<EPV>(wf, v_lo, v_hi, P.prefix, P.target, scan, tid, lane, warp);
+        if (tid == 0) a.token[row] = virt >= 0 ? virt - g.pre : R.idx;
+    }
+}
+
+// ------------------------------------------------------------------ row statistics (verify, phase 1)
+
+struct StatsArgs {
+    const void* logits;
+    long row_stride;
+    int V;
+    float c;
+    int draft_rows;          // 0: unit = row.  1: unit = (sequence, position) of a draft row
+    int K;
+    const int32_t* cu;
+    long q_seq_stride, q_pos_stride;
+    float2* out_stats;       // (m, Z) per row, indexed by target-row number
+    int32_t* out_argmax;
+    unsigned* status;
+};
+
+template <int DT, int kMode>
+__global__ void __launch_bounds__(kThreads) row_stats_kernel(StatsArgs a) {
+    cg::cluster_group cluster = cg::this_cluster();
+    const int S = cluster.dim_blocks().x;
+    const int rank = cluster.block_rank();
+    const int unit = blockIdx.x / S;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __shared__ SegEntry seg[kWarps];
+
+    long in_row = unit;
+    int out_row = unit;
+    if (a.draft_rows) {
+        int i = unit / a.K, j = unit - i * a.K;
+        int row0 = a.cu ? a.cu[i] : i * (a.K + 1);
+        int Ki = a.cu ? a.cu[i + 1] - row0 - 1 : a.K;
+        if (j >= Ki) return;   // the whole cluster leaves together
+        in_row = a.q_seq_stride < 0 ? static_cast<long>(row0 - i + j)
+                                    : i * a.q_seq_stride + j * a.q_pos_stride;
+        out_row = row0 + j;
+    }
+    const char* rp = static_cast<const char*>(a.logits) +
+                     static_cast<size_t>(in_row) * a.row_stride * ElemTraits<DT>::kBytes;
+    const RowGeom g = make_geom<DT>(rp, a.V, S * kWarps);
+    Partial t = reduce_segment<DT, kMode>(g, rank * kWarps + warp, a.c, lane);
+    t = warp_merge<kMode>(t, a.c);
+    if (lane == 0) { seg[warp].m = t.m; seg[warp].idx = t.idx; seg[warp].Z = t.Z; seg[warp].A = 0.f; }
+    cluster.sync();
+    if (rank == 0 && warp == 0) {
+        Partial r; SegPick p;
+        combine_segments<kMode>(cluster, seg, S, a.c, 0.f, lane, r, p);
+        if (lane == 0) {
+            bool ok = fabsf(r.m) <= 3.0e38f && (kMode == 0 || r.Z > 0.f);
+            if (!ok) atomicOr(a.status, SVIP_STATUS_NONFINITE_ROW);
+            if (kMode >= 1) a.out_stats[out_row] = make_float2(r.m, r.Z);
+            if (a.out_argmax) a.out_argmax[out_row] = (r.idx >= 0 && r.idx < a.V) ? r.idx : 0;
+        }
+    }
+    cluster.sync();
+}
+
+// ------------------------------------------------------------------ verify, phase 2 (sampling)
+
+struct FinishArgs {
+    const int32_t* draft_tokens;
+    const void* q_logits;
+    long q_row_stride;
+    const float2* q_stats_user;   // indexed by draft row, or NULL
+    const float2* q_stats_ws;     // indexed by target row (used when q_stats_user is NULL)
+    long q_seq_stride, q_pos_stride;
+    const void* t_logits;
+    long t_row_stride;
+    const float2* p_stats;        // indexed by target row
+    const int32_t* cu;
+    int K, V;
+    float c;
+    const float* uniforms;
+    int32_t* n_accepted;
+    int32_t* next_token;
+    unsigned* status;
+};
+
+// Weights max(0, p - q) of Algorithm 4 (or p alone for the bonus token) for one vector.
+template <int DT>
+struct ResidualWeights {
+    RowGeom gt, gq;
+    const void* qrow;
+    float c, Mp, rZp, Mq, rZq;
+    int bonus;
+    __device__ __forceinline__ void operator()(int vi, float (&w)[ElemTraits<DT>::kEPV]) const {
+        constexpr int EPV = ElemTraits<DT>::kEPV;
+        float x[EPV];
+        unpack_masked<DT>(__ldg(gt.base + vi), vi, gt, x);
+#pragma unroll
+        for (int j = 0; j < EPV; ++j)
+            w[j] = ex2_approx(fmaxf(__fmaf_rn(x[j], c, -Mp), kArgFloor)) * rZp;
+        if (bonus) return;
+        float d[EPV];
+        if (gq.pre == gt.pre) {
+            unpack_masked<DT>(__ldg(gq.base + vi), vi, gq, d);
+        } else {
+            // rows with different 16-byte phase: element loads
+#pragma unroll
+            for (int j = 0; j < EPV; ++j) {
+                int i = vi * EPV + j - gt.pre;
+                d[j] = (i >= 0 && i < gt.V) ? ElemTraits<DT>::load_one(qrow, i) : neg_inf();
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) {
+            float q = ex2_approx(fmaxf(__fmaf_rn(d[j], c, -Mq), kArgFloor)) * rZq;
+            w[j] = fmaxf(w[j] - q, 0.f);
+        }
+    }
+};
+
+struct FinishShared {
+    int n_acc;
+    SegPick pick;
+};
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads) verify_finish_kernel(FinishArgs a) {
+    using E = ElemTraits<DT>;
+    constexpr int EPV = E::kEPV;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int S = cluster.dim_blocks().x;
+    const int rank = cluster.block_rank();
+    const int i = blockIdx.x / S;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __shared__ SegEntry seg[kWarps];
+    __shared__ ScanShared scan;
+    __shared__ FinishShared fs;
+
+    const int row0 = a.cu ? a.cu[i] : i * (a.K + 1);
+    const int Ki = a.cu ? a.cu[i + 1] - row0 - 1 : a.K;
+    const long dbase = a.q_seq_stride < 0 ? static_cast<long>(row0 - i) : i * a.q_seq_stride;
+    const long dstep = a.q_seq_stride < 0 ? 1 : a.q_pos_stride;
+    const char* tl = static_cast<const char*>(a.t_logits);
+    const char* ql = static_cast<const char*>(a.q_logits);
+
+    // Algorithm 2 at every position at once; the first rejection is the lowest set bit.
+    if (warp == 0) {
+        int n_acc = Ki;
+        for (int j0 = 0; j0 < Ki; j0 += 32) {
+            int j = j0 + lane;
+            bool rej = false;
+            if (j < Ki) {
+                long dr = dbase + j * dstep;
+                int x = a.draft_tokens[dr];
+                bool acc = false;
+                if (x >= 0 && x < a.V) {
+                    float tv = E::load_one(tl + static_cast<size_t>(row0 + j) * a.t_row_stride * E::kBytes, x);
+                    float dv = E::load_one(ql + static_cast<size_t>(dr) * a.q_row_stride * E::kBytes, x);
+                    float2 ps = a.p_stats[row0 + j];
+                    float2 qs = a.q_stats_user ? a.q_stats_user[dr] : a.q_stats_ws[row0 + j];
+                    float ep = exp2f(fmaxf(__fmaf_rn(tv, a.c, -__fmul_rn(ps.x, a.c)), kArgFloor));
+                    float eq = exp2f(fmaxf(__fmaf_rn(dv, a.c, -__fmul_rn(qs.x, a.c)), kArgFloor));
+                    if (!(tv > neg_inf())) ep = 0.f;
+                    if (!(dv > neg_inf())) eq = 0.f;
+                    // r < (ep/Zp)/(eq/Zq) without the division; eq == 0 accepts iff ep > 0
+                    float r = a.uniforms[row0 + j];
+                    acc = __fmul_rn(__fmul_rn(r, eq), ps.y) < __fmul_rn(ep, qs.y);
+                }
+                rej = !acc;
+            }
+            unsigned mask = __ballot_sync(0xffffffffu, rej);
+            if (mask) { n_acc = j0 + __ffs(mask) - 1; break; }
+        }
+        if (lane == 0) fs.n_acc = n_acc;
+    }
+    __syncthreads();
+    const int n_acc = fs.n_acc;
+    const float u = a.uniforms[row0 + Ki];
+
+    ResidualWeights<DT> wf;
+    const char* trow = tl + static_cast<size_t>(row0 + n_acc) * a.t_row_stride * E::kBytes;
+    wf.gt = make_geom<DT>(trow, a.V, S * kWarps);
+    wf.c = a.c;
+    {
+        float2 ps = a.p_stats[row0 + n_acc];
+        wf.Mp = __fmul_rn(ps.x, a.c);
+        wf.rZp = 1.0f / ps.y;
+    }
+    wf.bonus = n_acc >= Ki;
+    wf.qrow = nullptr; wf.gq = wf.gt; wf.Mq = 0.f; wf.rZq = 0.f;
+    if (!wf.bonus) {
+        long dr = dbase + n_acc * dstep;
+        wf.qrow = ql + static_cast<size_t>(dr) * a.q_row_stride * E::kBytes;
+        wf.gq = make_geom<DT>(wf.qrow, a.V, S * kWarps);
+        float2 qs = a.q_stats_user ? a.q_stats_user[dr] : a.q_stats_ws[row0 + n_acc];
+        wf.Mq = __fmul_rn(qs.x, a.c);
+        wf.rZq = 1.0f / qs.y;
+    }
+
+    int token = -1;
+    for (int pass = 0; pass < 2; ++pass) {
+        // mass of this warp's segment
+        int v_lo, v_hi;
+        seg_range(wf.gt, rank * kWarps + warp, v_lo, v_hi);
+        float acc = 0.f;
+#pragma unroll 2
+        for (int vi = v_lo + lane; vi < v_hi; vi += 32) {
+            float w[EPV];
+            wf(vi, w);
+            float s = 0.f;
+#pragma unroll
+            for (int j = 0; j < EPV; ++j) s += w[j];
+            acc += s;
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) { seg[warp].m = 0.f; seg[warp].idx = 0; seg[warp].Z = acc; seg[warp].A = 0.f; }
+        cluster.sync();
+        if (warp == 0) {
+            const int nseg = S * kWarps;
+            const int per = (nseg + 31) / 32;
+            float mass[kSegPerLane];
+#pragma unroll
+            for (int k = 0; k < kSegPerLane; ++k) {
+                int s = lane * per + k;
+                mass[k] = 0.f;
+                if (k < per && s < nseg) mass[k] = cluster.map_shared_rank(seg, s / kWarps)[s % kWarps].Z;
+            }
+            SegPick p = pick_segment(mass, per, nseg, u, lane);
+            if (lane == 0) fs.pick = p;
+        }
+        cluster.sync();
+        const SegPick P = fs.pick;
+        if (P.total > 0.f) {
+            if (P.seg / kWarps == rank) {
+                seg_range(wf.gt, P.seg, v_lo, v_hi);
+                int virt = fine_scan<EPV>(wf, v_lo, v_hi, P.prefix, P.target, scan, tid, lane, warp);
+                token = virt >= 0 ? virt - wf.gt.pre : 0;
+            }
+            break;
+        }
+        // No residual mass (p == q wherever it matters): fall back to sampling from p.
+        if (wf.bonus) {
+            if (rank == 0 && tid == 0) atomicOr(a.status, SVIP_STATUS_NONFINITE_ROW);
+            if (rank == 0) token = 0;
+            break;
+        }
+        wf.bonus = 1;
+    }
+    if (tid == 0) {
+        if (rank == 0) a.n_accepted[i] = n_acc;
+        if (token >= 0) a.next_token[i] = token;
+    }
+}
+
+// ------------------------------------------------------------------ verify, phase 2 (greedy)
+
+struct GreedyArgs {
+    const int32_t* draft_tokens;
+    const int32_t* p_argmax;
+    const int32_t* cu;
+    long q_seq_stride, q_pos_stride;
+    int B, K;
+    int32_t* n_accepted;
+    int32_t* next_token;
+};
+
+__global__ void __launch_bounds__(kThreads) verify_greedy_kernel(GreedyArgs a) {
+    const int lane = threadIdx.x & 31;
+    const int i = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if (i >= a.B) return;
+    const int row0 = a.cu ? a.cu[i] : i * (a.K + 1);
+    const int Ki = a.cu ? a.cu[i + 1] - row0 - 1 : a.K;
+    const long dbase = a.q_seq_stride < 0 ? static_cast<long>(row0 - i) : i * a.q_seq_stride;
+    const long dstep = a.q_seq_stride < 0 ? 1 : a.q_pos_stride;
+    int n_acc = Ki;
+    for (int j0 = 0; j0 < Ki; j0 += 32) {
+        int j = j0 + lane;
+        bool rej = false;
+        if (j < Ki) rej = a.draft_tokens[dbase + j * dstep] != a.p_argmax[row0 + j];
+        unsigned mask = __ballot_sync(0xffffffffu, rej);
+        if (mask) { n_acc = j0 + __ffs(mask) - 1; break; }
+    }
+    if (lane == 0) {
+        a.n_accepted[i] = n_acc;
+        a.next_token[i] = a.p_argmax[row0 + n_acc];
+    }
+}
+
+// ------------------------------------------------------------------ ragged packing
+
+constexpr int kPackThreads = 1024;
+
+__global__ void __launch_bounds__(kPackThreads) pack_ragged_kernel(const int32_t* draft_len, int B, int K_max,
+                                                                   int32_t* cu, int32_t* row_seq,
+                                                                   int32_t* row_pos, unsigned* status) {
+    __shared__ int wsum[32];
+    __shared__ int carry;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) carry = 0;
+    __syncthreads();
+    for (int base = 0; base < B; base += kPackThreads) {
+        int i = base + tid;
+        int k = 0;
+        if (i < B) {
+            k = draft_len[i];
+            if (k < 1 || k > K_max) {
+                atomicOr(status, SVIP_STATUS_BAD_DRAFT_LEN);
+                k = k < 1 ? 1 : K_max;
+            }
+            k += 1;
+        }
+        int inc = k;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int n = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += n;
+        }
+        if (lane == 31) wsum[warp] = inc;
+        __syncthreads();
+        int before = 0, tot = 0;
+        for (int w = 0; w < 32; ++w) {
+            int s = wsum[w];
+            if (w < warp) before += s;
+            tot += s;
+        }
+        int c0 = carry;
+        if (i < B) cu[i] = c0 + before + inc - k;
+        __syncthreads();
+        if (tid == 0) carry = c0 + tot;
+        __syncthreads();
+    }
+    const int total = carry;
+    if (tid == 0) cu[B] = total;
+    __syncthreads();
+    if (row_seq || row_pos) {
+        for (int r = tid; r < total; r += kPackThreads) {
+            int lo = 0, hi = B;           // largest i with cu[i] <= r
+            while (hi - lo > 1) {
+                int mid = (lo + hi) >> 1;
+                if (cu[mid] <= r) lo = mid; else hi = mid;
+            }
+            if (row_seq) row_seq[r] = lo;
+            if (row_pos) row_pos[r] = r - cu[lo];
+        }
+    }
+}
+
+}  // namespace svip
+
+// ==================================================================== host side / C ABI
+
+using namespace svip;
+
+struct svip_ctx {
+    int device;
+    int max_rows;
+    int num_sms;
+    int cluster_override;
+    long launches;
+    int last_cuda;
+    int capturing;
+    float2* p_stats;
+    float2* q_stats;
+    int32_t* p_argmax;
+    unsigned* status;
+};
+
+struct svip_graph {
+    cudaGraphExec_t exec;
+    cudaGraph_t graph;
+};
+
+namespace {
+
+int cuda_fail(svip_ctx* ctx, cudaError_t e) {
+    if (ctx) ctx->last_cuda = static_cast<int>(e);
+    return SVIP_ERR_CUDA;
+}
+
+template <class Args>
+cudaError_t launch_clustered(void (*kernel)(Args), long units, int S, const Args& args, cudaStream_t st) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(units * S), 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = S;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args);
+}
+
+// Blocks per row: enough blocks to give every SM two, while every thread still has a vector.
+int pick_cluster(const svip_ctx* ctx, long rows, int V, int dtype) {
+    if (ctx->cluster_override > 0) return ctx->cluster_override;
+    long nvec = (static_cast<long>(V) * (dtype == SVIP_BF16 ? 2 : 4) + 15) / 16;
+    int S = 1;
+    while (S < kMaxCluster && rows * S < 2L * ctx->num_sms && nvec / (2 * S) >= kThreads) S *= 2;
+    return S;
+}
+
+bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+float scale_for(float T) { return static_cast<float>(1.4426950408889634 / (T > 0.f ? static_cast<double>(T) : 1.0)); }
+
+}  // namespace
+
+extern "C" {
+
+const char* svip_strerror(int status) {
+    switch (status) {
+        case SVIP_OK: return "ok";
+        case SVIP_ERR_INVALID_ARG: return "invalid argument";
+        case SVIP_ERR_UNSUPPORTED: return "unsupported dtype or device";
+        case SVIP_ERR_WORKSPACE: return "more rows than the context's workspace holds";
+        case SVIP_ERR_CUDA: return "CUDA runtime error";
+        case SVIP_ERR_STATE: return "call not valid in the context's current state";
+        default: return "unknown status";
+    }
+}
+
+int svip_version(void) { return 100; }
+
+int svip_last_cuda_error(const svip_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
+
+int svip_create(svip_ctx** out, int device, int max_rows) {
+    if (!out || max_rows < 1 || device < 0) return SVIP_ERR_INVALID_ARG;
+    int prev = 0;
+    if (cudaGetDevice(&prev) != cudaSuccess) { cudaGetLastError(); return SVIP_ERR_CUDA; }
+    if (cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return SVIP_ERR_CUDA; }
+    int rc = SVIP_OK;
+    svip_ctx* c = new (std::nothrow) svip_ctx();
+    if (!c) { cudaSetDevice(prev); return SVIP_ERR_CUDA; }
+    c->device = device;
+    c->max_rows = max_rows;
+    int major = 0, sms = 0;
+    cudaError_t e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+    if (e != cudaSuccess) rc = SVIP_ERR_CUDA;
+    else if (major != 10) rc = SVIP_ERR_UNSUPPORTED;
+    c->num_sms = sms;
+    if (rc == SVIP_OK) {
+        size_t n = static_cast<size_t>(max_rows);
+        if (cudaMalloc(&c->p_stats, n * sizeof(float2)) != cudaSuccess ||
+            cudaMalloc(&c->q_stats, n * sizeof(float2)) != cudaSuccess ||
+            cudaMalloc(&c->p_argmax, n * sizeof(int32_t)) != cudaSuccess ||
+            cudaMalloc(&c->status, sizeof(unsigned)) != cudaSuccess ||
+            cudaMemset(c->status, 0, sizeof(unsigned)) != cudaSuccess) {
+            rc = SVIP_ERR_CUDA;
+        }
+    }
+    if (rc != SVIP_OK) {
+        cudaGetLastError();
+        cudaFree(c->p_stats); cudaFree(c->q_stats); cudaFree(c->p_argmax); cudaFree(c->status);
+        delete c;
+    } else {
+        *out = c;
+    }
+    cudaSetDevice(prev);
+    return rc;
+}
+
+int svip_destroy(svip_ctx* ctx) {
+    if (!ctx) return SVIP_ERR_INVALID_ARG;
+    int prev = 0;
+    cudaGetDevice(&prev);
+    cudaSetDevice(ctx->device);
+    cudaFree(ctx->p_stats); cudaFree(ctx->q_stats); cudaFree(ctx->p_argmax); cudaFree(ctx->status);
+    cudaSetDevice(prev);
+    delete ctx;
+    return SVIP_OK;
+}
+
+int svip_set_cluster_size(svip_ctx* ctx, int cluster_size) {
+    if (!ctx) return SVIP_ERR_INVALID_ARG;
+    if (cluster_size != 0 && cluster_size != 1 && cluster_size != 2 && cluster_size != 4 && cluster_size != 8)
+        return SVIP_ERR_INVALID_ARG;
+    ctx->cluster_override = cluster_size;
+    return SVIP_OK;
+}
+
+long svip_launch_count(const svip_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int svip_read_status(svip_ctx* ctx, unsigned* flags, void* stream) {
+    if (!ctx || !flags) return SVIP_ERR_INVALID_ARG;
+    if (ctx->capturing) return SVIP_ERR_STATE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned v = 0;
+    cudaError_t e = cudaMemcpyAsync(&v, ctx->status, sizeof v, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->status, 0, sizeof v, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    *flags = v;
+    return SVIP_OK;
+}
+
+int svip_draft_step(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, int V, long row_stride,
+                    float T, float thresh, const float* uniforms, int32_t* token, float* entropy,
+                    uint8_t* stop, float* row_stats, void* stream) {
+    if (!ctx || !logits || !token || !entropy || !stop) return SVIP_ERR_INVALID_ARG;
+    if (dtype != SVIP_F32 && dtype != SVIP_BF16) return SVIP_ERR_UNSUPPORTED;
+    if (B < 0 || V < 1 || V > 0x7fffffe0 || row_stride < 0) return SVIP_ERR_INVALID_ARG;
+    if (!(T >= 0.f) || std::isinf(T) || std::isnan(thresh)) return SVIP_ERR_INVALID_ARG;
+    if (T > 0.f && !uniforms) return SVIP_ERR_INVALID_ARG;
+    if (!aligned_to(logits, dtype == SVIP_BF16 ? 2 : 4)) return SVIP_ERR_INVALID_ARG;
+    if (B == 0) return SVIP_OK;
+    DraftArgs a;
+    a.logits = logits; a.row_stride = row_stride; a.V = V; a.c = scale_for(T); a.thresh = thresh;
+    a.greedy = T > 0.f ? 0 : 1; a.uniforms = uniforms; a.token = token; a.entropy = entropy;
+    a.stop = stop; a.row_stats = row_stats; a.status = ctx->status;
+    int S = pick_cluster(ctx, B, V, dtype);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = dtype == SVIP_BF16 ? launch_clustered(draft_step_kernel<kBF16>, B, S, a, st)
+                                       : launch_clustered(draft_step_kernel<kF32>, B, S, a, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    return SVIP_OK;
+}
+
+int svip_pack_ragged(svip_ctx* ctx, const int32_t* draft_len, int B, int K_max, int32_t* cu_rows,
+                     int32_t* row_seq, int32_t* row_pos, void* stream) {
+    if (!ctx || !draft_len || !cu_rows) return SVIP_ERR_INVALID_ARG;
+    if (B < 1 || B > 65536 || K_max < 1) return SVIP_ERR_INVALID_ARG;
+    if (static_cast<long>(B) * (static_cast<long>(K_max) + 1) >= 0x7fffffffL) return SVIP_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    pack_ragged_kernel<<<1, kPackThreads, 0, st>>>(draft_len, B, K_max, cu_rows, row_seq, row_pos, ctx->status);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    return SVIP_OK;
+}
+
+int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits, long q_row_stride,
+                const float* q_stats, long q_seq_stride, long q_pos_stride, const void* target_logits,
+                long t_row_stride, svip_dtype dtype, const int32_t* cu_rows, int B, int K,
+                int n_target_rows, int V, float T, const float* uniforms, int32_t* n_accepted,
+                int32_t* next_token, void* stream) {
+    if (!ctx || !draft_tokens || !target_logits || !n_accepted || !next_token) return SVIP_ERR_INVALID_ARG;
+    if (dtype != SVIP_F32 && dtype != SVIP_BF16) return SVIP_ERR_UNSUPPORTED;
+    if (B < 0 || K < 1 || V < 1 || V > 0x7fffffe0 || t_row_stride < 0 || q_row_stride < 0) return SVIP_ERR_INVALID_ARG;
+    if (!(T >= 0.f) || std::isinf(T)) return SVIP_ERR_INVALID_ARG;
+    const bool sampling = T > 0.f;
+    if (sampling && (!q_logits || !uniforms)) return SVIP_ERR_INVALID_ARG;
+    if (q_seq_stride < 0 && q_seq_stride != SVIP_Q_PACKED) return SVIP_ERR_INVALID_ARG;
+    if (q_seq_stride >= 0 && q_pos_stride < 0) return SVIP_ERR_INVALID_ARG;
+    const size_t esz = dtype == SVIP_BF16 ? 2 : 4;
+    if (!aligned_to(target_logits, esz) || (q_logits && !aligned_to(q_logits, esz))) return SVIP_ERR_INVALID_ARG;
+    if (static_cast<long>(B) * (static_cast<long>(K) + 1) >= 0x7fffffffL) return SVIP_ERR_INVALID_ARG;
+    if (B == 0) return n_target_rows == 0 ? SVIP_OK : SVIP_ERR_INVALID_ARG;
+    if (n_target_rows < 2 * B || n_target_rows > B * (K + 1)) return SVIP_ERR_INVALID_ARG;
+    if (!cu_rows && n_target_rows != B * (K + 1)) return SVIP_ERR_INVALID_ARG;
+    if (n_target_rows > ctx->max_rows) return SVIP_ERR_WORKSPACE;
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const float c = scale_for(T);
+    cudaError_t e;
+
+    StatsArgs s;
+    s.logits = target_logits; s.row_stride = t_row_stride; s.V = V; s.c = c; s.draft_rows = 0; s.K = K;
+    s.cu = cu_rows; s.q_seq_stride = q_seq_stride; s.q_pos_stride = q_pos_stride;
+    s.out_stats = ctx->p_stats; s.out_argmax = sampling ? nullptr : ctx->p_argmax; s.status = ctx->status;
+    int S = pick_cluster(ctx, n_target_rows, V, dtype);
+    if (sampling)
+        e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 1>, n_target_rows, S, s, st)
+                               : launch_clustered(row_stats_kernel<kF32, 1>, n_target_rows, S, s, st);
+    else
+        e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 0>, n_target_rows, S, s, st)
+                               : launch_clustered(row_stats_kernel<kF32, 0>, n_target_rows, S, s, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+
+    if (!sampling) {
+        GreedyArgs g;
+        g.draft_tokens = draft_tokens; g.p_argmax = ctx->p_argmax; g.cu = cu_rows;
+        g.q_seq_stride = q_seq_stride; g.q_pos_stride = q_pos_stride; g.B = B; g.K = K;
+        g.n_accepted = n_accepted; g.next_token = next_token;
+        verify_greedy_kernel<<<(B + kWarps - 1) / kWarps, kThreads, 0, st>>>(g);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        ctx->launches += 1;
+        return SVIP_OK;
+    }
+
+    if (!q_stats) {
+        StatsArgs d = s;
+        d.logits = q_logits; d.row_stride = q_row_stride; d.draft_rows = 1;
+        d.out_stats = ctx->q_stats; d.out_argmax = nullptr;
+        long units = static_cast<long>(B) * K;
+        int Sd = pick_cluster(ctx, n_target_rows - B, V, dtype);
+        e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 1>, units, Sd, d, st)
+                               : launch_clustered(row_stats_kernel<kF32, 1>, units, Sd, d, st);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        ctx->launches += 1;
+    }
+
+    FinishArgs f;
+    f.draft_tokens = draft_tokens; f.q_logits = q_logits; f.q_row_stride = q_row_stride;
+    f.q_stats_user = reinterpret_cast<const float2*>(q_stats); f.q_stats_ws = ctx->q_stats;
+    f.q_seq_stride = q_seq_stride; f.q_pos_stride = q_pos_stride; f.t_logits = target_logits;
+    f.t_row_stride = t_row_stride; f.p_stats = ctx->p_stats; f.cu = cu_rows; f.K = K; f.V = V; f.c = c;
+    f.uniforms = uniforms; f.n_accepted = n_accepted; f.next_token = next_token; f.status = ctx->status;
+    int Sf = pick_cluster(ctx, B, V, dtype);
+    e = dtype == SVIP_BF16 ? launch_clustered(verify_finish_kernel<kBF16>, B, Sf, f, st)
+                           : launch_clustered(verify_finish_kernel<kF32>, B, Sf, f, st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    return SVIP_OK;
+}
+
+int svip_graph_begin(svip_ctx* ctx, void* stream) {
+    if (!ctx) return SVIP_ERR_INVALID_ARG;
+    if (ctx->capturing) return SVIP_ERR_STATE;
+    cudaError_t e = cudaStreamBeginCapture(static_cast<cudaStream_t>(stream), cudaStreamCaptureModeThreadLocal);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->capturing = 1;
+    return SVIP_OK;
+}
+
+int svip_graph_end(svip_ctx* ctx, void* stream, svip_graph** graph) {
+    if (!ctx || !graph) return SVIP_ERR_INVALID_ARG;
+    if (!ctx->capturing) return SVIP_ERR_STATE;
+    ctx->capturing = 0;
+    cudaGraph_t g = nullptr;
+    cudaError_t e = cudaStreamEndCapture(static_cast<cudaStream_t>(stream), &g);
+    if (e != cudaSuccess || !g) return cuda_fail(ctx, e);
+    cudaGraphExec_t ex = nullptr;
+    e = cudaGraphInstantiate(&ex, g, 0);
+    if (e != cudaSuccess) { cudaGraphDestroy(g); return cuda_fail(ctx, e); }
+    svip_graph* out = new (std::nothrow) svip_graph();
+    if (!out) { cudaGraphExecDestroy(ex); cudaGraphDestroy(g); return SVIP_ERR_CUDA; }
+    out->exec = ex; out->graph = g;
+    *graph = out;
+    return SVIP_OK;
+}
+
+int svip_graph_launch(svip_graph* graph, void* stream) {
+    if (!graph) return SVIP_ERR_INVALID_ARG;
+    return cudaGraphLaunch(graph->exec, static_cast<cudaStream_t>(stream)) == cudaSuccess ? SVIP_OK : SVIP_ERR_CUDA;
+}
+
+int svip_graph_destroy(svip_graph* graph) {
+    if (!graph) return SVIP_ERR_INVALID_ARG;
+    cudaGraphExecDestroy(graph->exec);
+    cudaGraphDestroy(graph->graph);
+    delete graph;
+    return SVIP_OK;
+}
+
+}  // extern "C"

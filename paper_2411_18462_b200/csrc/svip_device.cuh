@@ -1,0 +1,346 @@
+// Device-side building blocks shared by the SVIP kernels (sm_100a).
+//
+// A logits row is streamed once from HBM with 128-bit loads.  The row is cut
+// into NSEG = (blocks per cluster) x (warps per block) contiguous segments, one
+// per warp, so that a warp's partial sum is the mass of a contiguous index
+// range: inverse-CDF sampling then only has to re-read ONE segment (an L2 hit)
+// after the normaliser is known, instead of the whole row.
+//
+// Per-thread state while streaming:
+//   m   running maximum of the raw logits (exact in fp32)
+//   Z   sum of 2^(x*c - M),            M = rn(m*c),  c = log2(e)/T
+//   A   sum of 2^(x*c - M) * (x*c - M)               (log2 units, for the entropy)
+//   idx lowest index attaining m
+// Two partials merge by rescaling both to the larger maximum.
+#pragma once
+#include <cooperative_groups.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace svip {
+
+namespace cg = cooperative_groups;
+
+constexpr int kWarps = 16;              // warps per thread block
+constexpr int kThreads = kWarps * 32;   // threads per thread block
+constexpr int kMaxCluster = 8;          // portable cluster size limit
+constexpr int kMaxSeg = kMaxCluster * kWarps;
+constexpr int kSegPerLane = kMaxSeg / 32;
+constexpr int kF32 = 0;
+constexpr int kBF16 = 1;
+constexpr float kArgFloor = -127.0f;    // 2^x flushes to zero below this (ftz)
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr int kIntMax = 0x7fffffff;
+
+__device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
+
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// 128-bit streaming load: read-only path, no L1 allocation (each byte is used once).
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+template <int DT> struct ElemTraits;
+template <> struct ElemTraits<kF32> {
+    static constexpr int kEPV = 4;      // elements per 16-byte vector
+    static constexpr int kBytes = 4;
+    __device__ static __forceinline__ void unpack(const uint4& v, float (&x)[4]) {
+        x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y);
+        x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
+    }
+    __device__ static __forceinline__ float load_one(const void* row, int i) {
+        return __ldg(reinterpret_cast<const float*>(row) + i);
+    }
+};
+template <> struct ElemTraits<kBF16> {
+    static constexpr int kEPV = 8;
+    static constexpr int kBytes = 2;
+    // bfloat16 is the upper half of an fp32: element 2k sits in the low half-word.
+    __device__ static __forceinline__ void unpack(const uint4& v, float (&x)[8]) {
+        x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xffff0000u);
+        x[2] = __uint_as_float(v.y << 16); x[3] = __uint_as_float(v.y & 0xffff0000u);
+        x[4] = __uint_as_float(v.z << 16); x[5] = __uint_as_float(v.z & 0xffff0000u);
+        x[6] = __uint_as_float(v.w << 16); x[7] = __uint_as_float(v.w & 0xffff0000u);
+    }
+    __device__ static __forceinline__ float load_one(const void* row, int i) {
+        unsigned short h = __ldg(reinterpret_cast<const unsigned short*>(row) + i);
+        return __uint_as_float(static_cast<uint32_t>(h) << 16);
+    }
+};
+
+// Geometry of one row seen as 16-byte vectors.  The row may start anywhere:
+// the vectors start at the 16-byte boundary at or below the first element, and
+// `pre` counts the elements of the first vector that lie before the row.
+// Those, and the elements of the last vector past the row, are masked to -inf.
+// (They lie in the same 16-byte granule as valid data, so the load is safe.)
+struct RowGeom {
+    const uint4* base;
+    int pre;    // leading pad elements in vector 0
+    int V;      // valid elements
+    int nvec;   // vectors covering [0, pre + V)
+    int vps;    // vectors per segment (multiple of 8 = one 128-byte line)
+};
+
+template <int DT>
+__device__ __forceinline__ RowGeom make_geom(const void* row, int V, int nseg) {
+    using E = ElemTraits<DT>;
+    RowGeom g;
+    uintptr_t p = reinterpret_cast<uintptr_t>(row);
+    int mis = static_cast<int>(p & 15);
+    g.base = reinterpret_cast<const uint4*>(p - mis);
+    g.pre = mis / E::kBytes;
+    g.V = V;
+    g.nvec = (g.pre + V + E::kEPV - 1) / E::kEPV;
+    int vps = (g.nvec + nseg - 1) / nseg;
+    g.vps = (vps + 7) & ~7;
+    return g;
+}
+
+__device__ __forceinline__ void seg_range(const RowGeom& g, int seg, int& v_lo, int& v_hi) {
+    long lo = static_cast<long>(seg) * g.vps;
+    v_lo = lo < g.nvec ? static_cast<int>(lo) : g.nvec;
+    v_hi = min(v_lo + g.vps, g.nvec);
+}
+
+// Unpacks vector vi of the row and masks the elements outside the row to -inf.
+template <int DT>
+__device__ __forceinline__ void unpack_masked(const uint4& raw, int vi, const RowGeom& g,
+                                              float (&x)[ElemTraits<DT>::kEPV]) {
+    constexpr int EPV = ElemTraits<DT>::kEPV;
+    ElemTraits<DT>::unpack(raw, x);
+    if (vi == 0 || vi == g.nvec - 1) {
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) {
+            int e = vi * EPV + j;
+            if (e < g.pre || e >= g.pre + g.V) x[j] = neg_inf();
+        }
+    }
+}
+
+struct Partial {
+    float m;   // maximum raw logit (-inf if nothing seen)
+    int idx;   // lowest index attaining m (kIntMax if nothing seen)
+    float Z;   // mass relative to rn(m*c)
+    float A;   // sum of mass * log2-argument, relative to rn(m*c)
+};
+
+template <int EPV>
+__device__ __forceinline__ float vec_max(const float (&x)[EPV]) {
+    float t = fmaxf(x[0], x[1]);
+#pragma unroll
+    for (int j = 2; j < EPV; ++j) t = fmaxf(t, x[j]);
+    return t;
+}
+
+// Folds one vector into the thread's partial.  kMode: 0 = max/argmax only,
+// 1 = max + Z, 2 = max + Z + A.
+template <int DT, int kMode>
+__device__ __forceinline__ void fold_vector(const uint4& raw, int vi, const RowGeom& g, float c,
+                                            Partial& t, float& M) {
+    constexpr int EPV = ElemTraits<DT>::kEPV;
+    float x[EPV];
+    unpack_masked<DT>(raw, vi, g, x);
+    float tmax = vec_max<EPV>(x);
+    if (tmax > t.m) {
+        float Mn = __fmul_rn(tmax, c);
+        if (kMode >= 1 && t.m != neg_inf()) {
+            float d = M - Mn;
+            float s = ex2_approx(fmaxf(d, kArgFloor));
+            if (kMode == 2) t.A = s * __fmaf_rn(d, t.Z, t.A);
+            t.Z *= s;
+        }
+        int first = 0;
+#pragma unroll
+        for (int j = EPV - 1; j >= 0; --j)
+            if (x[j] == tmax) first = j;
+        t.m = tmax;
+        t.idx = vi * EPV + first - g.pre;
+        M = Mn;
+    }
+    if (kMode >= 1) {
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) {
+            float a = fmaxf(__fmaf_rn(x[j], c, -M), kArgFloor);   // NaN -> floor: zero mass
+            float e = ex2_approx(a);
+            t.Z += e;
+            if (kMode == 2) t.A = __fmaf_rn(e, a, t.A);
+        }
+    }
+}
+
+// Streams segment `seg` of the row with the calling warp.
+template <int DT, int kMode>
+__device__ __forceinline__ Partial reduce_segment(const RowGeom& g, int seg, float c, int lane) {
+    Partial t;
+    t.m = neg_inf(); t.idx = kIntMax; t.Z = 0.f; t.A = 0.f;
+    float M = neg_inf();
+    int v_lo, v_hi;
+    seg_range(g, seg, v_lo, v_hi);
+    int vi = v_lo + lane;
+    for (; vi + 96 < v_hi; vi += 128) {
+        uint4 r0 = ld_stream(g.base + vi);
+        uint4 r1 = ld_stream(g.base + vi + 32);
+        uint4 r2 = ld_stream(g.base + vi + 64);
+        uint4 r3 = ld_stream(g.base + vi + 96);
+        fold_vector<DT, kMode>(r0, vi, g, c, t, M);
+        fold_vector<DT, kMode>(r1, vi + 32, g, c, t, M);
+        fold_vector<DT, kMode>(r2, vi + 64, g, c, t, M);
+        fold_vector<DT, kMode>(r3, vi + 96, g, c, t, M);
+    }
+    for (; vi < v_hi; vi += 32) {
+        uint4 r0 = ld_stream(g.base + vi);
+        fold_vector<DT, kMode>(r0, vi, g, c, t, M);
+    }
+    return t;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ int warp_min_int(int v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = min(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// Rescales a partial from its own maximum to the maximum m_to (m_to >= t.m).
+template <int kMode>
+__device__ __forceinline__ void rescale_to(Partial& t, float m_to, float c) {
+    if (kMode == 0) return;
+    if (t.m == neg_inf() || !(t.Z > 0.f)) { t.Z = 0.f; t.A = 0.f; return; }
+    float d = __fmul_rn(t.m, c) - __fmul_rn(m_to, c);
+    float s = ex2_approx(fmaxf(d, kArgFloor));
+    if (kMode == 2) t.A = s * __fmaf_rn(d, t.Z, t.A);
+    t.Z *= s;
+}
+
+// All lanes return the merge of the 32 lanes' partials.
+template <int kMode>
+__device__ __forceinline__ Partial warp_merge(Partial t, float c) {
+    float m = warp_max(t.m);
+    int idx = warp_min_int(t.m == m ? t.idx : kIntMax);
+    rescale_to<kMode>(t, m, c);
+    Partial r;
+    r.m = m; r.idx = idx;
+    r.Z = kMode >= 1 ? warp_sum(t.Z) : 0.f;
+    r.A = kMode == 2 ? warp_sum(t.A) : 0.f;
+    return r;
+}
+
+// Inclusive warp scan.
+__device__ __forceinline__ float warp_scan_incl(float v, int lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        float n = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += n;
+    }
+    return v;
+}
+
+// Block-wide exclusive scan of one float per thread; also returns the block total.
+// `wsum` is shared scratch of kWarps floats.  Contains two __syncthreads().
+__device__ __forceinline__ float block_scan_excl(float v, float* wsum, int lane, int warp, float& total) {
+    float inc = warp_scan_incl(v, lane);
+    __syncthreads();   // wsum may still be read from the previous round
+    if (lane == 31) wsum[warp] = inc;
+    __syncthreads();
+    float before = 0.f, tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+        float s = wsum[w];
+        if (w < warp) before += s;
+        tot += s;
+    }
+    total = tot;
+    return before + (inc - v);
+}
+
+// ---------------------------------------------------------------------------
+// Locating a sample among the segments of a row.
+//
+// Each block of the cluster publishes, per warp, the mass of its segment in
+// shared memory.  Warp 0 of EVERY block then reads all segments of the cluster
+// through distributed shared memory, in the same order with the same
+// arithmetic, so all blocks agree bit for bit on the total, on the target mass
+// u * total and on the segment that holds it; the block that owns the segment
+// does the fine scan.
+
+struct SegPick {
+    float total;    // sum of all segment masses = last inclusive prefix
+    int seg;        // selected segment
+    float prefix;   // exclusive prefix of the selected segment
+    float target;   // u * total
+};
+
+// `mass[k]` is the mass of segment lane*per + k (0 beyond nseg).  Warp-collective.
+__device__ __forceinline__ SegPick pick_segment(const float (&mass)[kSegPerLane], int per, int nseg,
+                                                float u, int lane) {
+    float run[kSegPerLane];
+    float acc = 0.f;
+#pragma unroll
+    for (int k = 0; k < kSegPerLane; ++k) {
+        if (k < per) acc += mass[k];
+        run[k] = acc;                       // inclusive within the lane
+    }
+    float incl = warp_scan_incl(acc, lane);
+    float before = incl - acc;
+    SegPick r;
+    r.total = __shfl_sync(0xffffffffu, incl, 31);
+    r.target = u * r.total;
+    int cand = kIntMax;
+    float cpre = 0.f;
+#pragma unroll
+    for (int k = kSegPerLane - 1; k >= 0; --k) {
+        if (k < per && lane * per + k < nseg && before + run[k] > r.target) {
+            cand = lane * per + k;
+            cpre = before + (run[k] - mass[k]);
+        }
+    }
+    int best = warp_min_int(cand);
+    if (best == kIntMax) {
+        // rounding left no prefix above the target: take the last segment with mass
+        int lastpos = -1;
+        float lpre = 0.f;
+#pragma unroll
+        for (int k = 0; k < kSegPerLane; ++k) {
+            if (k < per && lane * per + k < nseg && mass[k] > 0.f) {
+                lastpos = lane * per + k;
+                lpre = before + (run[k] - mass[k]);
+            }
+        }
+        int hi = -warp_min_int(-lastpos);
+        best = hi < 0 ? 0 : hi;
+        cand = (lastpos == best) ? best : kIntMax;
+        cpre = lpre;
+    }
+    unsigned who = __ballot_sync(0xffffffffu, cand == best);
+    int src = who ? __ffs(who) - 1 : 0;
+    r.seg = best;
+    r.prefix = __shfl_sync(0xffffffffu, cpre, src);
+    return r;
+}
+
+// Shared scratch of the fine scan.
+struct ScanShared {
+    float wsum[kWarps];
+    int hit;       // lowest virtual element index whose cumulative mass exceeds the target
+    int lastpos;   // highest virtual element index with positive weight
+};
+
+}  // namespace svip
