@@ -1,0 +1,208 @@
+"""GPU parity of svip_verify and svip_pack_ragged (through the C ABI) against the fp64 oracle."""
+import numpy as np
+import pytest
+
+import svip_testlib as tl
+from paper_2411_18462_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2411_18462_b200 import Context, build
+    build.build()
+    c = Context(0, 1 << 14)
+    yield c
+    c.destroy()
+
+
+def small_case(rng, B, V, K_max, bf16, noise=0.5, ragged=True):
+    lens = rng.integers(1, K_max + 1, size=B).astype(np.int32) if ragged else np.full(B, K_max, np.int32)
+    cu = np.concatenate([[0], np.cumsum(lens + 1)]).astype(np.int64)
+    Rp = int(cu[-1]); Rq = Rp - B
+    scale = np.exp(rng.uniform(np.log(0.3), np.log(6.0), size=(Rp, 1)))
+    base = (rng.standard_normal((Rp, V)) * scale).astype(np.float32)
+    tgt = base + (rng.standard_normal((Rp, V)) * noise).astype(np.float32)
+    q = np.empty((Rq, V), np.float32)
+    for i in range(B):
+        q[cu[i] - i: cu[i] - i + lens[i]] = base[cu[i]: cu[i] + lens[i]]
+    if bf16:
+        q = W.to_bf16_bits(q); tgt = W.to_bf16_bits(tgt)
+    return lens, cu, q, tgt, rng.random(Rq).astype(np.float32), rng.random(Rp).astype(np.float32)
+
+
+def run_case(ctx, oracle, lens, cu, q, tgt, ud, uv, T, K_max, label, with_stats=True, fixed=False):
+    tok, _, _ = oracle.draft_step(q, T, 0.3, ud, threads=8)
+    tok = tok.astype(np.int32)
+    uv, moved = tl.guard_accept_uniforms(oracle, tok, q, tgt, cu, T, uv)
+    stats = None
+    if with_stats and T > 0:
+        stats = tl.gpu_draft_step(ctx, q, T, 0.3, ud)[3]
+    got = tl.gpu_verify(ctx, tok, q, tgt, cu, K_max, T, uv if T > 0 else None, q_stats=stats, fixed_K=fixed)
+    return tl.check_verify_against_oracle(oracle, tok, q, tgt, cu, T, uv, got, label)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("V", [2, 8, 33, 1000, 4099, 32000])
+def test_small_ragged_all_cluster_sizes(ctx, oracle, V, bf16):
+    rng = np.random.default_rng(4000 + V + int(bf16))
+    lens, cu, q, tgt, ud, uv = small_case(rng, 6, V, 5, bf16)
+    for T in (1.0, 0.7, 0.0):
+        for S in (1, 2, 4, 8, 0):
+            ctx.set_cluster_size(S)
+            run_case(ctx, oracle, lens, cu, q, tgt, ud, uv, T, 5, "V=%d S=%d T=%g" % (V, S, T),
+                     with_stats=(S % 2 == 0))
+    ctx.set_cluster_size(0)
+    assert ctx.read_status() == 0
+
+
+def test_fixed_k_and_long_drafts(ctx, oracle):
+    rng = np.random.default_rng(9)
+    for K in (1, 3, 40, 64, 70):
+        lens, cu, q, tgt, ud, uv = small_case(rng, 3, 300, K, False, noise=0.15, ragged=False)
+        for T in (1.0, 0.0):
+            c = run_case(ctx, oracle, lens, cu, q, tgt, ud, uv, T, K, "K=%d T=%g" % (K, T), fixed=True)
+    assert ctx.read_status() == 0
+
+
+def test_all_accept_gives_bonus_and_reject_at_zero(ctx, oracle):
+    rng = np.random.default_rng(10)
+    lens, cu, q, tgt, ud, uv = small_case(rng, 4, 2000, 6, True)
+    # target == draft on every draft position: every token accepted for any uniform
+    for i in range(4):
+        tgt[cu[i]: cu[i] + lens[i]] = q[cu[i] - i: cu[i] - i + lens[i]]
+    tok, _, _ = oracle.draft_step(q, 1.0, 0.3, ud)
+    uv2 = uv.copy(); uv2[:] = 1.0 - 2.0 ** -24
+    got = tl.gpu_verify(ctx, tok.astype(np.int32), q, tgt, cu, 6, 1.0, uv2)
+    assert np.array_equal(got[0], lens)
+    tl.check_verify_against_oracle(oracle, tok.astype(np.int32), q, tgt, cu, 1.0, uv2, got, "all-accept")
+    # p(x) = 0 at the first draft token: rejected at position 0 whatever the uniform
+    tgt2 = W.bf16_bits_to_f32(tgt).copy()
+    for i in range(4):
+        tgt2[cu[i], tok[cu[i] - i]] = -np.inf
+    tgt2 = W.to_bf16_bits(tgt2)
+    uv3 = uv.copy(); uv3[cu[:-1]] = 0.0
+    got = tl.gpu_verify(ctx, tok.astype(np.int32), q, tgt2, cu, 6, 1.0, uv3)
+    assert np.all(got[0] == 0)
+    tl.check_verify_against_oracle(oracle, tok.astype(np.int32), q, tgt2, cu, 1.0, uv3, got, "reject-at-0")
+
+
+def test_position_major_draft_layout(ctx, oracle):
+    """Draft-side arrays laid out [K_max, B] (one logits buffer per draft step) via the two strides."""
+    rng = np.random.default_rng(12)
+    B, V, K = 5, 777, 4
+    lens, cu, q, tgt, ud, uv = small_case(rng, B, V, K, True)
+    tok, _, _ = oracle.draft_step(q, 1.0, 0.3, ud)
+    q_pm = np.zeros((K * B, V), np.uint16); tok_pm = np.zeros(K * B, np.int32)
+    for i in range(B):
+        for j in range(lens[i]):
+            q_pm[j * B + i] = q[cu[i] - i + j]; tok_pm[j * B + i] = tok[cu[i] - i + j]
+    uv, _ = tl.guard_accept_uniforms(oracle, tok.astype(np.int32), q, tgt, cu, 1.0, uv)
+    got = tl.gpu_verify(ctx, tok_pm, q_pm, tgt, cu, K, 1.0, uv, layout="strided", q_seq_stride=1, q_pos_stride=B)
+    tl.check_verify_against_oracle(oracle, tok.astype(np.int32), q, tgt, cu, 1.0, uv, got, "position-major")
+
+
+def test_pack_ragged(ctx, oracle):
+    import torch
+    rng = np.random.default_rng(3)
+    for B, K_max in ((1, 1), (7, 64), (128, 64), (1500, 9), (65536, 2)):
+        lens = rng.integers(1, K_max + 1, size=B).astype(np.int32)
+        cu_o, seq_o, pos_o = oracle.pack_ragged(lens)
+        d = torch.from_numpy(lens).cuda()
+        cu = torch.zeros(B + 1, dtype=torch.int32, device="cuda")
+        seq = torch.full((B * (K_max + 1),), -1, dtype=torch.int32, device="cuda")
+        pos = torch.full((B * (K_max + 1),), -1, dtype=torch.int32, device="cuda")
+        ctx.pack_ragged(d, B, K_max, cu, seq, pos)
+        torch.cuda.synchronize()
+        R = int(cu_o[-1])
+        assert np.array_equal(cu.cpu().numpy(), cu_o)
+        assert np.array_equal(seq.cpu().numpy()[:R], seq_o) and np.array_equal(pos.cpu().numpy()[:R], pos_o)
+        assert np.all(seq.cpu().numpy()[R:] == -1)
+    assert ctx.read_status() == 0
+    bad = torch.tensor([3, 0, 99, 2], dtype=torch.int32, device="cuda")
+    cu = torch.zeros(5, dtype=torch.int32, device="cuda")
+    ctx.pack_ragged(bad, 4, 8, cu)
+    assert ctx.read_status() == 2
+    assert cu.cpu().tolist() == [0, 4, 6, 15, 18]
+
+
+def test_workspace_limit_and_bad_arguments():
+    import torch
+    from paper_2411_18462_b200 import Context, SvipError
+    c = Context(0, 8)
+    t = torch.zeros(64, device="cuda"); i = torch.zeros(64, dtype=torch.int32, device="cuda")
+    with pytest.raises(SvipError) as e:
+        c.verify(i, t, 4, None, -1, 0, t, 4, 0, None, 3, 2, 9, 4, 1.0, t, i, i)
+    assert e.value.code == -3
+    with pytest.raises(SvipError):   # fixed K needs exactly B*(K+1) rows
+        c.verify(i, t, 4, None, -1, 0, t, 4, 0, None, 2, 2, 5, 4, 1.0, t, i, i)
+    with pytest.raises(SvipError):   # sampling needs uniforms
+        c.verify(i, t, 4, None, -1, 0, t, 4, 0, None, 2, 2, 6, 4, 1.0, None, i, i)
+    c.destroy()
+
+
+def test_graph_replay_matches_direct_calls(ctx, oracle):
+    """B = 1: eight draft steps, packing and the verify round recorded once, replayed on new inputs."""
+    import torch
+    w = W.make_workload("tiny")
+    K, V = w.K_max, w.V
+    dq = tl.to_device(w.q_logits); dt = tl.to_device(w.target_logits)
+    ud = tl.to_device(w.draft_uniforms); uv = tl.to_device(w.verify_uniforms)
+    tok = torch.zeros(K, dtype=torch.int32, device="cuda"); ent = torch.zeros(K, device="cuda")
+    stop = torch.zeros(K, dtype=torch.uint8, device="cuda"); stats = torch.zeros(K, 2, device="cuda")
+    lens = torch.tensor([K], dtype=torch.int32, device="cuda"); cu = torch.zeros(2, dtype=torch.int32, device="cuda")
+    nacc = torch.zeros(1, dtype=torch.int32, device="cuda"); nxt = torch.zeros(1, dtype=torch.int32, device="cuda")
+    st = torch.cuda.Stream()
+
+    def enqueue():
+        for j in range(K):
+            ctx.draft_step(dq.data_ptr() + j * V * 4, 0, 1, V, V, 1.0, w.h, ud.data_ptr() + 4 * j,
+                           tok.data_ptr() + 4 * j, ent.data_ptr() + 4 * j, stop.data_ptr() + j,
+                           stats.data_ptr() + 8 * j, st)
+        ctx.pack_ragged(lens, 1, K, cu, None, None, st)
+        ctx.verify(tok, dq, V, stats, -1, 0, dt, V, 0, cu, 1, K, K + 1, V, 1.0, uv, nacc, nxt, st)
+
+    enqueue(); st.synchronize()
+    direct = (tok.cpu().numpy().copy(), nacc.item(), nxt.item())
+    ctx.graph_begin(st); enqueue(); g = ctx.graph_end(st)
+    # new inputs in place: target := draft (all accepted), replay must see them
+    dt[:K].copy_(dq)
+    g.launch(st); st.synchronize()
+    assert nacc.item() == K
+    dt.copy_(tl.to_device(w.target_logits))
+    tok.zero_(); nacc.zero_(); nxt.zero_()
+    g.launch(st); st.synchronize()
+    assert np.array_equal(tok.cpu().numpy(), direct[0]) and (nacc.item(), nxt.item()) == direct[1:]
+    g.destroy()
+    tok_o, _, _ = oracle.draft_step(w.q_logits, 1.0, w.h, w.draft_uniforms)
+    assert np.array_equal(direct[0], tok_o)
+
+
+@pytest.mark.parametrize("name", ["tiny", "chat", "reasoning", "ragged", "stress"])
+def test_published_configs(ctx, oracle, name):
+    """Each published configuration at full size, automatic launch shape, q_stats from the draft step."""
+    w = W.make_workload(name)
+    temps = {"tiny": (1.0, 0.0), "chat": (1.0, 0.0), "reasoning": (0.7,), "ragged": (1.0,), "stress": (1.0, 0.0)}[name]
+    fixed = name != "ragged"
+    for T in temps:
+        tok, _, _ = oracle.draft_step(w.q_logits, T, w.h, w.draft_uniforms, threads=16)
+        tok = tok.astype(np.int32)
+        uv, moved = tl.guard_accept_uniforms(oracle, tok, w.q_logits, w.target_logits, w.cu_rows, T,
+                                             w.verify_uniforms, threads=16)
+        stats = tl.gpu_draft_step(ctx, w.q_logits, T, w.h, w.draft_uniforms)[3] if T > 0 else None
+        got = tl.gpu_verify(ctx, tok, w.q_logits, w.target_logits, w.cu_rows, w.K_max, T,
+                            uv if T > 0 else None, q_stats=stats, fixed_K=fixed)
+        c = tl.check_verify_against_oracle(oracle, tok, w.q_logits, w.target_logits, w.cu_rows, T, uv, got,
+                                           "%s T=%g" % (name, T), threads=16)
+        print("verify parity", name, "T=%g" % T, c, "uniforms moved off the accept boundary:", moved)
+        assert c["next_boundary"] <= max(1, c["sequences"] // 50)
+    if name == "tiny":   # target := draft everywhere: all K accepted, bonus token from row K
+        t2 = w.target_logits.copy(); t2[:w.K_max] = w.q_logits
+        tok, _, _ = oracle.draft_step(w.q_logits, 1.0, w.h, w.draft_uniforms)
+        got = tl.gpu_verify(ctx, tok.astype(np.int32), w.q_logits, t2, w.cu_rows, w.K_max, 1.0, w.verify_uniforms,
+                            fixed_K=True)
+        assert got[0][0] == w.K_max
+        tl.check_verify_against_oracle(oracle, tok.astype(np.int32), w.q_logits, t2, w.cu_rows, 1.0,
+                                       w.verify_uniforms, got, "tiny all-accept")
+    assert ctx.read_status() == 0
