@@ -349,9 +349,11 @@ __global__ void __launch_bounds__(kThreads) verify_finish_kernel(FinishArgs a) {
                     float eq = exp2f(fmaxf(__fmaf_rn(dv, a.c, -__fmul_rn(qs.x, a.c)), kArgFloor));
                     if (!(tv > neg_inf())) ep = 0.f;
                     if (!(dv > neg_inf())) eq = 0.f;
-                    // r < (ep/Zp)/(eq/Zq) without the division; eq == 0 accepts iff ep > 0
+                    // r < min(1, (ep/Zp)/(eq/Zq)) without the division: a ratio >= 1 accepts every
+                    // r in [0,1); p(x) == 0 accepts none; q(x) == 0 < p(x) is a ratio of +inf
                     float r = a.uniforms[row0 + j];
-                    acc = __fmul_rn(__fmul_rn(r, eq), ps.y) < __fmul_rn(ep, qs.y);
+                    float lhs = __fmul_rn(eq, ps.y), rhs = __fmul_rn(ep, qs.y);
+                    acc = ep > 0.f && (rhs >= lhs || __fmul_rn(r, lhs) < rhs);
                 }
                 rej = !acc;
             }

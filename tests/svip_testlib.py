@@ -4,8 +4,9 @@ boundary predicates of the stated tolerances.
 Tolerances (the numbers every parity test uses):
   ENTROPY_ATOL    entropy agrees within 1e-4 nats (fp32 accumulation against the fp64 oracle)
   CDF_TOL         a sampled token may differ from the oracle's only if the uniform lies within 1e-5
-                  (in units of the total weight) of a boundary of the oracle's CDF; such cases are
-                  counted and reported
+                  (in units of the total weight) of that token's own interval of the oracle's fp64
+                  CDF, i.e. only across a CDF boundary closer than 1e-5; such cases are counted
+                  and reported (flat tails of a 256000-token row have boundaries every ~1e-7)
   ACCEPT_GUARD    accept draws closer than 1e-4 to the oracle's acceptance probability are moved
                   away before both sides see them, so accept counts must then be bit-exact
   STOP_GUARD      stop flags must be bit-exact wherever |sqrt(H) - h| > 1e-3 (oracle value)
@@ -116,13 +117,17 @@ def guard_accept_uniforms(oracle, draft_tokens, q_logits, target_logits, cu_rows
     return u, moved
 
 
-def near_cdf_boundary(weights: np.ndarray, u: float, tol: float = CDF_TOL) -> bool:
-    """True if u * total lies within tol * total of some cumulative sum of `weights` (fp64)."""
+def within_cdf_tolerance(weights: np.ndarray, u: float, token: int, tol: float = CDF_TOL) -> bool:
+    """True if `token` is what the inverse CDF returns for some u' with |u' - u| <= tol, i.e. if
+    u * total lies within tol * total of the token's own interval [c_{token-1}, c_token) of the fp64
+    cumulative sums, and the token has positive weight."""
     c = np.cumsum(weights.astype(np.float64))
     total = c[-1]
-    if not total > 0:
-        return True
-    return bool(np.min(np.abs(c / total - float(u))) <= tol)
+    if not total > 0 or not (0 <= token < len(c)) or not weights[token] > 0:
+        return False
+    lo = (c[token - 1] if token > 0 else 0.0) / total
+    hi = c[token] / total
+    return bool(lo - tol <= float(u) <= hi + tol)
 
 
 def check_draft_against_oracle(oracle, logits, T, h, uniforms, got, label="", threads=8):
@@ -141,9 +146,8 @@ def check_draft_against_oracle(oracle, logits, T, h, uniforms, got, label="", th
         return counters
     for b in bad:
         q = oracle.softmax(logits[b], T)
-        assert near_cdf_boundary(q, uniforms[b]), "%s row %d: token %d vs oracle %d, off any CDF boundary" % (
-            label, b, tok_g[b], tok_o[b])
-        assert abs(int(tok_g[b]) - int(tok_o[b])) >= 1
+        assert within_cdf_tolerance(q, uniforms[b], int(tok_g[b])), \
+            "%s row %d: token %d vs oracle %d, beyond the CDF tolerance" % (label, b, tok_g[b], tok_o[b])
         counters["token_boundary"] += 1
     return counters
 
@@ -172,7 +176,7 @@ def check_verify_against_oracle(oracle, draft_tokens, q_logits, target_logits, c
                 w = p
         else:
             w = p
-        assert near_cdf_boundary(w, uniforms[r0 + K]), "%s seq %d: next %d vs oracle %d off any CDF boundary" % (
-            label, i, nx_g[i], nx_o[i])
+        assert within_cdf_tolerance(w, uniforms[r0 + K], int(nx_g[i])), \
+            "%s seq %d: next %d vs oracle %d, beyond the CDF tolerance" % (label, i, nx_g[i], nx_o[i])
         counters["next_boundary"] += 1
     return counters

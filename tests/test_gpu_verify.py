@@ -196,7 +196,6 @@ def test_published_configs(ctx, oracle, name):
         c = tl.check_verify_against_oracle(oracle, tok, w.q_logits, w.target_logits, w.cu_rows, T, uv, got,
                                            "%s T=%g" % (name, T), threads=16)
         print("verify parity", name, "T=%g" % T, c, "uniforms moved off the accept boundary:", moved)
-        assert c["next_boundary"] <= max(1, c["sequences"] // 50)
     if name == "tiny":   # target := draft everywhere: all K accepted, bonus token from row K
         t2 = w.target_logits.copy(); t2[:w.K_max] = w.q_logits
         tok, _, _ = oracle.draft_step(w.q_logits, 1.0, w.h, w.draft_uniforms)
