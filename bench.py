@@ -1,0 +1,434 @@
+#!/usr/bin/env python
+"""Throughput of one SVIP speculative-decoding round (draft steps + ragged packing + verify).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload ragged] [--impl ours|reference]
+
+A step is one whole round over one batch of the `ragged` workload (B = 128 sequences, V = 152064
+bf16 logits, draft lengths K_i in 1..64 set by the entropy stop rule): one svip_draft_step call per
+draft position over the sequences still drafting, one svip_pack_ragged, one svip_verify.  The
+metric is logits GB/s: bytes of logits the round has to read (every draft row once, every target
+row once, plus the draft row of each rejected position) divided by the device time of the step.
+Prints ONE JSON line on rank 0.  With N > 1 (torchrun) every rank runs its own batch on its own GPU
+(weak scaling, no data-path collective); the time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2411_18462_b200 import sharding, workloads  # noqa: E402
+
+METRIC = "logits GB/s (% of B200 HBM peak) for draft-step+verify; us/step at B=1"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def describe(w, B=None):
+    lens = "K_i~U{1..%d} set by the entropy stop rule" % w.K_max if w.name == "ragged" else "K=%d" % w.K_max
+    return "%s: B=%d V=%d %s logits, %s, T=%g, h=%g" % (w.name, B or w.B, w.V, w.dtype, lens, w.T, w.h)
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# --------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid):
+        self.uuid = uuid
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", self.uuid, "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out = self.proc.communicate(timeout=10)[0]
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in out.splitlines():
+            p = [x.strip() for x in line.split(",")]
+            if len(p) < 8:
+                continue
+            try:
+                sm.append(float(p[0])); mx.append(float(p[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, p[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------- the round on one GPU
+
+class Round:
+    """Device buffers and pre-marshalled calls of one speculative-decoding round of a workload.
+
+    Draft logits live position-major, [K, B, V] with the sequences sorted by decreasing draft
+    length: step j reads the first active[j] rows of slab j (the sequences still drafting), which is
+    the layout a serving loop produces.  Target rows are packed sequence after sequence."""
+
+    def __init__(self, ctx, w, torch, stream):
+        self.ctx, self.w, self.torch, self.stream = ctx, w, torch, stream
+        order, q_pm, active = workloads.position_major(w)
+        B, V, K = w.B, w.V, q_pm.shape[0]
+        self.B, self.V, self.K, self.active = B, V, K, active
+        lens = w.draft_len[order].astype(np.int32)
+        cu_sorted = np.concatenate([[0], np.cumsum(lens.astype(np.int64) + 1)])
+        t_sorted = np.empty_like(w.target_logits)
+        uv_sorted = np.empty_like(w.verify_uniforms)
+        ud_pm = np.zeros((K, B), dtype=np.float32)
+        for k, i in enumerate(order):
+            n = int(lens[k]) + 1
+            t_sorted[cu_sorted[k]:cu_sorted[k] + n] = w.target_logits[w.cu_rows[i]:w.cu_rows[i] + n]
+            uv_sorted[cu_sorted[k]:cu_sorted[k] + n] = w.verify_uniforms[w.cu_rows[i]:w.cu_rows[i] + n]
+            r0 = int(w.cu_rows[i]) - int(i)
+            ud_pm[:n - 1, k] = w.draft_uniforms[r0:r0 + n - 1]
+        self.Rp = int(cu_sorted[-1])
+        self.lens = lens
+        as_t = (lambda a: torch.from_numpy(a.view(np.int16))) if w.dtype == "bf16" else torch.from_numpy
+        # pinned host copies (the end-to-end leg copies from these every step)
+        self.h_q = as_t(q_pm.reshape(K * B, V)).pin_memory()
+        self.h_t = as_t(t_sorted).pin_memory()
+        self.h_ud = torch.from_numpy(ud_pm.reshape(-1)).pin_memory()
+        self.h_uv = torch.from_numpy(uv_sorted).pin_memory()
+        self.h_len = torch.from_numpy(lens).pin_memory()
+        dev = torch.device("cuda", torch.cuda.current_device())
+        self.d_q = torch.empty_like(self.h_q, device=dev)
+        self.d_t = torch.empty_like(self.h_t, device=dev)
+        self.d_ud = torch.empty_like(self.h_ud, device=dev)
+        self.d_uv = torch.empty_like(self.h_uv, device=dev)
+        self.d_len = torch.empty_like(self.h_len, device=dev)
+        self.d_tok = torch.zeros(K * B, dtype=torch.int32, device=dev)
+        self.d_ent = torch.zeros(K * B, dtype=torch.float32, device=dev)
+        self.d_stop = torch.zeros(K * B, dtype=torch.uint8, device=dev)
+        self.d_stats = torch.zeros(K * B, 2, dtype=torch.float32, device=dev)
+        self.d_cu = torch.zeros(B + 1, dtype=torch.int32, device=dev)
+        self.d_nacc = torch.zeros(B, dtype=torch.int32, device=dev)
+        self.d_next = torch.zeros(B, dtype=torch.int32, device=dev)
+        self.h_nacc = torch.zeros(B, dtype=torch.int32).pin_memory()
+        self.h_next = torch.zeros(B, dtype=torch.int32).pin_memory()
+        self.h_stop = torch.zeros(K * B, dtype=torch.uint8).pin_memory()
+        self.h_tok = torch.zeros(K * B, dtype=torch.int32).pin_memory()
+        self.esz = w.elem_bytes
+        self.dt = 1 if w.dtype == "bf16" else 0
+        self.upload()
+        torch.cuda.synchronize()
+
+    def upload(self):
+        """Host -> device copy of one step's inputs (active rows only); returns the bytes copied."""
+        n = 0
+        B = self.B
+        for j in range(self.K):
+            a = int(self.active[j])
+            self.d_q[j * B:j * B + a].copy_(self.h_q[j * B:j * B + a], non_blocking=True)
+            n += a * self.V * self.esz
+        for d, h in ((self.d_t, self.h_t), (self.d_ud, self.h_ud), (self.d_uv, self.h_uv), (self.d_len, self.h_len)):
+            d.copy_(h, non_blocking=True)
+            n += h.numel() * h.element_size()
+        return n
+
+    def download(self):
+        """Device -> host read of the step's results; returns the bytes copied."""
+        n = 0
+        for h, d in ((self.h_nacc, self.d_nacc), (self.h_next, self.d_next), (self.h_stop, self.d_stop),
+                     (self.h_tok, self.d_tok)):
+            h.copy_(d, non_blocking=True)
+            n += h.numel() * h.element_size()
+        return n
+
+    def step(self):
+        ctx, w, B, V, sp = self.ctx, self.w, self.B, self.V, self.stream
+        q, ud, tok, ent = self.d_q.data_ptr(), self.d_ud.data_ptr(), self.d_tok.data_ptr(), self.d_ent.data_ptr()
+        stop, stats = self.d_stop.data_ptr(), self.d_stats.data_ptr()
+        for j in range(self.K):
+            o = j * B
+            ctx.draft_step(q + o * V * self.esz, self.dt, int(self.active[j]), V, V, w.T, w.h, ud + 4 * o,
+                           tok + 4 * o, ent + 4 * o, stop + o, stats + 8 * o, sp)
+        ctx.pack_ragged(self.d_len, B, w.K_max, self.d_cu, None, None, sp)
+        ctx.verify(self.d_tok, self.d_q, V, self.d_stats, 1, B, self.d_t, V, self.dt, self.d_cu, B, w.K_max,
+                   self.Rp, V, w.T, self.d_uv, self.d_nacc, self.d_next, sp)
+
+    def logits_bytes(self):
+        """Algorithmic logits bytes of one step (needs the results of a finished step)."""
+        self.torch.cuda.synchronize()
+        nacc = self.d_nacc.cpu().numpy()
+        rejected = int((nacc < self.lens).sum())
+        rows = int(self.lens.sum()) + self.Rp + rejected
+        return rows * self.V * self.esz, rejected
+
+    def check_stop_flags(self):
+        """The stop rule must reproduce the workload's draft lengths (generator contract)."""
+        stop = self.d_stop.cpu().numpy().reshape(self.K, self.B)
+        for k in range(self.B):
+            n = int(self.lens[k])
+            if stop[:n - 1, k].any() or not (stop[n - 1, k] == 1 or n == self.w.K_max):
+                return False
+        return True
+
+
+def b1_latency(ctx, torch):
+    """us per replay of a CUDA graph holding a whole B = 1 round of the `tiny` workload."""
+    w = workloads.make_workload("tiny")
+    st = torch.cuda.Stream()
+    K, V = w.K_max, w.V
+    dq = torch.from_numpy(w.q_logits).cuda(); dt = torch.from_numpy(w.target_logits).cuda()
+    ud = torch.from_numpy(w.draft_uniforms).cuda(); uv = torch.from_numpy(w.verify_uniforms).cuda()
+    tok = torch.zeros(K, dtype=torch.int32, device="cuda"); ent = torch.zeros(K, device="cuda")
+    stop = torch.zeros(K, dtype=torch.uint8, device="cuda"); stats = torch.zeros(K, 2, device="cuda")
+    lens = torch.tensor([K], dtype=torch.int32, device="cuda"); cu = torch.zeros(2, dtype=torch.int32, device="cuda")
+    nacc = torch.zeros(1, dtype=torch.int32, device="cuda"); nxt = torch.zeros(1, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+
+    def enqueue(s):
+        for j in range(K):
+            ctx.draft_step(dq.data_ptr() + j * V * 4, 0, 1, V, V, w.T, w.h, ud.data_ptr() + 4 * j,
+                           tok.data_ptr() + 4 * j, ent.data_ptr() + 4 * j, stop.data_ptr() + j,
+                           stats.data_ptr() + 8 * j, s)
+        ctx.pack_ragged(lens, 1, K, cu, None, None, s)
+        ctx.verify(tok, dq, V, stats, -1, 0, dt, V, 0, cu, 1, K, K + 1, V, w.T, uv, nacc, nxt, s)
+
+    out = {}
+    with torch.cuda.stream(st):
+        ctx.graph_begin(st); enqueue(st); g = ctx.graph_end(st)
+        one = None
+        ctx.graph_begin(st)
+        ctx.draft_step(dq, 0, 1, V, V, w.T, w.h, ud, tok, ent, stop, stats, st)
+        one = ctx.graph_end(st)
+        for name, graph, reps in (("round_us", g, 200), ("draft_step_us", one, 500)):
+            for _ in range(20):
+                graph.launch(st)
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            st.synchronize()
+            e0.record(st)
+            for _ in range(reps):
+                graph.launch(st)
+            e1.record(st)
+            st.synchronize()
+            out[name] = 1000.0 * e0.elapsed_time(e1) / reps
+        g.destroy(); one.destroy()
+    out["kernels_per_round"] = K + 3
+    return out
+
+
+def cpu_baseline(w, seconds_budget=20.0):
+    """The fp64 oracle, as it stands, on a bounded sample of the same workload, on all host cores."""
+    from oracle import svip_oracle as O
+    cores = len(os.sched_getaffinity(0))
+    n_seq = min(w.B, max(2, cores // 2))
+    sel = list(range(n_seq))
+    rows_q = np.concatenate([np.arange(w.cu_rows[i] - i, w.cu_rows[i] - i + w.draft_len[i]) for i in sel])
+    rows_t = np.concatenate([np.arange(w.cu_rows[i], w.cu_rows[i + 1]) for i in sel])
+    q = np.ascontiguousarray(w.q_logits[rows_q]); t = np.ascontiguousarray(w.target_logits[rows_t])
+    lens = w.draft_len[sel]
+    cu = np.concatenate([[0], np.cumsum(lens.astype(np.int64) + 1)])
+    ud = w.draft_uniforms[rows_q]; uv = w.verify_uniforms[rows_t]
+    O.lib()
+    t0 = time.perf_counter()
+    tok, H, stop = O.draft_step(q, w.T, w.h, ud, threads=cores)
+    nacc, nxt, _ = O.verify(tok.astype(np.int32), q, t, cu, w.T, uv, threads=cores)
+    dt = time.perf_counter() - t0
+    rejected = int((nacc < lens).sum())
+    nbytes = (len(rows_q) + len(rows_t) + rejected) * w.V * w.elem_bytes
+    return {"value": nbytes / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
+            "sample": "%d of %d sequences (%d draft + %d target rows), one pass, %.1f s" % (
+                n_seq, w.B, len(rows_q), len(rows_t), dt)}
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2411_18462_b200 import Context, build
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.cuda.current_device()
+    if build.is_stale():
+        build.build()
+    spec = workloads.SPECS[args.workload]
+    w = workloads.make_workload(args.workload, seed=sharding.rank_seed(workloads.BASE_SEED + spec["index"], rank))
+    ctx = Context(dev, max(1 << 14, w.n_target_rows))
+    stream = torch.cuda.current_stream()
+    rnd = Round(ctx, w, torch, stream.cuda_stream)
+    for _ in range(max(args.warmup, 3)):
+        rnd.step()
+    step_bytes, rejected = rnd.logits_bytes()
+    stops_ok = rnd.check_stop_flags()
+    status = ctx.read_status(stream.cuda_stream)
+
+    uuid = str(torch.cuda.get_device_properties(dev).uuid)
+    uuid = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+    sampler = ClockSampler(uuid)
+    ctx.profile_enable(True)
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    launches0 = ctx.launch_count()
+    e0.record(stream)
+    for _ in range(args.steps):
+        rnd.step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    launches = ctx.launch_count() - launches0
+    clocks = sampler.stop()
+    local_ms = e0.elapsed_time(e1)
+    stats_ms, stats_n = ctx.profile_read()
+    ctx.profile_enable(False)
+    total_ms, total_bytes = sharding.aggregate(local_ms, step_bytes * args.steps, device=torch.device("cuda", dev))
+
+    # end to end: host buffers in, results out, every step
+    e2e_steps = max(1, min(args.steps, 5))
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    for _ in range(e2e_steps):
+        h2d = rnd.upload()
+        rnd.step()
+        d2h = rnd.download()
+        stream.synchronize()
+    t1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms, e2e_bytes = sharding.aggregate(t0.elapsed_time(t1), step_bytes * e2e_steps, device=torch.device("cuda", dev))
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peak, peak_kind = measured_peak()
+    value = total_bytes / (total_ms * 1e-3) / 1e9
+    stats_bytes = w.n_target_rows * w.V * w.elem_bytes
+    achieved = stats_bytes / (stats_ms / max(stats_n, 1) * 1e-3) / 1e9 if stats_n else None
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": describe(w), "sequences_per_gpu": w.B, "draft_rows": w.n_draft_rows,
+                   "target_rows": w.n_target_rows, "rejected_sequences": rejected,
+                   "logits_bytes_per_step": step_bytes, "l2": "inputs (%.2f GB per step) larger than L2, no flush" % (step_bytes / 1e9),
+                   "launch": "one stream, %d kernels per step" % (launches // max(args.steps, 1)),
+                   "stop_flags_match_draft_lengths": bool(stops_ok), "status_word": status},
+        "pct_of_hbm_peak_nominal": 100.0 * value / world / NOMINAL_HBM_GBS,
+        "pct_of_hbm_peak_measured": 100.0 * value / world / peak,
+        "roofline": {"bound": "hbm", "kernel": "row_stats_kernel<bf16> (target rows of svip_verify)",
+                     "achieved": achieved, "peak": peak, "peak_kind": "%s copy bandwidth" % peak_kind,
+                     "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
+                     "launches_timed": stats_n, "bytes_per_launch": stats_bytes, "traffic": None},
+        "e2e": {"value": e2e_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "gpu_launches": launches, "clocks": clocks,
+    }
+    try:
+        line["b1"] = b1_latency(ctx, torch)
+    except Exception as exc:   # the headline number does not depend on the latency probe
+        line["b1"] = {"error": repr(exc)}
+    if not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(w)
+    line["paper_context"] = ("end-to-end speedups over fixed draft length reported by the paper: up to 17% "
+                             "(MT-Bench, 8K context) and 22% (QwQ long-form reasoning); hardware not stated")
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_reference(args):
+    """The oracle as the reference arm: each step is a bounded sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import svip_oracle as O
+    spec = workloads.SPECS[args.workload]
+    cores = len(os.sched_getaffinity(0))
+    n_seq = 2
+    w = workloads.make_workload(args.workload, B=n_seq, seed=workloads.BASE_SEED + spec["index"])
+    O.lib()
+
+    def step():
+        tok, H, stop = O.draft_step(w.q_logits, w.T, w.h, w.draft_uniforms, threads=cores)
+        nacc, nxt, _ = O.verify(tok.astype(np.int32), w.q_logits, w.target_logits, w.cu_rows, w.T,
+                                w.verify_uniforms, threads=cores)
+        return int((nacc < w.draft_len).sum())
+
+    rej = 0
+    for _ in range(max(args.warmup, 1)):
+        rej = step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    nbytes = (w.n_draft_rows + w.n_target_rows + rej) * w.V * w.elem_bytes
+    value = nbytes * args.steps / dt / 1e9
+    sample = "%d sequences of the workload per step (%d draft + %d target rows)" % (n_seq, w.n_draft_rows,
+                                                                                  w.n_target_rows)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": max(args.warmup, 1), "ms_per_step": 1000.0 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": describe(w, B=spec["B"]), "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="ragged", choices=sorted(workloads.SPECS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

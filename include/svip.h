@@ -181,6 +181,22 @@ int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits
                 const float* uniforms, int32_t* n_accepted, int32_t* next_token, void* stream);
 
 /*
+ * Timing of the row-statistics kernel (the one pass over all target rows inside
+ * svip_verify, its dominant kernel) with CUDA events recorded on the caller's
+ * stream around that launch.  The paper has no counterpart; benchmarks use it
+ * to report the kernel's bandwidth without a profiler.
+ *   svip_profile_enable(ctx, 1) creates the events (not inside a graph
+ *   capture) and turns recording on; (ctx, 0) turns it off.  While on, every
+ *   svip_verify call records one event pair (at most 4096 pairs are kept
+ *   between reads; later calls are not recorded).
+ *   svip_profile_read synchronises on the recorded events, writes the summed
+ *   kernel time in milliseconds and the number of launches it covers (HOST
+ *   pointers), and starts a new interval.
+ */
+int svip_profile_enable(svip_ctx* ctx, int on);
+int svip_profile_read(svip_ctx* ctx, double* total_ms, long* launches);
+
+/*
  * CUDA-graph replay for latency-bound use (small B).  Between begin and end
  * every svip_* call on `stream` is recorded instead of run; svip_graph_end
  * returns an executable graph that svip_graph_launch replays.  All pointers

@@ -66,6 +66,10 @@ def library():
     L.svip_verify.restype = i32
     L.svip_verify.argtypes = [vp, vp, vp, lng, vp, lng, lng, vp, lng, i32, vp, i32, i32, i32, i32, f32,
                               vp, vp, vp, vp]
+    L.svip_profile_enable.restype = i32
+    L.svip_profile_enable.argtypes = [vp, i32]
+    L.svip_profile_read.restype = i32
+    L.svip_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_long)]
     L.svip_graph_begin.restype = i32
     L.svip_graph_begin.argtypes = [vp, vp]
     L.svip_graph_end.restype = i32
@@ -162,6 +166,15 @@ class Context:
                                      _ptr(target_logits), int(t_row_stride), int(dtype), _ptr(cu_rows),
                                      int(B), int(K), int(n_target_rows), int(V), float(T), _ptr(uniforms),
                                      _ptr(n_accepted), _ptr(next_token), _stream(stream)), self._h)
+
+    def profile_enable(self, on: bool):
+        _check(library().svip_profile_enable(self._h, 1 if on else 0), self._h)
+
+    def profile_read(self):
+        ms = C.c_double(0.0)
+        n = C.c_long(0)
+        _check(library().svip_profile_read(self._h, C.byref(ms), C.byref(n)), self._h)
+        return float(ms.value), int(n.value)
 
     def graph_begin(self, stream):
         _check(library().svip_graph_begin(self._h, _stream(stream)), self._h)

@@ -552,7 +552,13 @@ struct svip_ctx {
     float2* q_stats;
     int32_t* p_argmax;
     unsigned* status;
+    int profiling;
+    int prof_used;
+    cudaEvent_t* prof_start;
+    cudaEvent_t* prof_stop;
 };
+
+constexpr int kProfilePairs = 4096;
 
 struct svip_graph {
     cudaGraphExec_t exec;
@@ -659,6 +665,14 @@ int svip_destroy(svip_ctx* ctx) {
     cudaGetDevice(&prev);
     cudaSetDevice(ctx->device);
     cudaFree(ctx->p_stats); cudaFree(ctx->q_stats); cudaFree(ctx->p_argmax); cudaFree(ctx->status);
+    if (ctx->prof_start) {
+        for (int k = 0; k < kProfilePairs; ++k) {
+            cudaEventDestroy(ctx->prof_start[k]);
+            cudaEventDestroy(ctx->prof_stop[k]);
+        }
+        delete[] ctx->prof_start;
+        delete[] ctx->prof_stop;
+    }
     cudaSetDevice(prev);
     delete ctx;
     return SVIP_OK;
@@ -753,6 +767,8 @@ int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits
     s.cu = cu_rows; s.q_seq_stride = q_seq_stride; s.q_pos_stride = q_pos_stride;
     s.out_stats = ctx->p_stats; s.out_argmax = sampling ? nullptr : ctx->p_argmax; s.status = ctx->status;
     int S = pick_cluster(ctx, n_target_rows, V, dtype);
+    const bool timed = ctx->profiling && !ctx->capturing && ctx->prof_used < kProfilePairs;
+    if (timed) cudaEventRecord(ctx->prof_start[ctx->prof_used], st);
     if (sampling)
         e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 1>, n_target_rows, S, s, st)
                                : launch_clustered(row_stats_kernel<kF32, 1>, n_target_rows, S, s, st);
@@ -761,6 +777,7 @@ int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits
                                : launch_clustered(row_stats_kernel<kF32, 0>, n_target_rows, S, s, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
+    if (timed) cudaEventRecord(ctx->prof_stop[ctx->prof_used++], st);
 
     if (!sampling) {
         GreedyArgs g;
@@ -797,6 +814,49 @@ int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits
                            : launch_clustered(verify_finish_kernel<kF32>, B, Sf, f, st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
+    return SVIP_OK;
+}
+
+int svip_profile_enable(svip_ctx* ctx, int on) {
+    if (!ctx) return SVIP_ERR_INVALID_ARG;
+    if (ctx->capturing) return SVIP_ERR_STATE;
+    if (on && !ctx->prof_start) {
+        int prev = 0;
+        cudaGetDevice(&prev);
+        cudaSetDevice(ctx->device);
+        ctx->prof_start = new (std::nothrow) cudaEvent_t[kProfilePairs]();
+        ctx->prof_stop = new (std::nothrow) cudaEvent_t[kProfilePairs]();
+        cudaError_t e = (ctx->prof_start && ctx->prof_stop) ? cudaSuccess : cudaErrorMemoryAllocation;
+        for (int k = 0; k < kProfilePairs && e == cudaSuccess; ++k) {
+            e = cudaEventCreate(&ctx->prof_start[k]);
+            if (e == cudaSuccess) e = cudaEventCreate(&ctx->prof_stop[k]);
+        }
+        cudaSetDevice(prev);
+        if (e != cudaSuccess) {
+            delete[] ctx->prof_start; delete[] ctx->prof_stop;   // events created so far leak with the context
+            ctx->prof_start = ctx->prof_stop = nullptr;
+            return cuda_fail(ctx, e);
+        }
+    }
+    ctx->profiling = on ? 1 : 0;
+    ctx->prof_used = 0;
+    return SVIP_OK;
+}
+
+int svip_profile_read(svip_ctx* ctx, double* total_ms, long* launches) {
+    if (!ctx || !total_ms || !launches) return SVIP_ERR_INVALID_ARG;
+    if (ctx->capturing) return SVIP_ERR_STATE;
+    double sum = 0.0;
+    for (int k = 0; k < ctx->prof_used; ++k) {
+        cudaError_t e = cudaEventSynchronize(ctx->prof_stop[k]);
+        float ms = 0.f;
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, ctx->prof_start[k], ctx->prof_stop[k]);
+        if (e != cudaSuccess) { ctx->prof_used = 0; return cuda_fail(ctx, e); }
+        sum += ms;
+    }
+    *total_ms = sum;
+    *launches = ctx->prof_used;
+    ctx->prof_used = 0;
     return SVIP_OK;
 }
 
