@@ -149,6 +149,7 @@ class Round:
         self.esz = w.elem_bytes
         self.dt = 1 if w.dtype == "bf16" else 0
         self.upload()
+        self.prepare()
         torch.cuda.synchronize()
 
     def upload(self):
@@ -173,17 +174,24 @@ class Round:
             n += h.numel() * h.element_size()
         return n
 
-    def step(self):
+    def prepare(self):
+        """Pre-marshals the calls of one step (the pointers and shapes never change)."""
         ctx, w, B, V, sp = self.ctx, self.w, self.B, self.V, self.stream
         q, ud, tok, ent = self.d_q.data_ptr(), self.d_ud.data_ptr(), self.d_tok.data_ptr(), self.d_ent.data_ptr()
         stop, stats = self.d_stop.data_ptr(), self.d_stats.data_ptr()
+        calls = []
         for j in range(self.K):
             o = j * B
-            ctx.draft_step(q + o * V * self.esz, self.dt, int(self.active[j]), V, V, w.T, w.h, ud + 4 * o,
-                           tok + 4 * o, ent + 4 * o, stop + o, stats + 8 * o, sp)
-        ctx.pack_ragged(self.d_len, B, w.K_max, self.d_cu, None, None, sp)
-        ctx.verify(self.d_tok, self.d_q, V, self.d_stats, 1, B, self.d_t, V, self.dt, self.d_cu, B, w.K_max,
-                   self.Rp, V, w.T, self.d_uv, self.d_nacc, self.d_next, sp)
+            calls.append(ctx.bind("draft_step", q + o * V * self.esz, self.dt, int(self.active[j]), V, V, w.T, w.h,
+                                  ud + 4 * o, tok + 4 * o, ent + 4 * o, stop + o, stats + 8 * o, sp))
+        calls.append(ctx.bind("pack_ragged", self.d_len, B, w.K_max, self.d_cu, None, None, sp))
+        calls.append(ctx.bind("verify", self.d_tok, self.d_q, V, self.d_stats, 1, B, self.d_t, V, self.dt,
+                              self.d_cu, B, w.K_max, self.Rp, V, w.T, self.d_uv, self.d_nacc, self.d_next, sp))
+        self.calls = calls
+
+    def step(self):
+        for c in self.calls:
+            c()
 
     def logits_bytes(self):
         """Algorithmic logits bytes of one step (needs the results of a finished step)."""
@@ -251,7 +259,7 @@ def cpu_baseline(w, seconds_budget=20.0):
     """The fp64 oracle, as it stands, on a bounded sample of the same workload, on all host cores."""
     from oracle import svip_oracle as O
     cores = len(os.sched_getaffinity(0))
-    n_seq = min(w.B, max(2, cores // 2))
+    n_seq = min(w.B, 64)
     sel = list(range(n_seq))
     rows_q = np.concatenate([np.arange(w.cu_rows[i] - i, w.cu_rows[i] - i + w.draft_len[i]) for i in sel])
     rows_t = np.concatenate([np.arange(w.cu_rows[i], w.cu_rows[i + 1]) for i in sel])
@@ -321,7 +329,8 @@ def run_ours(args):
     total_ms, total_bytes = sharding.aggregate(local_ms, step_bytes * args.steps, device=torch.device("cuda", dev))
 
     # end to end: host buffers in, results out, every step
-    e2e_steps = max(1, min(args.steps, 5))
+    e2e_steps = 0 if args.skip_extras else max(1, min(args.steps, 5))
+    h2d = d2h = 0
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
@@ -359,15 +368,16 @@ def run_ours(args):
                      "achieved": achieved, "peak": peak, "peak_kind": "%s copy bandwidth" % peak_kind,
                      "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
                      "launches_timed": stats_n, "bytes_per_launch": stats_bytes, "traffic": None},
-        "e2e": {"value": e2e_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "e2e": {"value": (e2e_bytes / (e2e_ms * 1e-3) / 1e9) if e2e_steps else None, "unit": "GB/s",
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": launches, "clocks": clocks,
     }
-    try:
-        line["b1"] = b1_latency(ctx, torch)
-    except Exception as exc:   # the headline number does not depend on the latency probe
-        line["b1"] = {"error": repr(exc)}
-    if not args.no_cpu_baseline:
+    if not args.skip_extras:
+        try:
+            line["b1"] = b1_latency(ctx, torch)
+        except Exception as exc:   # the headline number does not depend on the latency probe
+            line["b1"] = {"error": repr(exc)}
+    if not args.no_cpu_baseline and not args.skip_extras:
         line["cpu_baseline"] = cpu_baseline(w)
     line["paper_context"] = ("end-to-end speedups over fixed draft length reported by the paper: up to 17% "
                              "(MT-Bench, 8K context) and 22% (QwQ long-form reasoning); hardware not stated")
@@ -418,11 +428,13 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="ragged", choices=sorted(workloads.SPECS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--skip-extras", action="store_true",
+                    help="only the timed region: no end-to-end leg, no B=1 latency, no CPU baseline (for profiling)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -176,6 +176,26 @@ class Context:
         _check(library().svip_profile_read(self._h, C.byref(ms), C.byref(n)), self._h)
         return float(ms.value), int(n.value)
 
+    def bind(self, name: str, *args):
+        """Pre-marshals one call: returns a zero-argument callable that runs ``svip_<name>(ctx, *args)``
+        and raises on a non-zero status.  Saves the per-call conversion cost in launch-bound loops."""
+        fn = getattr(library(), "svip_" + name)
+        conv = []
+        for a, t in zip(args, fn.argtypes[1:]):
+            if t is C.c_void_p:
+                a = _ptr(a) if not hasattr(a, "cuda_stream") else a.cuda_stream
+                conv.append(C.c_void_p(a))
+            else:
+                conv.append(t(a))
+        h = self._h
+        conv = tuple(conv)
+
+        def call():
+            rc = fn(h, *conv)
+            if rc != 0:
+                _check(rc, h)
+        return call
+
     def graph_begin(self, stream):
         _check(library().svip_graph_begin(self._h, _stream(stream)), self._h)
 

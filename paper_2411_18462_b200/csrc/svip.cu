@@ -146,9 +146,10 @@ struct RowShared {
     SegPick pick;
 };
 
-template <int DT>
+template <int DT, bool kGreedy>
 __global__ void __launch_bounds__(kThreads) draft_step_kernel(DraftArgs a) {
     constexpr int EPV = ElemTraits<DT>::kEPV;
+    extern __shared__ uint4 ring[];
     cg::cluster_group cluster = cg::this_cluster();
     const int S = cluster.dim_blocks().x;
     const int rank = cluster.block_rank();
@@ -161,12 +162,12 @@ __global__ void __launch_bounds__(kThreads) draft_step_kernel(DraftArgs a) {
     const char* rp = static_cast<const char*>(a.logits) +
                      static_cast<size_t>(row) * a.row_stride * ElemTraits<DT>::kBytes;
     const RowGeom g = make_geom<DT>(rp, a.V, S * kWarps);
-    Partial t = reduce_segment<DT, 2>(g, rank * kWarps + warp, a.c, lane);
-    t = warp_merge<2>(t, a.c);
+    const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
+    Partial t = reduce_segment<DT, 2, kGreedy>(g, rank * kWarps + warp, a.c, lane, slot0);
     if (lane == 0) { seg[warp].m = t.m; seg[warp].idx = t.idx; seg[warp].Z = t.Z; seg[warp].A = t.A; }
     cluster.sync();
     if (warp == 0) {
-        float u = a.greedy ? 0.f : a.uniforms[row];
+        float u = kGreedy ? 0.f : a.uniforms[row];
         Partial r; SegPick p;
         combine_segments<2>(cluster, seg, S, a.c, u, lane, r, p);
         if (lane == 0) { res.row = r; res.pick = p; }
@@ -174,7 +175,7 @@ __global__ void __launch_bounds__(kThreads) draft_step_kernel(DraftArgs a) {
     cluster.sync();   // remote reads are done (blocks may now exit); res is visible block-wide
     const Partial R = res.row;
     const SegPick P = res.pick;
-    const bool ok = (R.Z > 0.f) && (fabsf(R.m) <= 3.0e38f);
+    const bool ok = (R.Z > 0.f) && (fabsf(R.m) <= kMaxLogit);
     if (rank == 0 && tid == 0) {
         float H = 0.f;
         if (ok) H = fmaxf(kLn2 * (log2f(R.Z) - R.A / R.Z), 0.f);
@@ -182,15 +183,15 @@ __global__ void __launch_bounds__(kThreads) draft_step_kernel(DraftArgs a) {
         a.entropy[row] = H;
         a.stop[row] = __fsqrt_rn(H) > a.thresh ? 1 : 0;
         if (a.row_stats) { a.row_stats[2 * row] = R.m; a.row_stats[2 * row + 1] = R.Z; }
-        if (a.greedy || !ok) a.token[row] = (R.idx >= 0 && R.idx < a.V) ? R.idx : 0;
+        if (kGreedy || !ok) a.token[row] = (R.idx >= 0 && R.idx < a.V) ? R.idx : 0;
     }
-    if (!a.greedy && ok && P.seg / kWarps == rank) {
+    if (!kGreedy && ok && P.seg / kWarps == rank) {
         SoftmaxWeights<DT> wf;
         wf.g = g; wf.c = a.c; wf.M = __fmul_rn(R.m, a.c);
         int v_lo, v_hi;
         seg_range(g, P.seg, v_lo, v_hi);
         int virt = fine_scan<EPV>(wf, v_lo, v_hi, P.prefix, P.target, scan, tid, lane, warp);
-        if (tid == 0) a.token[row] = virt >= 0 ? virt - g.pre : R.idx;
+        if (tid == 0) a.token[row] = virt >= 0 ? virt - g.pre : 0;
     }
 }
 
@@ -218,6 +219,7 @@ __global__ void __launch_bounds__(kThreads) row_stats_kernel(StatsArgs a) {
     const int unit = blockIdx.x / S;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     __shared__ SegEntry seg[kWarps];
+    extern __shared__ uint4 ring[];
 
     long in_row = unit;
     int out_row = unit;
@@ -233,15 +235,15 @@ __global__ void __launch_bounds__(kThreads) row_stats_kernel(StatsArgs a) {
     const char* rp = static_cast<const char*>(a.logits) +
                      static_cast<size_t>(in_row) * a.row_stride * ElemTraits<DT>::kBytes;
     const RowGeom g = make_geom<DT>(rp, a.V, S * kWarps);
-    Partial t = reduce_segment<DT, kMode>(g, rank * kWarps + warp, a.c, lane);
-    t = warp_merge<kMode>(t, a.c);
+    const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
+    Partial t = reduce_segment<DT, kMode, kMode == 0>(g, rank * kWarps + warp, a.c, lane, slot0);
     if (lane == 0) { seg[warp].m = t.m; seg[warp].idx = t.idx; seg[warp].Z = t.Z; seg[warp].A = 0.f; }
     cluster.sync();
     if (rank == 0 && warp == 0) {
         Partial r; SegPick p;
         combine_segments<kMode>(cluster, seg, S, a.c, 0.f, lane, r, p);
         if (lane == 0) {
-            bool ok = fabsf(r.m) <= 3.0e38f && (kMode == 0 || r.Z > 0.f);
+            bool ok = fabsf(r.m) <= kMaxLogit && (kMode == 0 || r.Z > 0.f);
             if (!ok) atomicOr(a.status, SVIP_STATUS_NONFINITE_ROW);
             if (kMode >= 1) a.out_stats[out_row] = make_float2(r.m, r.Z);
             if (a.out_argmax) a.out_argmax[out_row] = (r.idx >= 0 && r.idx < a.V) ? r.idx : 0;
@@ -573,11 +575,12 @@ int cuda_fail(svip_ctx* ctx, cudaError_t e) {
 }
 
 template <class Args>
-cudaError_t launch_clustered(void (*kernel)(Args), long units, int S, const Args& args, cudaStream_t st) {
+cudaError_t launch_clustered(void (*kernel)(Args), long units, int S, const Args& args, cudaStream_t st,
+                             size_t dyn_smem) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(units * S), 1, 1);
     cfg.blockDim = dim3(kThreads, 1, 1);
-    cfg.dynamicSmemBytes = 0;
+    cfg.dynamicSmemBytes = dyn_smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -638,6 +641,17 @@ int svip_create(svip_ctx** out, int device, int max_rows) {
     if (e != cudaSuccess) rc = SVIP_ERR_CUDA;
     else if (major != 10) rc = SVIP_ERR_UNSUPPORTED;
     c->num_sms = sms;
+    if (rc == SVIP_OK) {
+        // the cp.async rings need more dynamic shared memory than the default limit
+        const void* ringed[] = {
+            (const void*)draft_step_kernel<kBF16, true>, (const void*)draft_step_kernel<kBF16, false>,
+            (const void*)draft_step_kernel<kF32, true>,  (const void*)draft_step_kernel<kF32, false>,
+            (const void*)row_stats_kernel<kBF16, 0>,     (const void*)row_stats_kernel<kBF16, 1>,
+            (const void*)row_stats_kernel<kF32, 0>,      (const void*)row_stats_kernel<kF32, 1>};
+        for (const void* k : ringed)
+            if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes) != cudaSuccess)
+                rc = SVIP_ERR_CUDA;
+    }
     if (rc == SVIP_OK) {
         size_t n = static_cast<size_t>(max_rows);
         if (cudaMalloc(&c->p_stats, n * sizeof(float2)) != cudaSuccess ||
@@ -717,8 +731,13 @@ int svip_draft_step(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, 
     a.stop = stop; a.row_stats = row_stats; a.status = ctx->status;
     int S = pick_cluster(ctx, B, V, dtype);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e = dtype == SVIP_BF16 ? launch_clustered(draft_step_kernel<kBF16>, B, S, a, st)
-                                       : launch_clustered(draft_step_kernel<kF32>, B, S, a, st);
+    cudaError_t e;
+    if (a.greedy)
+        e = dtype == SVIP_BF16 ? launch_clustered(draft_step_kernel<kBF16, true>, B, S, a, st, kRingBytes)
+                               : launch_clustered(draft_step_kernel<kF32, true>, B, S, a, st, kRingBytes);
+    else
+        e = dtype == SVIP_BF16 ? launch_clustered(draft_step_kernel<kBF16, false>, B, S, a, st, kRingBytes)
+                               : launch_clustered(draft_step_kernel<kF32, false>, B, S, a, st, kRingBytes);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
     return SVIP_OK;
@@ -770,11 +789,11 @@ int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits
     const bool timed = ctx->profiling && !ctx->capturing && ctx->prof_used < kProfilePairs;
     if (timed) cudaEventRecord(ctx->prof_start[ctx->prof_used], st);
     if (sampling)
-        e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 1>, n_target_rows, S, s, st)
-                               : launch_clustered(row_stats_kernel<kF32, 1>, n_target_rows, S, s, st);
+        e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 1>, n_target_rows, S, s, st, kRingBytes)
+                               : launch_clustered(row_stats_kernel<kF32, 1>, n_target_rows, S, s, st, kRingBytes);
     else
-        e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 0>, n_target_rows, S, s, st)
-                               : launch_clustered(row_stats_kernel<kF32, 0>, n_target_rows, S, s, st);
+        e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 0>, n_target_rows, S, s, st, kRingBytes)
+                               : launch_clustered(row_stats_kernel<kF32, 0>, n_target_rows, S, s, st, kRingBytes);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
     if (timed) cudaEventRecord(ctx->prof_stop[ctx->prof_used++], st);
@@ -797,8 +816,8 @@ int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits
         d.out_stats = ctx->q_stats; d.out_argmax = nullptr;
         long units = static_cast<long>(B) * K;
         int Sd = pick_cluster(ctx, n_target_rows - B, V, dtype);
-        e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 1>, units, Sd, d, st)
-                               : launch_clustered(row_stats_kernel<kF32, 1>, units, Sd, d, st);
+        e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 1>, units, Sd, d, st, kRingBytes)
+                               : launch_clustered(row_stats_kernel<kF32, 1>, units, Sd, d, st, kRingBytes);
         if (e != cudaSuccess) return cuda_fail(ctx, e);
         ctx->launches += 1;
     }
@@ -810,8 +829,8 @@ int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits
     f.t_row_stride = t_row_stride; f.p_stats = ctx->p_stats; f.cu = cu_rows; f.K = K; f.V = V; f.c = c;
     f.uniforms = uniforms; f.n_accepted = n_accepted; f.next_token = next_token; f.status = ctx->status;
     int Sf = pick_cluster(ctx, B, V, dtype);
-    e = dtype == SVIP_BF16 ? launch_clustered(verify_finish_kernel<kBF16>, B, Sf, f, st)
-                           : launch_clustered(verify_finish_kernel<kF32>, B, Sf, f, st);
+    e = dtype == SVIP_BF16 ? launch_clustered(verify_finish_kernel<kBF16>, B, Sf, f, st, 0)
+                           : launch_clustered(verify_finish_kernel<kF32>, B, Sf, f, st, 0);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
     return SVIP_OK;

@@ -6,12 +6,23 @@
 // range: inverse-CDF sampling then only has to re-read ONE segment (an L2 hit)
 // after the normaliser is known, instead of the whole row.
 //
-// Per-thread state while streaming:
-//   m   running maximum of the raw logits (exact in fp32)
-//   Z   sum of 2^(x*c - M),            M = rn(m*c),  c = log2(e)/T
-//   A   sum of 2^(x*c - M) * (x*c - M)               (log2 units, for the entropy)
-//   idx lowest index attaining m
-// Two partials merge by rescaling both to the larger maximum.
+// Per-thread state while streaming (fast path):
+//   rmax running maximum of the raw logits (exact in fp32), tracked without branches
+//   ref  reference logit of the exponentials; Mref = rn(ref*c), c = log2(e)/T
+//   Z    sum of 2^(x*c - Mref)                      (two packed fp32 accumulators)
+//   A    sum of 2^(x*c - Mref) * (x*c - Mref)       (log2 units, for the entropy)
+// The reference is NOT kept equal to the running maximum: it is only moved up (and Z, A rescaled)
+// when the maximum has run more than 2^64 ahead of it, which almost never happens, so the warp
+// does not diverge on the common "some lane saw a new maximum" event.  Exponents up to +64 are
+// harmless in fp32.  Partials merge by rescaling to the larger maximum.
+//
+// Loads go through a per-thread ring of cp.async slots in shared memory (kStages x 16 bytes per
+// thread): up to kStages loads per thread stay in flight while the thread computes, with no
+// registers held and no barriers (a thread only reads the slots it filled itself).
+//
+// The fast path has no special cases: -inf logits make 0 * -inf = NaN in A and NaN logits make
+// NaN in Z, and a warp whose result is NaN redoes its segment on the slow path, which masks
+// such logits to zero mass.
 #pragma once
 #include <cooperative_groups.h>
 #include <cuda_runtime.h>
@@ -31,6 +42,12 @@ constexpr int kBF16 = 1;
 constexpr float kArgFloor = -127.0f;    // 2^x flushes to zero below this (ftz)
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kIntMax = 0x7fffffff;
+constexpr int kStages = 8;              // cp.async slots per thread
+constexpr int kRingBytes = kStages * kThreads * 16;
+constexpr float kRebase = 64.0f;        // move the reference when the maximum is 2^64 ahead of it
+constexpr float kNoRef = -1.0e30f;      // "no reference yet", finite so that differences stay finite
+constexpr float kMasked = -1.0e30f;     // fast-path stand-in for elements outside the row
+constexpr float kMaxLogit = 1.0e29f;    // rows whose maximum lies outside +-1e29 are reported as non-finite
 
 __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
 
@@ -177,30 +194,141 @@ __device__ __forceinline__ void fold_vector(const uint4& raw, int vi, const RowG
     }
 }
 
-// Streams segment `seg` of the row with the calling warp.
+// Slow path: streams segment `seg` with plain loads, an exact per-lane running maximum and
+// masking of -inf / NaN logits to zero mass.
 template <int DT, int kMode>
-__device__ __forceinline__ Partial reduce_segment(const RowGeom& g, int seg, float c, int lane) {
+__device__ __noinline__ Partial reduce_segment_slow(const RowGeom& g, int seg, float c, int lane) {
     Partial t;
     t.m = neg_inf(); t.idx = kIntMax; t.Z = 0.f; t.A = 0.f;
     float M = neg_inf();
     int v_lo, v_hi;
     seg_range(g, seg, v_lo, v_hi);
-    int vi = v_lo + lane;
-    for (; vi + 96 < v_hi; vi += 128) {
-        uint4 r0 = ld_stream(g.base + vi);
-        uint4 r1 = ld_stream(g.base + vi + 32);
-        uint4 r2 = ld_stream(g.base + vi + 64);
-        uint4 r3 = ld_stream(g.base + vi + 96);
-        fold_vector<DT, kMode>(r0, vi, g, c, t, M);
-        fold_vector<DT, kMode>(r1, vi + 32, g, c, t, M);
-        fold_vector<DT, kMode>(r2, vi + 64, g, c, t, M);
-        fold_vector<DT, kMode>(r3, vi + 96, g, c, t, M);
-    }
-    for (; vi < v_hi; vi += 32) {
+    for (int vi = v_lo + lane; vi < v_hi; vi += 32) {
         uint4 r0 = ld_stream(g.base + vi);
         fold_vector<DT, kMode>(r0, vi, g, c, t, M);
     }
     return t;
+}
+
+// ---------------------------------------------------------------------------
+// Fast path: cp.async ring + packed fp32x2 arithmetic.
+
+__device__ __forceinline__ void cp_async16(uint32_t saddr, const void* gptr) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(saddr), "l"(gptr) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t saddr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "r"(saddr)
+                 : "memory");
+    return v;
+}
+
+typedef unsigned long long f32x2;   // two packed fp32 values
+__device__ __forceinline__ f32x2 pack2(float a, float b) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& a, float& b) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+    f32x2 r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
+struct Acc {
+    float rmax;    // running maximum of the raw logits
+    int ivec;      // vector that first attained rmax (tracked only when asked for)
+    float ref;     // reference logit
+    float Mref;    // rn(ref * c)
+    f32x2 Z2;
+    f32x2 A2;
+};
+
+__device__ __forceinline__ void acc_init(Acc& t, float c) {
+    t.rmax = neg_inf(); t.ivec = kIntMax; t.ref = kNoRef; t.Mref = __fmul_rn(kNoRef, c);
+    t.Z2 = pack2(0.f, 0.f); t.A2 = pack2(0.f, 0.f);
+}
+
+// Moves the reference up to the running maximum.
+template <int kMode>
+__device__ __noinline__ void acc_rebase(Acc& t, float c) {
+    float Mn = __fmul_rn(t.rmax, c);
+    float d = t.Mref - Mn;
+    float s = ex2_approx(fmaxf(d, kArgFloor));
+    f32x2 s2 = pack2(s, s);
+    if (kMode == 2) t.A2 = mul2(s2, fma2(pack2(d, d), t.Z2, t.A2));
+    t.Z2 = mul2(s2, t.Z2);
+    t.ref = t.rmax;
+    t.Mref = Mn;
+}
+
+// Folds EPV unpacked logits (no special values expected) into the accumulator.
+template <int EPV, int kMode, bool kIdx>
+__device__ __forceinline__ void fold_fast(const float (&x)[EPV], int vi, float c, Acc& t) {
+    float old = t.rmax;
+    if (EPV == 8) {
+        float a = max3(old, x[0], x[1]);
+        float b = max3(x[2], x[3], x[4]);
+        float d = max3(x[5], x[6], x[7]);
+        t.rmax = max3(a, b, d);
+    } else {
+        float a = max3(old, x[0], x[1]);
+        t.rmax = max3(a, x[2], x[3]);
+    }
+    if (kIdx) {
+        if (t.rmax > old) t.ivec = vi;
+    }
+    if (kMode == 0) return;
+    if (__fmaf_rn(t.rmax, c, -t.Mref) > kRebase) acc_rebase<kMode>(t, c);
+    const f32x2 c2 = pack2(c, c);
+    const f32x2 nm2 = pack2(-t.Mref, -t.Mref);
+#pragma unroll
+    for (int j = 0; j < EPV; j += 2) {
+        f32x2 a2 = fma2(pack2(x[j], x[j + 1]), c2, nm2);
+        float a0, a1;
+        unpack2(a2, a0, a1);
+        f32x2 e2 = pack2(ex2_approx(a0), ex2_approx(a1));
+        t.Z2 = add2(t.Z2, e2);
+        if (kMode == 2) t.A2 = fma2(e2, a2, t.A2);
+    }
+}
+
+// Unpacks vector vi and replaces the elements outside the row by a very negative finite value.
+template <int DT>
+__device__ __forceinline__ void unpack_edge(const uint4& raw, int vi, const RowGeom& g,
+                                            float (&x)[ElemTraits<DT>::kEPV]) {
+    constexpr int EPV = ElemTraits<DT>::kEPV;
+    ElemTraits<DT>::unpack(raw, x);
+#pragma unroll
+    for (int j = 0; j < EPV; ++j) {
+        int e = vi * EPV + j;
+        if (e < g.pre || e >= g.pre + g.V) x[j] = kMasked;
+    }
 }
 
 __device__ __forceinline__ float warp_sum(float v) {
@@ -240,6 +368,94 @@ __device__ __forceinline__ Partial warp_merge(Partial t, float c) {
     r.m = m; r.idx = idx;
     r.Z = kMode >= 1 ? warp_sum(t.Z) : 0.f;
     r.A = kMode == 2 ? warp_sum(t.A) : 0.f;
+    return r;
+}
+
+// Streams segment `seg` of the row with the calling warp and returns the warp's merged partial
+// (all lanes hold it).  `slot0` is the shared-memory address of this thread's first ring slot;
+// slot s lives kThreads * 16 bytes further.  kIdx asks for the index of the maximum.
+template <int DT, int kMode, bool kIdx>
+__device__ __forceinline__ Partial reduce_segment(const RowGeom& g, int seg, float c, int lane,
+                                                  uint32_t slot0) {
+    constexpr int EPV = ElemTraits<DT>::kEPV;
+    constexpr uint32_t kSlotStride = kThreads * 16;
+    Acc t;
+    acc_init(t, c);
+    int v_lo, v_hi;
+    seg_range(g, seg, v_lo, v_hi);
+    // vectors that stick out of the row are folded apart, by lane 0, with their outside masked
+    const bool head_edge = g.pre > 0;
+    const bool tail_edge = ((g.pre + g.V) % EPV) != 0;
+    int i_lo = v_lo, i_hi = v_hi;
+    if (head_edge && v_lo == 0 && v_hi > 0) i_lo = 1;
+    if (tail_edge && v_hi == g.nvec && i_hi > i_lo) i_hi = g.nvec - 1;
+    if (lane == 0 && head_edge && v_lo == 0 && v_hi > 0) {
+        float x[EPV];
+        unpack_edge<DT>(ld_stream(g.base), 0, g, x);
+        fold_fast<EPV, kMode, kIdx>(x, 0, c, t);
+    }
+    const int vi0 = i_lo + lane;
+    const int n = i_hi > vi0 ? (i_hi - vi0 + 31) >> 5 : 0;
+#pragma unroll
+    for (int s = 0; s < kStages; ++s) {
+        if (s < n) cp_async16(slot0 + s * kSlotStride, g.base + vi0 + 32 * s);
+        cp_async_commit();
+    }
+    for (int it = 0; it < n; ++it) {
+        cp_async_wait<kStages - 1>();
+        const uint32_t sa = slot0 + (it & (kStages - 1)) * kSlotStride;
+        const uint4 raw = lds128(sa);
+        const int nx = it + kStages;
+        if (nx < n) cp_async16(sa, g.base + vi0 + 32 * nx);
+        cp_async_commit();
+        float x[EPV];
+        ElemTraits<DT>::unpack(raw, x);
+        fold_fast<EPV, kMode, kIdx>(x, vi0 + 32 * it, c, t);
+    }
+    cp_async_wait<0>();
+    if (lane == 0 && tail_edge && v_hi == g.nvec && v_lo < v_hi && !(g.nvec == 1 && head_edge)) {
+        float x[EPV];
+        unpack_edge<DT>(ld_stream(g.base + g.nvec - 1), g.nvec - 1, g, x);
+        fold_fast<EPV, kMode, kIdx>(x, g.nvec - 1, c, t);
+    }
+
+    float z0, z1, a0, a1;
+    unpack2(t.Z2, z0, z1);
+    unpack2(t.A2, a0, a1);
+    float Z = z0 + z1, A = a0 + a1;
+    const bool bad = kMode >= 1 && (!(Z == Z) || !(A == A));
+    if (__any_sync(0xffffffffu, bad)) {
+        Partial p = reduce_segment_slow<DT, kMode>(g, seg, c, lane);
+        return warp_merge<kMode>(p, c);
+    }
+    Partial r;
+    r.m = warp_max(t.rmax);
+    r.idx = kIntMax;
+    r.Z = 0.f; r.A = 0.f;
+    if (kMode >= 1) {
+        if (Z > 0.f) {
+            float d = t.Mref - __fmul_rn(r.m, c);
+            float sc = ex2_approx(fmaxf(d, kArgFloor));
+            if (kMode == 2) A = sc * __fmaf_rn(d, Z, A);
+            Z *= sc;
+        } else {
+            Z = 0.f; A = 0.f;
+        }
+        r.Z = warp_sum(Z);
+        if (kMode == 2) r.A = warp_sum(A);
+    }
+    if (kIdx) {
+        int iv = warp_min_int(t.rmax == r.m ? t.ivec : kIntMax);
+        if (iv != kIntMax) {
+            float x[EPV];
+            unpack_masked<DT>(g.base[iv], iv, g, x);
+            int first = -1;
+#pragma unroll
+            for (int j = EPV - 1; j >= 0; --j)
+                if (x[j] == r.m) first = j;
+            if (first >= 0) r.idx = iv * EPV + first - g.pre;
+        }
+    }
     return r;
 }
 
