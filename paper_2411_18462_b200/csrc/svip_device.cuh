@@ -276,7 +276,7 @@ __device__ __forceinline__ void acc_init(Acc& t, float c) {
 
 // Moves the reference up to the running maximum.
 template <int kMode>
-__device__ __noinline__ void acc_rebase(Acc& t, float c) {
+__device__ __forceinline__ void acc_rebase(Acc& t, float c) {
     float Mn = __fmul_rn(t.rmax, c);
     float d = t.Mref - Mn;
     float s = ex2_approx(fmaxf(d, kArgFloor));
