@@ -209,6 +209,46 @@ int svip_graph_end(svip_ctx* ctx, void* stream, svip_graph** graph);
 int svip_graph_launch(svip_graph* graph, void* stream);
 int svip_graph_destroy(svip_graph* graph);
 
+/*
+ * svip_verify for callers that must not allocate device memory.
+ *
+ * The paper has no counterpart; this entry point exists for integration.  Some
+ * hosts of this library cannot call cudaMalloc where they run the verify
+ * round: code executing inside a region where the serving framework has
+ * frozen its memory pool (for example while it records or replays a fixed
+ * memory plan), plugins that are handed a stream but no allocator, and
+ * processes whose device memory is fully pre-partitioned at start-up.  They
+ * cannot create an svip_ctx either, because svip_create allocates the
+ * workspace.  This call takes no context: its workspace (the per-row
+ * normalisers, per-row argmax and the status word of one verify round) is a
+ * fixed array that lives in the library's own device image.
+ *
+ * Same arguments, semantics and results as svip_verify, with these differences
+ *   - `device` is the GPU whose memory the pointers refer to; it must be the
+ *     calling thread's current device.
+ *   - n_target_rows must be <= SVIP_NOALLOC_MAX_ROWS, otherwise the call
+ *     returns SVIP_ERR_WORKSPACE and launches nothing.
+ *   - `status` (DEVICE, may be NULL) receives the status bits of this call;
+ *     the call clears it first.  With NULL the bits are dropped.
+ *   - The call never calls cudaMalloc, cudaFree or any allocating routine.
+ *     The first call on each device looks up the array's device address and
+ *     raises the kernels' shared-memory limit; make that first call outside
+ *     any stream capture.
+ *   - The array costs about 160 KB of device memory on every GPU that loads
+ *     the library, for the life of the process.
+ *   - All calls on one device share the array and it keeps the previous
+ *     call's contents: calls that overlap on the GPU (different streams, or
+ *     the same stream from several threads) race.  Run them one after another
+ *     on one stream, or order them with events.
+ */
+#define SVIP_NOALLOC_MAX_ROWS 8192
+int svip_verify_noalloc(int device, const int32_t* draft_tokens, const void* q_logits,
+                        long q_row_stride, const float* q_stats, long q_seq_stride,
+                        long q_pos_stride, const void* target_logits, long t_row_stride,
+                        svip_dtype dtype, const int32_t* cu_rows, int B, int K, int n_target_rows,
+                        int V, float T, const float* uniforms, int32_t* n_accepted,
+                        int32_t* next_token, unsigned* status, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

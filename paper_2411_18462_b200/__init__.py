@@ -7,8 +7,8 @@ synthetic workloads (``workloads``).  There is no CPU fallback: without the
 compiled library every call raises.
 """
 from .binding import (  # noqa: F401
-    SVIP_BF16, SVIP_F32, SVIP_Q_PACKED, Context, Graph, SvipError, library, library_path,
+    SVIP_BF16, SVIP_F32, SVIP_Q_PACKED, Context, Graph, SvipError, library, library_path, verify_noalloc,
 )
 
 __all__ = ["SVIP_BF16", "SVIP_F32", "SVIP_Q_PACKED", "Context", "Graph", "SvipError", "library",
-           "library_path"]
+           "library_path", "verify_noalloc"]

@@ -70,6 +70,9 @@ def library():
     L.svip_profile_enable.argtypes = [vp, i32]
     L.svip_profile_read.restype = i32
     L.svip_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_long)]
+    L.svip_verify_noalloc.restype = i32
+    L.svip_verify_noalloc.argtypes = [i32, vp, vp, lng, vp, lng, lng, vp, lng, i32, vp, i32, i32, i32, i32, f32,
+                                      vp, vp, vp, vp, vp]
     L.svip_graph_begin.restype = i32
     L.svip_graph_begin.argtypes = [vp, vp]
     L.svip_graph_end.restype = i32
@@ -104,6 +107,17 @@ def _check(code: int, ctx=None):
         if code == -4 and ctx is not None:
             text += " (cudaError %d)" % library().svip_last_cuda_error(ctx)
         raise SvipError(code, text)
+
+
+def verify_noalloc(device, draft_tokens, q_logits, q_row_stride, q_stats, q_seq_stride, q_pos_stride,
+                   target_logits, t_row_stride, dtype, cu_rows, B, K, n_target_rows, V, T, uniforms,
+                   n_accepted, next_token, status=None, stream=None):
+    """``svip_verify_noalloc``: the verify round without a context and without any allocation."""
+    _check(library().svip_verify_noalloc(int(device), _ptr(draft_tokens), _ptr(q_logits), int(q_row_stride),
+                                         _ptr(q_stats), int(q_seq_stride), int(q_pos_stride),
+                                         _ptr(target_logits), int(t_row_stride), int(dtype), _ptr(cu_rows),
+                                         int(B), int(K), int(n_target_rows), int(V), float(T), _ptr(uniforms),
+                                         _ptr(n_accepted), _ptr(next_token), _ptr(status), _stream(stream)))
 
 
 class Graph:

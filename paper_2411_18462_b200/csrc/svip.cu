@@ -918,4 +918,97 @@ int svip_graph_destroy(svip_graph* graph) {
     return SVIP_OK;
 }
 
+// ------------------------------------------------------------------ verify without allocation
+//
+// Workspace of svip_verify_noalloc: one fixed array in the library's device image instead of
+// cudaMalloc'ed memory.  Layout: [p_stats | q_stats | p_argmax | status word].  Every call on a
+// device reuses it, so calls that overlap on the GPU race (see include/svip.h).
+
+namespace {
+
+constexpr size_t kNoAllocRows = SVIP_NOALLOC_MAX_ROWS;
+constexpr size_t kNoAllocStatsBytes = kNoAllocRows * sizeof(float2);
+constexpr size_t kNoAllocBytes = 2 * kNoAllocStatsBytes + kNoAllocRows * sizeof(int32_t) + 256;
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
+
+constexpr int kNoAllocMaxDevices = 64;
+
+struct NoAllocDevice {
+    int ready;
+    int num_sms;
+    unsigned char* base;   // device address of g_noalloc_scratch on this device
+};
+NoAllocDevice g_noalloc_dev[kNoAllocMaxDevices];
+
+// Once per device, with that device current: the host-side name g_noalloc_scratch is not a device
+// address, so ask the runtime for the address the kernels must be given.
+int noalloc_setup(int device, NoAllocDevice** out) {
+    if (device < 0 || device >= kNoAllocMaxDevices) return SVIP_ERR_INVALID_ARG;
+    NoAllocDevice* d = &g_noalloc_dev[device];
+    if (!d->ready) {
+        int current = -1;
+        if (cudaGetDevice(&current) != cudaSuccess) { cudaGetLastError(); return SVIP_ERR_CUDA; }
+        if (current != device) return SVIP_ERR_INVALID_ARG;
+        int major = 0, sms = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
+            cudaGetLastError();
+            return SVIP_ERR_CUDA;
+        }
+        if (major != 10) return SVIP_ERR_UNSUPPORTED;
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) {
+            cudaGetLastError();
+            return SVIP_ERR_CUDA;
+        }
+        const void* ringed[] = {
+            (const void*)row_stats_kernel<kBF16, 0>, (const void*)row_stats_kernel<kBF16, 1>,
+            (const void*)row_stats_kernel<kF32, 0>,  (const void*)row_stats_kernel<kF32, 1>};
+        for (const void* k : ringed)
+            if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes) != cudaSuccess) {
+                cudaGetLastError();
+                return SVIP_ERR_CUDA;
+            }
+        d->num_sms = sms;
+        d->base = static_cast<unsigned char*>(ptr);
+        d->ready = 1;
+    }
+    *out = d;
+    return SVIP_OK;
+}
+
+}  // namespace
+
+int svip_verify_noalloc(int device, const int32_t* draft_tokens, const void* q_logits, long q_row_stride,
+                        const float* q_stats, long q_seq_stride, long q_pos_stride,
+                        const void* target_logits, long t_row_stride, svip_dtype dtype,
+                        const int32_t* cu_rows, int B, int K, int n_target_rows, int V, float T,
+                        const float* uniforms, int32_t* n_accepted, int32_t* next_token,
+                        unsigned* status, void* stream) {
+    if (n_target_rows > SVIP_NOALLOC_MAX_ROWS) return SVIP_ERR_WORKSPACE;
+    NoAllocDevice* d = nullptr;
+    int rc = noalloc_setup(device, &d);
+    if (rc != SVIP_OK) return rc;
+    // A context that lives on this call's stack and points into the fixed array; nothing is allocated.
+    svip_ctx view = {};
+    view.device = device;
+    view.max_rows = SVIP_NOALLOC_MAX_ROWS;
+    view.num_sms = d->num_sms;
+    view.p_stats = reinterpret_cast<float2*>(d->base);
+    view.q_stats = reinterpret_cast<float2*>(d->base + kNoAllocStatsBytes);
+    view.p_argmax = reinterpret_cast<int32_t*>(d->base + 2 * kNoAllocStatsBytes);
+    unsigned* own_status = reinterpret_cast<unsigned*>(d->base + 2 * kNoAllocStatsBytes +
+                                                       kNoAllocRows * sizeof(int32_t));
+    view.status = status ? status : own_status;
+    // the status word must start at zero; everything else in the array is written before it is read
+    if (cudaMemsetAsync(view.status, 0, sizeof(unsigned), static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        cudaGetLastError();
+        return SVIP_ERR_CUDA;
+    }
+    return svip_verify(&view, draft_tokens, q_logits, q_row_stride, q_stats, q_seq_stride, q_pos_stride,
+                       target_logits, t_row_stride, dtype, cu_rows, B, K, n_target_rows, V, T, uniforms,
+                       n_accepted, next_token, stream);
+}
+
 }  // extern "C"
