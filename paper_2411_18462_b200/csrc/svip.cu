@@ -592,12 +592,14 @@ cudaError_t launch_clustered(void (*kernel)(Args), long units, int S, const Args
     return cudaLaunchKernelEx(&cfg, kernel, args);
 }
 
-// Blocks per row: enough blocks to give every SM two, while every thread still has a vector.
+// Blocks per row.  Small launches are latency-bound: spread a row over more blocks as long as
+// the whole grid still fits on the GPU at once (two blocks per SM) and every thread keeps a vector;
+// a second wave of clusters would double the time of such a launch.
 int pick_cluster(const svip_ctx* ctx, long rows, int V, int dtype) {
     if (ctx->cluster_override > 0) return ctx->cluster_override;
     long nvec = (static_cast<long>(V) * (dtype == SVIP_BF16 ? 2 : 4) + 15) / 16;
     int S = 1;
-    while (S < kMaxCluster && rows * S < 2L * ctx->num_sms && nvec / (2 * S) >= kThreads) S *= 2;
+    while (S < kMaxCluster && rows * S * 2 <= 2L * ctx->num_sms && nvec / (2 * S) >= kThreads) S *= 2;
     return S;
 }
 
