@@ -69,46 +69,80 @@ __device__ __forceinline__ void combine_segments(cg::cluster_group& cluster, Seg
 }
 
 // Fine scan of one segment by the whole block.  `wf(vi, w)` yields the weights of the elements
-// of vector vi.  Returns the virtual element index (vector * EPV + lane element) of the first
-// element whose cumulative weight exceeds `target`, else the last element with positive weight,
-// else -1.
+// of vector vi.  Each thread sums a run of consecutive vectors, one block scan places the runs,
+// and the thread whose run crosses `target` walks its run again element by element.  Returns the
+// virtual element index (vector * EPV + element) of the first element whose cumulative weight
+// exceeds `target`, else the last element with positive weight, else -1.
 template <int EPV, class WF>
 __device__ __forceinline__ int fine_scan(WF& wf, int v_lo, int v_hi, float prefix, float target,
                                          ScanShared& sh, int tid, int lane, int warp) {
-    if (tid == 0) { sh.hit = kIntMax; sh.lastpos = -1; }
-    __syncthreads();
+    constexpr int kRun = 4;
+    const int nv = v_hi - v_lo;
+    const int run = min(kRun, max(1, (nv + kThreads - 1) / kThreads));
+    if (tid == 0) { sh.hit = kIntMax; sh.lastpos = -1; sh.result = -1; }
     float running = prefix;
-    for (int cb = v_lo; cb < v_hi; cb += kThreads) {
-        int vi = cb + tid;
-        float w[EPV];
+    for (int cb = v_lo; cb < v_hi; cb += kThreads * run) {
+        const int first = cb + tid * run;
         float ls = 0.f;
-        if (vi < v_hi) {
-            wf(vi, w);
+        int lastv = -1;
+        for (int k = 0; k < run; ++k) {
+            int vi = first + k;
+            if (vi < v_hi) {
+                float w[EPV];
+                wf(vi, w);
+                float sv = 0.f;
 #pragma unroll
-            for (int j = 0; j < EPV; ++j) ls += w[j];
-        } else {
-#pragma unroll
-            for (int j = 0; j < EPV; ++j) w[j] = 0.f;
-        }
-        float total;
-        float ex = block_scan_excl(ls, sh.wsum, lane, warp, total);
-        float cum = running + ex;
-        int myhit = kIntMax, mylast = -1;
-#pragma unroll
-        for (int j = 0; j < EPV; ++j) {
-            cum += w[j];
-            if (w[j] > 0.f) {
-                mylast = vi * EPV + j;
-                if (cum > target && myhit == kIntMax) myhit = vi * EPV + j;
+                for (int j = 0; j < EPV; ++j) sv += w[j];
+                if (sv > 0.f) lastv = vi;
+                ls += sv;
             }
         }
-        if (myhit != kIntMax) atomicMin(&sh.hit, myhit);
-        if (mylast >= 0) atomicMax(&sh.lastpos, mylast);
+        float total;
+        const float lo = running + block_scan_excl(ls, sh.wsum, lane, warp, total);
+        if (ls > 0.f && lo + ls > target) atomicMin(&sh.hit, tid);
+        if (lastv >= 0) atomicMax(&sh.lastpos, lastv);
         __syncthreads();
-        if (sh.hit != kIntMax) break;
+        const int win = sh.hit;
+        if (win != kIntMax) {
+            if (tid == win) {
+                float cum = lo;
+                int res = -1, last = -1;
+                for (int k = 0; k < run; ++k) {
+                    int vi = first + k;
+                    if (vi < v_hi) {
+                        float w[EPV];
+                        wf(vi, w);
+#pragma unroll
+                        for (int j = 0; j < EPV; ++j) {
+                            cum += w[j];
+                            if (w[j] > 0.f) {
+                                last = vi * EPV + j;
+                                if (cum > target && res < 0) res = last;
+                            }
+                        }
+                    }
+                }
+                sh.result = res >= 0 ? res : last;
+            }
+            __syncthreads();
+            return sh.result;
+        }
         running += total;
     }
-    return sh.hit != kIntMax ? sh.hit : sh.lastpos;
+    // rounding left nothing above the target: the last element with weight
+    const int lv = sh.lastpos;
+    if (lv < 0) return -1;
+    if (tid == 0) {
+        float w[EPV];
+        wf(lv, w);
+        int last = -1;
+#pragma unroll
+        for (int j = 0; j < EPV; ++j)
+            if (w[j] > 0.f) last = lv * EPV + j;
+        sh.result = last;
+    }
+    __syncthreads();
+    return sh.result;
 }
 
 // ------------------------------------------------------------------ draft step

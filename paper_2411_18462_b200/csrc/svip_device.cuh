@@ -555,8 +555,9 @@ __device__ __forceinline__ SegPick pick_segment(const float (&mass)[kSegPerLane]
 // Shared scratch of the fine scan.
 struct ScanShared {
     float wsum[kWarps];
-    int hit;       // lowest virtual element index whose cumulative mass exceeds the target
-    int lastpos;   // highest virtual element index with positive weight
+    int hit;       // lowest thread whose run of vectors crosses the target
+    int lastpos;   // highest vector with positive weight
+    int result;    // the element found
 };
 
 }  // namespace svip
