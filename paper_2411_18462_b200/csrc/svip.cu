@@ -16,6 +16,7 @@
 
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <new>
 
 #include "svip.h"
@@ -193,20 +194,24 @@ __global__ void __launch_bounds__(kThreads) draft_step_kernel(DraftArgs a) {
     __shared__ ScanShared scan;
     __shared__ RowShared res;
 
+    pdl_launch_dependents();
     const char* rp = static_cast<const char*>(a.logits) +
                      static_cast<size_t>(row) * a.row_stride * ElemTraits<DT>::kBytes;
     const RowGeom g = make_geom<DT>(rp, a.V, S * kWarps);
     const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
+    pdl_wait();
+    float u = 0.f;
+    if (!kGreedy && warp == 0) u = __ldg(a.uniforms + row);   // fetched now, used after the stream
     Partial t = reduce_segment<DT, 2, kGreedy>(g, rank * kWarps + warp, a.c, lane, slot0);
     if (lane == 0) { seg[warp].m = t.m; seg[warp].idx = t.idx; seg[warp].Z = t.Z; seg[warp].A = t.A; }
     cluster.sync();
     if (warp == 0) {
-        float u = kGreedy ? 0.f : a.uniforms[row];
         Partial r; SegPick p;
         combine_segments<2>(cluster, seg, S, a.c, u, lane, r, p);
         if (lane == 0) { res.row = r; res.pick = p; }
     }
-    cluster.sync();   // remote reads are done (blocks may now exit); res is visible block-wide
+    cluster_arrive();   // done with the peers' shared memory
+    __syncthreads();    // res is visible block-wide
     const Partial R = res.row;
     const SegPick P = res.pick;
     const bool ok = (R.Z > 0.f) && (fabsf(R.m) <= kMaxLogit);
@@ -227,6 +232,7 @@ __global__ void __launch_bounds__(kThreads) draft_step_kernel(DraftArgs a) {
         int virt = fine_scan<EPV>(wf, v_lo, v_hi, P.prefix, P.target, scan, tid, lane, warp);
         if (tid == 0) a.token[row] = virt >= 0 ? virt - g.pre : 0;
     }
+    cluster_wait();     // no block leaves while a peer may still read its shared memory
 }
 
 // ------------------------------------------------------------------ row statistics (verify, phase 1)
@@ -255,6 +261,8 @@ __global__ void __launch_bounds__(kThreads) row_stats_kernel(StatsArgs a) {
     __shared__ SegEntry seg[kWarps];
     extern __shared__ uint4 ring[];
 
+    pdl_launch_dependents();
+    pdl_wait();
     long in_row = unit;
     int out_row = unit;
     if (a.draft_rows) {
@@ -359,6 +367,8 @@ __global__ void __launch_bounds__(kThreads) verify_finish_kernel(FinishArgs a) {
     __shared__ ScanShared scan;
     __shared__ FinishShared fs;
 
+    pdl_launch_dependents();
+    pdl_wait();
     const int row0 = a.cu ? a.cu[i] : i * (a.K + 1);
     const int Ki = a.cu ? a.cu[i + 1] - row0 - 1 : a.K;
     const long dbase = a.q_seq_stride < 0 ? static_cast<long>(row0 - i) : i * a.q_seq_stride;
@@ -490,6 +500,8 @@ struct GreedyArgs {
 };
 
 __global__ void __launch_bounds__(kThreads) verify_greedy_kernel(GreedyArgs a) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int lane = threadIdx.x & 31;
     const int i = blockIdx.x * kWarps + (threadIdx.x >> 5);
     if (i >= a.B) return;
@@ -521,6 +533,8 @@ __global__ void __launch_bounds__(kPackThreads) pack_ragged_kernel(const int32_t
     __shared__ int wsum[32];
     __shared__ int carry;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    pdl_launch_dependents();
+    pdl_wait();
     if (tid == 0) carry = 0;
     __syncthreads();
     for (int base = 0; base < B; base += kPackThreads) {
@@ -603,27 +617,51 @@ struct svip_graph {
 
 namespace {
 
+// SVIP_NO_PDL=1 in the environment launches every kernel fully serialized (for A/B timing).
+const bool g_use_pdl = [] {
+    const char* v = std::getenv("SVIP_NO_PDL");
+    return !(v && v[0] == '1');
+}();
+
 int cuda_fail(svip_ctx* ctx, cudaError_t e) {
     if (ctx) ctx->last_cuda = static_cast<int>(e);
     return SVIP_ERR_CUDA;
 }
 
+// Every kernel goes through here: optional cluster dimension, dynamic shared memory, and the
+// programmatic-serialization attribute that lets the kernel be scheduled while its predecessor in
+// the stream drains (the kernels wait for the predecessor themselves, see pdl_wait()).
+template <class... KArgs, class... Args>
+cudaError_t launch_ex(void (*kernel)(KArgs...), unsigned grid, unsigned block, int S, size_t dyn_smem,
+                      cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(block, 1, 1);
+    cfg.dynamicSmemBytes = dyn_smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    if (S > 0) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = S;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    if (g_use_pdl) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 template <class Args>
 cudaError_t launch_clustered(void (*kernel)(Args), long units, int S, const Args& args, cudaStream_t st,
                              size_t dyn_smem) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(units * S), 1, 1);
-    cfg.blockDim = dim3(kThreads, 1, 1);
-    cfg.dynamicSmemBytes = dyn_smem;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = S;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, args);
+    return launch_ex(kernel, static_cast<unsigned>(units * S), kThreads, S, dyn_smem, st, args);
 }
 
 // Blocks per row.  Small launches are latency-bound: spread a row over more blocks as long as
@@ -785,8 +823,8 @@ int svip_pack_ragged(svip_ctx* ctx, const int32_t* draft_len, int B, int K_max, 
     if (B < 1 || B > 65536 || K_max < 1) return SVIP_ERR_INVALID_ARG;
     if (static_cast<long>(B) * (static_cast<long>(K_max) + 1) >= 0x7fffffffL) return SVIP_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    pack_ragged_kernel<<<1, kPackThreads, 0, st>>>(draft_len, B, K_max, cu_rows, row_seq, row_pos, ctx->status);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_ex(pack_ragged_kernel, 1, kPackThreads, 0, 0, st, draft_len, B, K_max, cu_rows, row_seq,
+                              row_pos, ctx->status);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
     return SVIP_OK;
@@ -839,8 +877,7 @@ int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits
         g.draft_tokens = draft_tokens; g.p_argmax = ctx->p_argmax; g.cu = cu_rows;
         g.q_seq_stride = q_seq_stride; g.q_pos_stride = q_pos_stride; g.B = B; g.K = K;
         g.n_accepted = n_accepted; g.next_token = next_token;
-        verify_greedy_kernel<<<(B + kWarps - 1) / kWarps, kThreads, 0, st>>>(g);
-        e = cudaGetLastError();
+        e = launch_ex(verify_greedy_kernel, static_cast<unsigned>((B + kWarps - 1) / kWarps), kThreads, 0, 0, st, g);
         if (e != cudaSuccess) return cuda_fail(ctx, e);
         ctx->launches += 1;
         return SVIP_OK;

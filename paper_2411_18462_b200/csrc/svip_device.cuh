@@ -230,6 +230,24 @@ __device__ __forceinline__ uint4 lds128(uint32_t saddr) {
     return v;
 }
 
+// Programmatic dependent launch: a kernel lets the next kernel of the stream be scheduled at once
+// (its blocks become resident and run their prologue) and itself waits, before it touches global
+// memory, until the previous kernel has completed and flushed.  Both are no-ops for a kernel that
+// was launched without the programmatic-serialization attribute.
+__device__ __forceinline__ void pdl_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Split cluster barrier: arrive as soon as this thread is done with its peers' shared memory,
+// wait only before leaving (a block must not exit while a peer may still read its memory).
+__device__ __forceinline__ void cluster_arrive() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait() {
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 typedef unsigned long long f32x2;   // two packed fp32 values
 __device__ __forceinline__ f32x2 pack2(float a, float b) {
     f32x2 r;
