@@ -11,10 +11,12 @@
 //   ref  reference logit of the exponentials; Mref = rn(ref*c), c = log2(e)/T
 //   Z    sum of 2^(x*c - Mref)                      (two packed fp32 accumulators)
 //   A    sum of 2^(x*c - Mref) * (x*c - Mref)       (log2 units, for the entropy)
-// The reference is NOT kept equal to the running maximum: it is only moved up (and Z, A rescaled)
-// when the maximum has run more than 2^64 ahead of it, which almost never happens, so the warp
-// does not diverge on the common "some lane saw a new maximum" event.  Exponents up to +64 are
-// harmless in fp32.  Partials merge by rescaling to the larger maximum.
+// The reference is NOT kept equal to the running maximum: it starts as the largest logit among the
+// warp's first vectors and is only moved up (and Z, A rescaled) when the maximum has run more than
+// 2^64 ahead of it, checked once per kStages vectors, which almost never happens, so the warp does
+// not diverge on the common "some lane saw a new maximum" event.  Exponents up to +64 are harmless
+// in fp32; a larger jump between two checks overflows to inf and sends the warp to the slow path.
+// Partials merge by rescaling to the larger maximum.
 //
 // Loads go through a per-thread ring of cp.async slots in shared memory (kStages x 16 bytes per
 // thread): up to kStages loads per thread stay in flight while the thread computes, with no
@@ -45,7 +47,6 @@ constexpr int kIntMax = 0x7fffffff;
 constexpr int kStages = 8;              // cp.async slots per thread
 constexpr int kRingBytes = kStages * kThreads * 16;
 constexpr float kRebase = 64.0f;        // move the reference when the maximum is 2^64 ahead of it
-constexpr float kNoRef = -1.0e30f;      // "no reference yet", finite so that differences stay finite
 constexpr float kMasked = -1.0e30f;     // fast-path stand-in for elements outside the row
 constexpr float kMaxLogit = 1.0e29f;    // rows whose maximum lies outside +-1e29 are reported as non-finite
 
@@ -281,14 +282,16 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 struct Acc {
     float rmax;    // running maximum of the raw logits
     int ivec;      // vector that first attained rmax (tracked only when asked for)
-    float ref;     // reference logit
-    float Mref;    // rn(ref * c)
+    float Mref;    // rn(reference logit * c)
+    f32x2 c2;      // (c, c)
+    f32x2 nm2;     // (-Mref, -Mref)
     f32x2 Z2;
     f32x2 A2;
 };
 
-__device__ __forceinline__ void acc_init(Acc& t, float c) {
-    t.rmax = neg_inf(); t.ivec = kIntMax; t.ref = kNoRef; t.Mref = __fmul_rn(kNoRef, c);
+__device__ __forceinline__ void acc_init(Acc& t, float ref, float c) {
+    t.rmax = neg_inf(); t.ivec = kIntMax; t.Mref = __fmul_rn(ref, c);
+    t.c2 = pack2(c, c); t.nm2 = pack2(-t.Mref, -t.Mref);
     t.Z2 = pack2(0.f, 0.f); t.A2 = pack2(0.f, 0.f);
 }
 
@@ -301,13 +304,14 @@ __device__ __forceinline__ void acc_rebase(Acc& t, float c) {
     f32x2 s2 = pack2(s, s);
     if (kMode == 2) t.A2 = mul2(s2, fma2(pack2(d, d), t.Z2, t.A2));
     t.Z2 = mul2(s2, t.Z2);
-    t.ref = t.rmax;
     t.Mref = Mn;
+    t.nm2 = pack2(-Mn, -Mn);
 }
 
-// Folds EPV unpacked logits (no special values expected) into the accumulator.
+// Folds EPV unpacked logits (no special values expected) into the accumulator.  The reference is
+// not touched here; the caller checks now and then whether it has to move (acc_check).
 template <int EPV, int kMode, bool kIdx>
-__device__ __forceinline__ void fold_fast(const float (&x)[EPV], int vi, float c, Acc& t) {
+__device__ __forceinline__ void fold_fast(const float (&x)[EPV], int vi, Acc& t) {
     float old = t.rmax;
     if (EPV == 8) {
         float a = max3(old, x[0], x[1]);
@@ -321,19 +325,24 @@ __device__ __forceinline__ void fold_fast(const float (&x)[EPV], int vi, float c
     if (kIdx) {
         if (t.rmax > old) t.ivec = vi;
     }
+    if (kMode >= 1) {
+#pragma unroll
+        for (int j = 0; j < EPV; j += 2) {
+            f32x2 a2 = fma2(pack2(x[j], x[j + 1]), t.c2, t.nm2);
+            float a0, a1;
+            unpack2(a2, a0, a1);
+            f32x2 e2 = pack2(ex2_approx(a0), ex2_approx(a1));
+            t.Z2 = add2(t.Z2, e2);
+            if (kMode == 2) t.A2 = fma2(e2, a2, t.A2);
+        }
+    }
+}
+
+// Moves the reference up if the running maximum has run far ahead of it.
+template <int kMode>
+__device__ __forceinline__ void acc_check(Acc& t, float c) {
     if (kMode == 0) return;
     if (__fmaf_rn(t.rmax, c, -t.Mref) > kRebase) acc_rebase<kMode>(t, c);
-    const f32x2 c2 = pack2(c, c);
-    const f32x2 nm2 = pack2(-t.Mref, -t.Mref);
-#pragma unroll
-    for (int j = 0; j < EPV; j += 2) {
-        f32x2 a2 = fma2(pack2(x[j], x[j + 1]), c2, nm2);
-        float a0, a1;
-        unpack2(a2, a0, a1);
-        f32x2 e2 = pack2(ex2_approx(a0), ex2_approx(a1));
-        t.Z2 = add2(t.Z2, e2);
-        if (kMode == 2) t.A2 = fma2(e2, a2, t.A2);
-    }
 }
 
 // Unpacks vector vi and replaces the elements outside the row by a very negative finite value.
@@ -397,8 +406,6 @@ __device__ __forceinline__ Partial reduce_segment(const RowGeom& g, int seg, flo
                                                   uint32_t slot0) {
     constexpr int EPV = ElemTraits<DT>::kEPV;
     constexpr uint32_t kSlotStride = kThreads * 16;
-    Acc t;
-    acc_init(t, c);
     int v_lo, v_hi;
     seg_range(g, seg, v_lo, v_hi);
     // vectors that stick out of the row are folded apart, by lane 0, with their outside masked
@@ -407,41 +414,93 @@ __device__ __forceinline__ Partial reduce_segment(const RowGeom& g, int seg, flo
     int i_lo = v_lo, i_hi = v_hi;
     if (head_edge && v_lo == 0 && v_hi > 0) i_lo = 1;
     if (tail_edge && v_hi == g.nvec && i_hi > i_lo) i_hi = g.nvec - 1;
-    if (lane == 0 && head_edge && v_lo == 0 && v_hi > 0) {
-        float x[EPV];
-        unpack_edge<DT>(ld_stream(g.base), 0, g, x);
-        fold_fast<EPV, kMode, kIdx>(x, 0, c, t);
-    }
+    const bool fold_head = lane == 0 && head_edge && v_lo == 0 && v_hi > 0;
+    const bool fold_tail = lane == 0 && tail_edge && v_hi == g.nvec && v_lo < v_hi && !(g.nvec == 1 && head_edge);
     const int vi0 = i_lo + lane;
     const int n = i_hi > vi0 ? (i_hi - vi0 + 31) >> 5 : 0;
+    const uint4* src = g.base + vi0;
 #pragma unroll
     for (int s = 0; s < kStages; ++s) {
-        if (s < n) cp_async16(slot0 + s * kSlotStride, g.base + vi0 + 32 * s);
+        if (s < n) cp_async16(slot0 + s * kSlotStride, src + 32 * s);
         cp_async_commit();
     }
-    for (int it = 0; it < n; ++it) {
+    // The reference of the exponentials: the largest logit among the warp's first vectors, the
+    // same for all lanes.  Later logits may exceed it by up to 2^kRebase before it is moved.
+    float ref = 0.f;
+    bool bad = false;
+    if (kMode >= 1) {
+        float fm = neg_inf();
+        if (fold_head) {
+            float x[EPV];
+            unpack_masked<DT>(ld_stream(g.base), 0, g, x);
+            fm = vec_max<EPV>(x);
+        }
+        if (fold_tail) {
+            float x[EPV];
+            unpack_masked<DT>(ld_stream(g.base + g.nvec - 1), g.nvec - 1, g, x);
+            fm = fmaxf(fm, vec_max<EPV>(x));
+        }
         cp_async_wait<kStages - 1>();
-        const uint32_t sa = slot0 + (it & (kStages - 1)) * kSlotStride;
-        const uint4 raw = lds128(sa);
-        const int nx = it + kStages;
-        if (nx < n) cp_async16(sa, g.base + vi0 + 32 * nx);
-        cp_async_commit();
-        float x[EPV];
-        ElemTraits<DT>::unpack(raw, x);
-        fold_fast<EPV, kMode, kIdx>(x, vi0 + 32 * it, c, t);
+        if (n > 0) {
+            float x[EPV];
+            ElemTraits<DT>::unpack(lds128(slot0), x);
+            fm = fmaxf(fm, vec_max<EPV>(x));
+        }
+        ref = warp_max(fm);
+        bad = !(fabsf(ref) <= kMaxLogit);   // nothing finite seen (or +inf): leave it to the slow path
+    }
+    Acc t;
+    acc_init(t, ref, c);
+    if (!bad) {
+        if (fold_head) {
+            float x[EPV];
+            unpack_edge<DT>(ld_stream(g.base), 0, g, x);
+            fold_fast<EPV, kMode, kIdx>(x, 0, t);
+        }
+        int it = 0;
+        // steady state: every prefetch is in range, slot numbers are compile-time constants
+        for (; it + 2 * kStages <= n; it += kStages) {
+            const uint4* p = src + 32 * it;
+#pragma unroll
+            for (int s = 0; s < kStages; ++s) {
+                cp_async_wait<kStages - 1>();
+                const uint4 raw = lds128(slot0 + s * kSlotStride);
+                cp_async16(slot0 + s * kSlotStride, p + 32 * (kStages + s));
+                cp_async_commit();
+                float x[EPV];
+                ElemTraits<DT>::unpack(raw, x);
+                fold_fast<EPV, kMode, kIdx>(x, vi0 + 32 * (it + s), t);
+            }
+            acc_check<kMode>(t, c);
+        }
+        // drain: `it` is a multiple of kStages, so the ring position is it & (kStages - 1)
+        for (; it < n; ++it) {
+            cp_async_wait<kStages - 1>();
+            const uint32_t sa = slot0 + (it & (kStages - 1)) * kSlotStride;
+            const uint4 raw = lds128(sa);
+            const int nx = it + kStages;
+            if (nx < n) cp_async16(sa, src + 32 * nx);
+            cp_async_commit();
+            float x[EPV];
+            ElemTraits<DT>::unpack(raw, x);
+            fold_fast<EPV, kMode, kIdx>(x, vi0 + 32 * it, t);
+            acc_check<kMode>(t, c);
+        }
+        if (fold_tail) {
+            float x[EPV];
+            unpack_edge<DT>(ld_stream(g.base + g.nvec - 1), g.nvec - 1, g, x);
+            fold_fast<EPV, kMode, kIdx>(x, g.nvec - 1, t);
+            acc_check<kMode>(t, c);
+        }
     }
     cp_async_wait<0>();
-    if (lane == 0 && tail_edge && v_hi == g.nvec && v_lo < v_hi && !(g.nvec == 1 && head_edge)) {
-        float x[EPV];
-        unpack_edge<DT>(ld_stream(g.base + g.nvec - 1), g.nvec - 1, g, x);
-        fold_fast<EPV, kMode, kIdx>(x, g.nvec - 1, c, t);
-    }
 
     float z0, z1, a0, a1;
     unpack2(t.Z2, z0, z1);
     unpack2(t.A2, a0, a1);
     float Z = z0 + z1, A = a0 + a1;
-    const bool bad = kMode >= 1 && (!(Z == Z) || !(A == A));
+    // +inf, NaN (from -inf or NaN logits, or an overflow between two checks): redo the segment
+    if (kMode >= 1) bad = bad || !(fabsf(Z) <= 3.0e38f) || !(fabsf(A) <= 3.0e38f);
     if (__any_sync(0xffffffffu, bad)) {
         Partial p = reduce_segment_slow<DT, kMode>(g, seg, c, lane);
         return warp_merge<kMode>(p, c);
