@@ -88,7 +88,7 @@ int svip_create(svip_ctx** ctx, int device, int max_rows);
 int svip_destroy(svip_ctx* ctx);
 
 /*
- * Launch-shape override, for tests and tuning: `cluster_size` in {0,1,2,4,8}
+ * Launch-shape override, for tests and tuning: `cluster_size` in 0..8
  * is the number of thread blocks (one cluster) that share one logits row;
  * 0 restores the automatic choice from (rows, V, dtype).  Every choice gives
  * the same integers, and entropies equal to within fp32 summation order.

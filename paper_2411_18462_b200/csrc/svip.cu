@@ -664,15 +664,18 @@ cudaError_t launch_clustered(void (*kernel)(Args), long units, int S, const Args
     return launch_ex(kernel, static_cast<unsigned>(units * S), kThreads, S, dyn_smem, st, args);
 }
 
-// Blocks per row.  Small launches are latency-bound: spread a row over more blocks as long as
-// the whole grid still fits on the GPU at once (two blocks per SM) and every thread keeps a vector;
-// a second wave of clusters would double the time of such a launch.
+// Blocks per row.  Small launches are latency-bound: spread a row over as many blocks (1..8, any
+// size) as still lets the whole grid sit on the GPU at once (two blocks per SM) while every thread
+// keeps a vector; a second wave of clusters would double the time of such a launch.
 int pick_cluster(const svip_ctx* ctx, long rows, int V, int dtype) {
     if (ctx->cluster_override > 0) return ctx->cluster_override;
     long nvec = (static_cast<long>(V) * (dtype == SVIP_BF16 ? 2 : 4) + 15) / 16;
-    int S = 1;
-    while (S < kMaxCluster && rows * S * 2 <= 2L * ctx->num_sms && nvec / (2 * S) >= kThreads) S *= 2;
-    return S;
+    long by_grid = rows > 0 ? (2L * ctx->num_sms) / rows : kMaxCluster;
+    long by_work = nvec / kThreads;
+    long S = by_grid < by_work ? by_grid : by_work;
+    if (S > kMaxCluster) S = kMaxCluster;
+    if (S < 1) S = 1;
+    return static_cast<int>(S);
 }
 
 bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
@@ -768,8 +771,7 @@ int svip_destroy(svip_ctx* ctx) {
 
 int svip_set_cluster_size(svip_ctx* ctx, int cluster_size) {
     if (!ctx) return SVIP_ERR_INVALID_ARG;
-    if (cluster_size != 0 && cluster_size != 1 && cluster_size != 2 && cluster_size != 4 && cluster_size != 8)
-        return SVIP_ERR_INVALID_ARG;
+    if (cluster_size < 0 || cluster_size > kMaxCluster) return SVIP_ERR_INVALID_ARG;
     ctx->cluster_override = cluster_size;
     return SVIP_OK;
 }

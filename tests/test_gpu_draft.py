@@ -36,7 +36,7 @@ def test_small_shapes_all_cluster_sizes(ctx, oracle, V, bf16):
     u = rng.random(B).astype(np.float32)
     ref = None
     for T in (1.0, 0.7, 0.0):
-        for S in (1, 2, 4, 8, 0):
+        for S in (1, 2, 3, 4, 5, 6, 7, 8, 0):
             ctx.set_cluster_size(S)
             got = tl.gpu_draft_step(ctx, logits, T, 0.3, u)
             tl.check_draft_against_oracle(oracle, logits, T, 0.3, u, got, "V=%d S=%d T=%g" % (V, S, T))
@@ -79,6 +79,47 @@ def test_closed_forms_and_stop_threshold(ctx):
         assert stats[0, 0] == 0.0 and abs(stats[0, 1] - V) < 1e-3 * V and stats[1, 1] == 1.0
         tok, H, stop, _ = tl.gpu_draft_step(ctx, W.to_bf16_bits(x), 0.0, 0.3, None)
         assert tok.tolist() == [0, V - 3, 5]
+    assert ctx.read_status() == 0
+
+
+def special_rows(V, bf16):
+    """Rows that leave the fast path of the streaming loop: a steep ramp (the reference of the
+    exponentials has to move many times), a late spike and a late cliff (the running sums overflow
+    between two checks), rows that start with masked logits, a NaN, and huge but finite logits."""
+    i = np.arange(V, dtype=np.float64)
+    rows = [
+        -300.0 + 600.0 * i / max(V - 1, 1),                 # ramp up
+        300.0 - 600.0 * i / max(V - 1, 1),                  # ramp down
+        np.where(i == V - 3, 400.0, np.sin(i)),             # spike far above everything, near the end
+        np.where(i >= V // 2, 250.0 + np.cos(i), -250.0),   # cliff in the middle
+        np.where(i < min(V // 3 + 1, 3000), -np.inf, np.cos(i) * 3),   # starts with masked logits
+        np.where(i % 97 == 5, -np.inf, np.sin(i) * 5),      # masked logits everywhere
+        np.sin(i) * 2.0,                                     # gets a NaN below
+        np.cos(i) * 1.0e4,                                   # huge spread
+    ]
+    x = np.stack(rows).astype(np.float32)
+    x[6, V // 2] = np.nan
+    return W.to_bf16_bits(x) if bf16 else x
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("V", [9000, 152064])
+def test_rows_off_the_fast_path(ctx, oracle, V, bf16):
+    logits = special_rows(V, bf16)
+    B = logits.shape[0]
+    u = np.linspace(0.05, 0.95, B).astype(np.float32)
+    # the oracle treats NaN like the library: as a masked logit
+    clean = logits.copy()
+    if bf16:
+        clean[6, V // 2] = 0xFF80
+    else:
+        clean[6, V // 2] = -np.inf
+    for T in (1.0, 0.25, 0.0):
+        for S in (0, 1, 3, 8):
+            ctx.set_cluster_size(S)
+            got = tl.gpu_draft_step(ctx, logits, T, 0.3, u)
+            tl.check_draft_against_oracle(oracle, clean, T, 0.3, u, got, "special V=%d S=%d T=%g" % (V, S, T))
+    ctx.set_cluster_size(0)
     assert ctx.read_status() == 0
 
 

@@ -49,7 +49,7 @@ def test_small_ragged_all_cluster_sizes(ctx, oracle, V, bf16):
     rng = np.random.default_rng(4000 + V + int(bf16))
     lens, cu, q, tgt, ud, uv = small_case(rng, 6, V, 5, bf16)
     for T in (1.0, 0.7, 0.0):
-        for S in (1, 2, 4, 8, 0):
+        for S in (1, 2, 3, 4, 5, 6, 7, 8, 0):
             ctx.set_cluster_size(S)
             run_case(ctx, oracle, lens, cu, q, tgt, ud, uv, T, 5, "V=%d S=%d T=%g" % (V, S, T),
                      with_stats=(S % 2 == 0))
