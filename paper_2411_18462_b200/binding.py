@@ -19,7 +19,8 @@ SVIP_STATUS_NONFINITE_ROW = 1
 SVIP_STATUS_BAD_DRAFT_LEN = 2
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "csrc", "libsvip.so")
+# SVIP_LIBRARY in the environment points at another build of the same ABI (a debug build, say)
+_LIB_PATH = os.environ.get("SVIP_LIBRARY") or os.path.join(_HERE, "csrc", "libsvip.so")
 _lib = None
 
 

@@ -670,7 +670,9 @@ cudaError_t launch_clustered(void (*kernel)(Args), long units, int S, const Args
 int pick_cluster(const svip_ctx* ctx, long rows, int V, int dtype) {
     if (ctx->cluster_override > 0) return ctx->cluster_override;
     long nvec = (static_cast<long>(V) * (dtype == SVIP_BF16 ? 2 : 4) + 15) / 16;
-    long by_grid = rows > 0 ? (2L * ctx->num_sms) / rows : kMaxCluster;
+    // measured: grids up to about 7/4 blocks per SM run as one wave next to the blocks of the
+    // following launch that programmatic launch makes resident early; fuller grids run as two
+    long by_grid = rows > 0 ? (7L * ctx->num_sms / 4) / rows : kMaxCluster;
     long by_work = nvec / kThreads;
     long S = by_grid < by_work ? by_grid : by_work;
     if (S > kMaxCluster) S = kMaxCluster;
