@@ -261,3 +261,40 @@ double svip_oracle_residual(const double *p, const double *q, long V, double *w)
     }
     return S;
 }
+
+/*
+ * The quantities of the paper's analysis for one (target row, draft row) pair, all in nats:
+ *   out[0] beta   = sum_x min(p, q)                                   (Eq. 1)
+ *   out[1] H_q    = entropy of the draft distribution                 (Eq. 4)
+ *   out[2] H_qp   = cross entropy -sum q ln p                         (Eq. 4)
+ *   out[3] KL     = KL(q || p) = H_qp - H_q                           (Eq. 3 / Eq. 4)
+ *   out[4] gamma  = H_qp / H_q                                        (Section 2.2)
+ *   out[5] 1 - sqrt(KL / 2)                 Pinsker "oracle bound"    (Eq. 3)
+ *   out[6] 1 - sqrt(1 - exp(-KL))           Bretagnolle-Huber bound   (Appendix B)
+ *   out[7] 1 - sqrt(c * H_q)                approximation bound       (Eq. 6)
+ * p = softmax(target row / T), q = softmax(draft row / T), T > 0.
+ */
+int svip_oracle_pair_stats(const void *t_row, const void *q_row, int dtype, long V, double T,
+                           double c_bound, double *out)
+{
+    double *p = (double *)malloc((size_t)V * sizeof(double));
+    double *q = (double *)malloc((size_t)V * sizeof(double));
+    if (!p || !q) { free(p); free(q); return -1; }
+    svip_oracle_softmax(t_row, dtype, V, T, p);
+    svip_oracle_softmax(q_row, dtype, V, T, q);
+    double beta = svip_oracle_beta(p, q, V);
+    double Hq = svip_oracle_entropy(q, V);
+    double Hqp = svip_oracle_cross_entropy(q, p, V);
+    double KL = Hqp - Hq;
+    out[0] = beta;
+    out[1] = Hq;
+    out[2] = Hqp;
+    out[3] = KL;
+    out[4] = Hqp / Hq;
+    out[5] = 1.0 - sqrt(0.5 * (KL > 0.0 ? KL : 0.0));
+    out[6] = 1.0 - sqrt(1.0 - exp(-(KL > 0.0 ? KL : 0.0)));
+    out[7] = 1.0 - sqrt(c_bound * Hq);
+    free(p);
+    free(q);
+    return 0;
+}

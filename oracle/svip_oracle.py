@@ -61,6 +61,8 @@ def lib():
             f = getattr(L, name)
             f.restype = C.c_double
             f.argtypes = [dp, dp, C.c_long]
+        L.svip_oracle_pair_stats.restype = C.c_int
+        L.svip_oracle_pair_stats.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_long, C.c_double, C.c_double, dp]
         L.svip_oracle_residual.restype = C.c_double
         L.svip_oracle_residual.argtypes = [dp, dp, C.c_long, dp]
         _lib = L
@@ -217,6 +219,27 @@ def verify(draft_tokens: np.ndarray, q_logits: np.ndarray, target_logits: np.nda
 
     _pmap(one, B, threads)
     return n_acc, nxt, (aprob if want_accept_prob else None)
+
+
+def pair_stats(target_logits: np.ndarray, q_logits: np.ndarray, T: float, c_bound: float, threads: int = 1):
+    """Rows of the two [n,V] arrays pairwise -> float64 [n,8]:
+    beta, H_q, H_qp, KL(q||p), gamma, Pinsker bound, Bretagnolle-Huber bound, approximation bound."""
+    t = _rows2d(target_logits); q = _rows2d(q_logits)
+    n, V = t.shape
+    code = _dtype_code(t)
+    assert q.shape == t.shape and _dtype_code(q) == code
+    out = np.empty((n, 8), dtype=np.float64)
+    L = lib()
+
+    def one(r):
+        rc = L.svip_oracle_pair_stats(t.ctypes.data + r * t.strides[0], q.ctypes.data + r * q.strides[0], code, V,
+                                      float(T), float(c_bound),
+                                      C.cast(out.ctypes.data + r * out.strides[0], C.POINTER(C.c_double)))
+        if rc != 0:
+            raise MemoryError("oracle pair_stats")
+
+    _pmap(one, n, threads)
+    return out
 
 
 def pack_ragged(draft_len):

@@ -417,6 +417,46 @@ def test_residual_sign_as_printed_would_fail(oracle):
     assert np.max(np.abs(law_bad - q)) < 1e-14 and np.max(np.abs(law_bad - p)) > 1e-2
 
 
+# ---------------------------------------------------------------- analysis quantities (Eq. 1-6, appendix B)
+
+def test_pair_stats_closed_forms(oracle):
+    """Two-token rows: everything has a closed form.  p = (a, 1-a), q = (b, 1-b)."""
+    consts = {k: float(v) for k, v in read_table("paper_constants.txt")}
+    for dp, dq in ((0.0, 0.0), (1.0, -0.5), (2.5, 0.25), (-1.0, 3.0)):
+        t = np.array([[dp, 0.0]], dtype=np.float32); d = np.array([[dq, 0.0]], dtype=np.float32)
+        for T in (1.0, 0.5):
+            a = 1.0 / (1.0 + math.exp(-dp / T)); b = 1.0 / (1.0 + math.exp(-dq / T))
+            out = oracle.pair_stats(t, d, T, consts["c"])[0]
+            beta = min(a, b) + min(1 - a, 1 - b)
+            Hq = -(b * math.log(b) + (1 - b) * math.log(1 - b))
+            Hqp = -(b * math.log(a) + (1 - b) * math.log(1 - a))
+            KL = b * math.log(b / a) + (1 - b) * math.log((1 - b) / (1 - a))
+            want = [beta, Hq, Hqp, KL, Hqp / Hq, 1 - math.sqrt(KL / 2), 1 - math.sqrt(1 - math.exp(-KL)),
+                    1 - math.sqrt(consts["c"] * Hq)]
+            assert np.allclose(out, want, rtol=1e-11, atol=1e-12), (dp, dq, T, out, want)
+            assert abs(out[3] - (out[2] - out[1])) < 1e-15
+
+
+def test_pair_stats_inequalities_and_gamma_condition(oracle):
+    """beta >= both lower bounds; the approximation bound is conservative exactly when
+    gamma <= 2c + 1 (the condition stated for the constant c); p == q gives beta = 1, KL = 0, gamma = 1."""
+    rng = np.random.default_rng(17)
+    V = 2000
+    d = (rng.standard_normal((40, V)) * rng.uniform(0.3, 4.0, size=(40, 1))).astype(np.float32)
+    t = (d + rng.standard_normal((40, V)).astype(np.float32) * rng.uniform(0.05, 1.5, size=(40, 1))).astype(np.float32)
+    for c in (0.18, 0.5, 2.0):
+        out = oracle.pair_stats(t, d, 1.0, c)
+        beta, Hq, Hqp, KL, gamma, pin, bh, approx = out.T
+        assert np.all(beta >= pin - 1e-12) and np.all(beta >= bh - 1e-12) and np.all(bh >= 0)
+        assert np.all(KL >= -1e-12) and np.all(gamma >= 1 - 1e-12)
+        conservative = approx <= pin + 1e-12
+        assert np.array_equal(conservative, gamma <= 2 * c + 1 + 1e-12)
+        assert np.allclose(pin, 1 - np.sqrt(0.5 * (gamma - 1) * Hq), atol=1e-12)     # Eq. 5
+    same = oracle.pair_stats(d[:3], d[:3], 0.7, 0.18)
+    assert np.allclose(same[:, 0], 1.0, atol=1e-12) and np.allclose(same[:, 3], 0.0, atol=1e-12)
+    assert np.allclose(same[:, 4], 1.0, atol=1e-12)
+
+
 # ---------------------------------------------------------------- ragged packing
 
 def test_pack_ragged_is_exclusive_scan(oracle):
