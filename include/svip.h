@@ -181,6 +181,29 @@ int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits
                 const float* uniforms, int32_t* n_accepted, int32_t* next_token, void* stream);
 
 /*
+ * The quantities of the paper's analysis for n_pairs (target row, draft row)
+ * pairs (Section 2.2: Eq. 1-6; appendix B), with p = softmax(target/T),
+ * q = softmax(draft/T), T > 0, all in nats:
+ *   out[r][0] beta  = sum_x min(p, q), the expected acceptance probability (Eq. 1)
+ *   out[r][1] H_q, the entropy of the draft distribution
+ *   out[r][2] H_qp, the cross entropy -sum q ln p
+ *   out[r][3] KL(q || p) = H_qp - H_q
+ *   out[r][4] gamma = H_qp / H_q
+ *   out[r][5] 1 - sqrt(KL / 2), the Pinsker ("oracle") bound (Eq. 3-4)
+ *   out[r][6] 1 - sqrt(1 - exp(-KL)), the Bretagnolle-Huber bound (appendix B)
+ *   out[r][7] 1 - sqrt(c_bound * H_q), the approximation bound (Eq. 6)
+ * Every entry of [5..7] is a lower bound on beta ([7] only when gamma <= 2*c_bound + 1).
+ * Pair r reads target row r (element r*t_row_stride) and draft row r (element
+ * r*q_row_stride).  `out` is DEVICE [n_pairs][8] fp32.  Where the target masks
+ * a token (-inf) that the draft gives mass, KL, H_qp and gamma are +inf.
+ * Needs n_pairs <= max_rows of svip_create.  Three kernels: the two rows'
+ * normalisers, then one pass over both rows.
+ */
+int svip_pair_stats(svip_ctx* ctx, const void* q_logits, long q_row_stride, const void* target_logits,
+                    long t_row_stride, svip_dtype dtype, int n_pairs, int V, float T, float c_bound,
+                    float* out, void* stream);
+
+/*
  * Timing of the row-statistics kernel (the one pass over all target rows inside
  * svip_verify, its dominant kernel) with CUDA events recorded on the caller's
  * stream around that launch.  The paper has no counterpart; benchmarks use it

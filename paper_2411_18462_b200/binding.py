@@ -71,6 +71,8 @@ def library():
     L.svip_profile_enable.argtypes = [vp, i32]
     L.svip_profile_read.restype = i32
     L.svip_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_long)]
+    L.svip_pair_stats.restype = i32
+    L.svip_pair_stats.argtypes = [vp, vp, lng, vp, lng, i32, i32, i32, f32, f32, vp, vp]
     L.svip_verify_noalloc.restype = i32
     L.svip_verify_noalloc.argtypes = [i32, vp, vp, lng, vp, lng, lng, vp, lng, i32, vp, i32, i32, i32, i32, f32,
                                       vp, vp, vp, vp, vp]
@@ -181,6 +183,12 @@ class Context:
                                      _ptr(target_logits), int(t_row_stride), int(dtype), _ptr(cu_rows),
                                      int(B), int(K), int(n_target_rows), int(V), float(T), _ptr(uniforms),
                                      _ptr(n_accepted), _ptr(next_token), _stream(stream)), self._h)
+
+    def pair_stats(self, q_logits, q_row_stride, target_logits, t_row_stride, dtype, n_pairs, V, T, c_bound, out,
+                   stream=None):
+        _check(library().svip_pair_stats(self._h, _ptr(q_logits), int(q_row_stride), _ptr(target_logits),
+                                         int(t_row_stride), int(dtype), int(n_pairs), int(V), float(T),
+                                         float(c_bound), _ptr(out), _stream(stream)), self._h)
 
     def profile_enable(self, on: bool):
         _check(library().svip_profile_enable(self._h, 1 if on else 0), self._h)
