@@ -125,6 +125,48 @@ int svip_draft_step(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, 
                     void* stream);
 
 /*
+ * svip_draft_step with a per-row mask: rows whose active[b] is 0 are skipped
+ * (their outputs are left untouched, their logits are not read).  `active` is
+ * DEVICE [B] uint8, or NULL for "all rows", which is svip_draft_step.  This is
+ * the draft step of a batch in which some sequences have already stopped
+ * drafting (the inner loop of Algorithm 1, run for B sequences at once).
+ */
+int svip_draft_step_masked(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, int V,
+                           long row_stride, float T, float thresh, const float* uniforms,
+                           const uint8_t* active, int32_t* token, float* entropy, uint8_t* stop,
+                           float* row_stats, void* stream);
+
+/*
+ * Draft-length policies, kept on the device so that the drafting loop needs no
+ * host round trip per token.
+ *   SVIP_POLICY_ENTROPY    the paper's rule: a sequence stops drafting when the
+ *                          draft step raised its stop flag (Eq. 7; Algorithm 1)
+ *   SVIP_POLICY_CONSTANT   baseline 1 of Section 3: exactly gamma[i] tokens
+ *   SVIP_POLICY_HEURISTIC  baseline 2 of Section 3: like CONSTANT, and after
+ *                          every verification gamma[i] grows by 2 if all draft
+ *                          tokens of the round were accepted, else shrinks by 1
+ * Every policy also stops at K_cap tokens (the paper caps the length at 40);
+ * gamma stays within [1, K_cap].
+ *
+ * svip_policy_advance, after each draft step: for every sequence with
+ * active[i] != 0, draft_len[i] += 1, then active[i] = 0 if the policy says
+ * stop.  *n_active (DEVICE int32, may be NULL) receives the number of
+ * sequences still drafting.  `stop` is read by ENTROPY only, `gamma` by the
+ * other two (either may be NULL when unused).  B <= any size; one thread block.
+ *
+ * svip_policy_update, after svip_verify: HEURISTIC adapts gamma[i] from
+ * n_accepted[i] == draft_len[i]; every policy then resets draft_len[i] = 0
+ * and active[i] = 1 for the next round.
+ * All arrays DEVICE: stop, active uint8 [B]; gamma, draft_len, n_accepted int32 [B].
+ */
+typedef enum { SVIP_POLICY_ENTROPY = 0, SVIP_POLICY_CONSTANT = 1, SVIP_POLICY_HEURISTIC = 2 } svip_policy;
+int svip_policy_advance(svip_ctx* ctx, int policy, const uint8_t* stop, const int32_t* gamma,
+                        int32_t* draft_len, uint8_t* active, int B, int K_cap, int32_t* n_active,
+                        void* stream);
+int svip_policy_update(svip_ctx* ctx, int policy, const int32_t* n_accepted, int32_t* draft_len,
+                       int32_t* gamma, uint8_t* active, int B, int K_cap, void* stream);
+
+/*
  * Ragged packing of per-sequence draft lengths (the per-sequence gamma that
  * Algorithm 1 sets when the stop test fires; batching sequences of different
  * gamma is an addition of this library -- the paper's algorithms handle one

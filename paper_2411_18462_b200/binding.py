@@ -71,6 +71,12 @@ def library():
     L.svip_profile_enable.argtypes = [vp, i32]
     L.svip_profile_read.restype = i32
     L.svip_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_long)]
+    L.svip_draft_step_masked.restype = i32
+    L.svip_draft_step_masked.argtypes = [vp, vp, i32, i32, i32, lng, f32, f32, vp, vp, vp, vp, vp, vp, vp]
+    L.svip_policy_advance.restype = i32
+    L.svip_policy_advance.argtypes = [vp, i32, vp, vp, vp, vp, i32, i32, vp, vp]
+    L.svip_policy_update.restype = i32
+    L.svip_policy_update.argtypes = [vp, i32, vp, vp, vp, vp, i32, i32, vp]
     L.svip_pair_stats.restype = i32
     L.svip_pair_stats.argtypes = [vp, vp, lng, vp, lng, i32, i32, i32, f32, f32, vp, vp]
     L.svip_verify_noalloc.restype = i32
@@ -170,6 +176,22 @@ class Context:
         _check(library().svip_draft_step(self._h, _ptr(logits), int(dtype), int(B), int(V), int(row_stride),
                                          float(T), float(thresh), _ptr(uniforms), _ptr(token), _ptr(entropy),
                                          _ptr(stop), _ptr(row_stats), _stream(stream)), self._h)
+
+    def draft_step_masked(self, logits, dtype, B, V, row_stride, T, thresh, uniforms, active, token, entropy, stop,
+                          row_stats=None, stream=None):
+        _check(library().svip_draft_step_masked(self._h, _ptr(logits), int(dtype), int(B), int(V), int(row_stride),
+                                                float(T), float(thresh), _ptr(uniforms), _ptr(active), _ptr(token),
+                                                _ptr(entropy), _ptr(stop), _ptr(row_stats), _stream(stream)),
+               self._h)
+
+    def policy_advance(self, policy, stop, gamma, draft_len, active, B, K_cap, n_active=None, stream=None):
+        _check(library().svip_policy_advance(self._h, int(policy), _ptr(stop), _ptr(gamma), _ptr(draft_len),
+                                             _ptr(active), int(B), int(K_cap), _ptr(n_active), _stream(stream)),
+               self._h)
+
+    def policy_update(self, policy, n_accepted, draft_len, gamma, active, B, K_cap, stream=None):
+        _check(library().svip_policy_update(self._h, int(policy), _ptr(n_accepted), _ptr(draft_len), _ptr(gamma),
+                                            _ptr(active), int(B), int(K_cap), _stream(stream)), self._h)
 
     def pack_ragged(self, draft_len, B, K_max, cu_rows, row_seq=None, row_pos=None, stream=None):
         _check(library().svip_pack_ragged(self._h, _ptr(draft_len), int(B), int(K_max), _ptr(cu_rows),

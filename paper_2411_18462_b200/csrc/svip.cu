@@ -23,6 +23,8 @@
 
 namespace svip {
 
+constexpr int kPolicyThreads = 256;
+
 struct SegEntry {
     float m;
     int idx;
@@ -161,6 +163,7 @@ struct DraftArgs {
     uint8_t* stop;
     float* row_stats;
     unsigned* status;
+    const uint8_t* active;   // NULL, or one flag per row: rows with 0 are skipped
 };
 
 template <int DT>
@@ -200,6 +203,7 @@ __global__ void __launch_bounds__(kThreads) draft_step_kernel(DraftArgs a) {
     const RowGeom g = make_geom<DT>(rp, a.V, S * kWarps);
     const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
     pdl_wait();
+    if (a.active && !a.active[row]) return;   // the whole cluster leaves together
     float u = 0.f;
     if (!kGreedy && warp == 0) u = __ldg(a.uniforms + row);   // fetched now, used after the stream
     Partial t = reduce_segment<DT, 2, kGreedy>(g, rank * kWarps + warp, a.c, lane, slot0);
@@ -633,6 +637,67 @@ __global__ void __launch_bounds__(kThreads) verify_greedy_kernel(GreedyArgs a) {
     }
 }
 
+// ------------------------------------------------------------------ draft-length policies
+//
+// Per-sequence drafting state on the device, so that the loop of Algorithm 1 needs no host round
+// trip per draft token.  ENTROPY is the paper's rule (Eq. 7 flag from the draft step); CONSTANT and
+// HEURISTIC are the two baselines of Section 3.
+
+struct AdvanceArgs {
+    int policy;
+    const uint8_t* stop;
+    const int32_t* gamma;
+    int32_t* draft_len;
+    uint8_t* active;
+    int B, K_cap;
+    int32_t* n_active;
+};
+
+__global__ void __launch_bounds__(kPolicyThreads) policy_advance_kernel(AdvanceArgs a) {
+    pdl_launch_dependents();
+    pdl_wait();
+    // one block: counts the sequences still drafting while it updates them
+    __shared__ int count;
+    if (threadIdx.x == 0) count = 0;
+    __syncthreads();
+    int mine = 0;
+    for (int i = threadIdx.x; i < a.B; i += kPolicyThreads) {
+        if (!a.active[i]) continue;
+        int len = a.draft_len[i] + 1;
+        a.draft_len[i] = len;
+        bool done;
+        if (a.policy == SVIP_POLICY_ENTROPY) done = a.stop[i] != 0 || len >= a.K_cap;
+        else done = len >= min(a.gamma[i], a.K_cap);
+        if (done) a.active[i] = 0; else ++mine;
+    }
+    if (mine) atomicAdd(&count, mine);
+    __syncthreads();
+    if (threadIdx.x == 0 && a.n_active) *a.n_active = count;
+}
+
+struct UpdateArgs {
+    int policy;
+    const int32_t* n_accepted;
+    int32_t* draft_len;
+    int32_t* gamma;
+    uint8_t* active;
+    int B, K_cap;
+};
+
+__global__ void __launch_bounds__(kPolicyThreads) policy_update_kernel(UpdateArgs a) {
+    pdl_launch_dependents();
+    pdl_wait();
+    int i = blockIdx.x * kPolicyThreads + threadIdx.x;
+    if (i >= a.B) return;
+    if (a.policy == SVIP_POLICY_HEURISTIC) {
+        int g = a.gamma[i];
+        g = a.n_accepted[i] == a.draft_len[i] ? min(g + 2, a.K_cap) : max(g - 1, 1);
+        a.gamma[i] = g;
+    }
+    a.draft_len[i] = 0;
+    a.active[i] = 1;
+}
+
 // ------------------------------------------------------------------ ragged packing
 
 constexpr int kPackThreads = 1024;
@@ -906,6 +971,13 @@ int svip_read_status(svip_ctx* ctx, unsigned* flags, void* stream) {
 int svip_draft_step(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, int V, long row_stride,
                     float T, float thresh, const float* uniforms, int32_t* token, float* entropy,
                     uint8_t* stop, float* row_stats, void* stream) {
+    return svip_draft_step_masked(ctx, logits, dtype, B, V, row_stride, T, thresh, uniforms, nullptr, token,
+                                  entropy, stop, row_stats, stream);
+}
+
+int svip_draft_step_masked(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, int V, long row_stride,
+                           float T, float thresh, const float* uniforms, const uint8_t* active,
+                           int32_t* token, float* entropy, uint8_t* stop, float* row_stats, void* stream) {
     if (!ctx || !logits || !token || !entropy || !stop) return SVIP_ERR_INVALID_ARG;
     if (dtype != SVIP_F32 && dtype != SVIP_BF16) return SVIP_ERR_UNSUPPORTED;
     if (B < 0 || V < 1 || V > 0x7fffffe0 || row_stride < 0) return SVIP_ERR_INVALID_ARG;
@@ -916,7 +988,7 @@ int svip_draft_step(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, 
     DraftArgs a;
     a.logits = logits; a.row_stride = row_stride; a.V = V; a.c = scale_for(T); a.thresh = thresh;
     a.greedy = T > 0.f ? 0 : 1; a.uniforms = uniforms; a.token = token; a.entropy = entropy;
-    a.stop = stop; a.row_stats = row_stats; a.status = ctx->status;
+    a.stop = stop; a.row_stats = row_stats; a.status = ctx->status; a.active = active;
     int S = pick_cluster(ctx, B, V, dtype);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e;
@@ -1063,6 +1135,40 @@ int svip_profile_read(svip_ctx* ctx, double* total_ms, long* launches) {
     *total_ms = sum;
     *launches = ctx->prof_used;
     ctx->prof_used = 0;
+    return SVIP_OK;
+}
+
+int svip_policy_advance(svip_ctx* ctx, int policy, const uint8_t* stop, const int32_t* gamma,
+                        int32_t* draft_len, uint8_t* active, int B, int K_cap, int32_t* n_active,
+                        void* stream) {
+    if (!ctx || !draft_len || !active || B < 0 || K_cap < 1) return SVIP_ERR_INVALID_ARG;
+    if (policy != SVIP_POLICY_ENTROPY && policy != SVIP_POLICY_CONSTANT && policy != SVIP_POLICY_HEURISTIC)
+        return SVIP_ERR_INVALID_ARG;
+    if (policy == SVIP_POLICY_ENTROPY ? !stop : !gamma) return SVIP_ERR_INVALID_ARG;
+    if (B == 0) return SVIP_OK;
+    AdvanceArgs a;
+    a.policy = policy; a.stop = stop; a.gamma = gamma; a.draft_len = draft_len; a.active = active;
+    a.B = B; a.K_cap = K_cap; a.n_active = n_active;
+    cudaError_t e = launch_ex(policy_advance_kernel, 1, kPolicyThreads, 0, 0, static_cast<cudaStream_t>(stream), a);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    return SVIP_OK;
+}
+
+int svip_policy_update(svip_ctx* ctx, int policy, const int32_t* n_accepted, int32_t* draft_len,
+                       int32_t* gamma, uint8_t* active, int B, int K_cap, void* stream) {
+    if (!ctx || !draft_len || !active || B < 0 || K_cap < 1) return SVIP_ERR_INVALID_ARG;
+    if (policy != SVIP_POLICY_ENTROPY && policy != SVIP_POLICY_CONSTANT && policy != SVIP_POLICY_HEURISTIC)
+        return SVIP_ERR_INVALID_ARG;
+    if (policy == SVIP_POLICY_HEURISTIC && (!gamma || !n_accepted)) return SVIP_ERR_INVALID_ARG;
+    if (B == 0) return SVIP_OK;
+    UpdateArgs a;
+    a.policy = policy; a.n_accepted = n_accepted; a.draft_len = draft_len; a.gamma = gamma; a.active = active;
+    a.B = B; a.K_cap = K_cap;
+    cudaError_t e = launch_ex(policy_update_kernel, static_cast<unsigned>((B + kPolicyThreads - 1) / kPolicyThreads),
+                              kPolicyThreads, 0, 0, static_cast<cudaStream_t>(stream), a);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
     return SVIP_OK;
 }
 
