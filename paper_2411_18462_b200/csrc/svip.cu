@@ -353,6 +353,113 @@ struct ResidualWeights {
     }
 };
 
+// Sum of the residual (or bonus) weights over one warp segment, streamed through the cp.async ring:
+// four stages for the target row and four for the draft row.  Same arithmetic as
+// ResidualWeights::weights (packed), without its masking: vectors that stick out of the row, and
+// rows whose draft row has another 16-byte phase, go through the functor instead.
+template <int DT>
+__device__ __forceinline__ float residual_segment_sum(const ResidualWeights<DT>& wf, int seg, int lane,
+                                                      uint32_t slot0) {
+    constexpr int EPV = ElemTraits<DT>::kEPV;
+    constexpr uint32_t kSlotStride = kThreads * 16;
+    constexpr int kDepth = kStages / 2;
+    const RowGeom& g = wf.gt;
+    int v_lo, v_hi;
+    seg_range(g, seg, v_lo, v_hi);
+    float acc = 0.f;
+    if (!wf.bonus && wf.gq.pre != g.pre) {
+        for (int vi = v_lo + lane; vi < v_hi; vi += 32) {
+            float w[EPV];
+            wf(vi, w);
+#pragma unroll
+            for (int j = 0; j < EPV; ++j) acc += w[j];
+        }
+        return acc;
+    }
+    const bool head_edge = g.pre > 0;
+    const bool tail_edge = ((g.pre + g.V) % EPV) != 0;
+    int i_lo = v_lo, i_hi = v_hi;
+    if (head_edge && v_lo == 0 && v_hi > 0) i_lo = 1;
+    if (tail_edge && v_hi == g.nvec && i_hi > i_lo) i_hi = g.nvec - 1;
+    const int vi0 = i_lo + lane;
+    const int n = i_hi > vi0 ? (i_hi - vi0 + 31) >> 5 : 0;
+    const uint4* st = g.base + vi0;
+    const uint4* sq = wf.gq.base + vi0;
+    const bool two = !wf.bonus;
+#pragma unroll
+    for (int s = 0; s < kDepth; ++s) {
+        if (s < n) {
+            cp_async16(slot0 + s * kSlotStride, st + 32 * s);
+            if (two) cp_async16(slot0 + (kDepth + s) * kSlotStride, sq + 32 * s);
+        }
+        cp_async_commit();
+    }
+    const f32x2 c2 = pack2(wf.c, wf.c);
+    const f32x2 nmp2 = pack2(-wf.Mp, -wf.Mp), nmq2 = pack2(-wf.Mq, -wf.Mq);
+    const f32x2 rzp2 = pack2(wf.rZp, wf.rZp), rzq2 = pack2(wf.rZq, wf.rZq);
+    float acc1 = 0.f;
+    for (int it = 0; it < n; ++it) {
+        cp_async_wait<kDepth - 1>();
+        const uint32_t sa = slot0 + (it & (kDepth - 1)) * kSlotStride;
+        const uint4 rt = lds128(sa);
+        uint4 rq = make_uint4(0, 0, 0, 0);
+        if (two) rq = lds128(sa + kDepth * kSlotStride);
+        const int nx = it + kDepth;
+        if (nx < n) {
+            cp_async16(sa, st + 32 * nx);
+            if (two) cp_async16(sa + kDepth * kSlotStride, sq + 32 * nx);
+        }
+        cp_async_commit();
+        float x[EPV], d[EPV];
+        ElemTraits<DT>::unpack(rt, x);
+        ElemTraits<DT>::unpack(rq, d);
+#pragma unroll
+        for (int j = 0; j < EPV; j += 2) {
+            float a0, a1;
+            unpack2(fma2(pack2(x[j], x[j + 1]), c2, nmp2), a0, a1);
+            f32x2 p2 = mul2(pack2(ex2_approx(a0), ex2_approx(a1)), rzp2);
+            float p0, p1;
+            unpack2(p2, p0, p1);
+            if (two) {
+                unpack2(fma2(pack2(d[j], d[j + 1]), c2, nmq2), a0, a1);
+                f32x2 q2 = mul2(pack2(ex2_approx(a0), ex2_approx(a1)), rzq2);
+                float q0, q1;
+                unpack2(q2, q0, q1);
+                p0 = fmaxf(p0 - q0, 0.f);
+                p1 = fmaxf(p1 - q1, 0.f);
+            }
+            acc += p0;
+            acc1 += p1;
+        }
+    }
+    cp_async_wait<0>();
+    acc += acc1;
+    if (lane == 0) {
+        float w[EPV];
+        if (head_edge && v_lo == 0 && v_hi > 0) {
+            wf(0, w);
+#pragma unroll
+            for (int j = 0; j < EPV; ++j) acc += w[j];
+        }
+        if (tail_edge && v_hi == g.nvec && v_lo < v_hi && !(g.nvec == 1 && head_edge)) {
+            wf(g.nvec - 1, w);
+#pragma unroll
+            for (int j = 0; j < EPV; ++j) acc += w[j];
+        }
+    }
+    // NaN weights (NaN logits) count as zero in the functor; here they would poison the sum
+    if (!(acc == acc)) {
+        acc = 0.f;
+        for (int vi = v_lo + lane; vi < v_hi; vi += 32) {
+            float w[EPV];
+            wf(vi, w);
+#pragma unroll
+            for (int j = 0; j < EPV; ++j) acc += w[j];
+        }
+    }
+    return acc;
+}
+
 struct FinishShared {
     int n_acc;
     SegPick pick;
@@ -370,6 +477,8 @@ __global__ void __launch_bounds__(kThreads) verify_finish_kernel(FinishArgs a) {
     __shared__ SegEntry seg[kWarps];
     __shared__ ScanShared scan;
     __shared__ FinishShared fs;
+    extern __shared__ uint4 ring[];
+    const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
 
     pdl_launch_dependents();
     pdl_wait();
@@ -440,17 +549,7 @@ __global__ void __launch_bounds__(kThreads) verify_finish_kernel(FinishArgs a) {
     for (int pass = 0; pass < 2; ++pass) {
         // mass of this warp's segment
         int v_lo, v_hi;
-        seg_range(wf.gt, rank * kWarps + warp, v_lo, v_hi);
-        float acc = 0.f;
-#pragma unroll 2
-        for (int vi = v_lo + lane; vi < v_hi; vi += 32) {
-            float w[EPV];
-            wf(vi, w);
-            float s = 0.f;
-#pragma unroll
-            for (int j = 0; j < EPV; ++j) s += w[j];
-            acc += s;
-        }
+        float acc = residual_segment_sum<DT>(wf, rank * kWarps + warp, lane, slot0);
         acc = warp_sum(acc);
         if (lane == 0) { seg[warp].m = 0.f; seg[warp].idx = 0; seg[warp].Z = acc; seg[warp].A = 0.f; }
         cluster.sync();
@@ -901,7 +1000,8 @@ int svip_create(svip_ctx** out, int device, int max_rows) {
             (const void*)draft_step_kernel<kBF16, true>, (const void*)draft_step_kernel<kBF16, false>,
             (const void*)draft_step_kernel<kF32, true>,  (const void*)draft_step_kernel<kF32, false>,
             (const void*)row_stats_kernel<kBF16, 0>,     (const void*)row_stats_kernel<kBF16, 1>,
-            (const void*)row_stats_kernel<kF32, 0>,      (const void*)row_stats_kernel<kF32, 1>};
+            (const void*)row_stats_kernel<kF32, 0>,      (const void*)row_stats_kernel<kF32, 1>,
+            (const void*)verify_finish_kernel<kBF16>,    (const void*)verify_finish_kernel<kF32>};
         for (const void* k : ringed)
             if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes) != cudaSuccess)
                 rc = SVIP_ERR_CUDA;
@@ -1087,9 +1187,16 @@ int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits
     f.q_seq_stride = q_seq_stride; f.q_pos_stride = q_pos_stride; f.t_logits = target_logits;
     f.t_row_stride = t_row_stride; f.p_stats = ctx->p_stats; f.cu = cu_rows; f.K = K; f.V = V; f.c = c;
     f.uniforms = uniforms; f.n_accepted = n_accepted; f.next_token = next_token; f.status = ctx->status;
+    // up to two rows per sequence are streamed: long rows are cut finer than the one-wave policy
+    // asks for (this kernel runs for many microseconds, so several waves are fine)
     int Sf = pick_cluster(ctx, B, V, dtype);
-    e = dtype == SVIP_BF16 ? launch_clustered(verify_finish_kernel<kBF16>, B, Sf, f, st, 0)
-                           : launch_clustered(verify_finish_kernel<kF32>, B, Sf, f, st, 0);
+    if (ctx->cluster_override == 0) {
+        const long row_bytes = static_cast<long>(V) * static_cast<long>(esz);
+        while (Sf < kMaxCluster && 2 * row_bytes / Sf > (512L << 10)) Sf *= 2;
+        if (Sf > kMaxCluster) Sf = kMaxCluster;
+    }
+    e = dtype == SVIP_BF16 ? launch_clustered(verify_finish_kernel<kBF16>, B, Sf, f, st, kRingBytes)
+                           : launch_clustered(verify_finish_kernel<kF32>, B, Sf, f, st, kRingBytes);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
     return SVIP_OK;
@@ -1294,7 +1401,8 @@ int noalloc_setup(int device, NoAllocDevice** out) {
         }
         const void* ringed[] = {
             (const void*)row_stats_kernel<kBF16, 0>, (const void*)row_stats_kernel<kBF16, 1>,
-            (const void*)row_stats_kernel<kF32, 0>,  (const void*)row_stats_kernel<kF32, 1>};
+            (const void*)row_stats_kernel<kF32, 0>,  (const void*)row_stats_kernel<kF32, 1>,
+            (const void*)verify_finish_kernel<kBF16>, (const void*)verify_finish_kernel<kF32>};
         for (const void* k : ringed)
             if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes) != cudaSuccess) {
                 cudaGetLastError();
