@@ -951,6 +951,13 @@ int pick_cluster(const svip_ctx* ctx, long rows, int V, int dtype) {
     long S = by_grid < by_work ? by_grid : by_work;
     if (S > kMaxCluster) S = kMaxCluster;
     if (S < 1) S = 1;
+    // many long rows (more than a wave of blocks anyway): rows above 512 KB are cut so that the
+    // two blocks of an SM finish close together (measured on 256 x 1 MB: 64 -> 55 us)
+    const long row_bytes = nvec * 16;
+    if (S == 1 && rows > ctx->num_sms && row_bytes > (512L << 10)) {
+        S = (row_bytes + (512L << 10) - 1) / (512L << 10);
+        if (S > 4) S = 4;
+    }
     return static_cast<int>(S);
 }
 
