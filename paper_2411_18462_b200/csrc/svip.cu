@@ -184,8 +184,11 @@ struct RowShared {
     SegPick pick;
 };
 
-template <int DT, bool kGreedy>
-__global__ void __launch_bounds__(kThreads) draft_step_kernel(DraftArgs a) {
+// kBlocks is the number of blocks the register budget must leave room for on one SM: 2 for
+// launches that fit the GPU in one wave (latency matters, registers are free), 3 for launches of
+// many waves, where a third resident block streams on while another one is in its epilogue.
+template <int DT, bool kGreedy, int kBlocks>
+__global__ void __launch_bounds__(kThreads, kBlocks) draft_step_kernel(DraftArgs a) {
     constexpr int EPV = ElemTraits<DT>::kEPV;
     extern __shared__ uint4 ring[];
     cg::cluster_group cluster = cg::this_cluster();
@@ -1004,8 +1007,10 @@ int svip_create(svip_ctx** out, int device, int max_rows) {
     if (rc == SVIP_OK) {
         // the cp.async rings need more dynamic shared memory than the default limit
         const void* ringed[] = {
-            (const void*)draft_step_kernel<kBF16, true>, (const void*)draft_step_kernel<kBF16, false>,
-            (const void*)draft_step_kernel<kF32, true>,  (const void*)draft_step_kernel<kF32, false>,
+            (const void*)draft_step_kernel<kBF16, true, 2>, (const void*)draft_step_kernel<kBF16, false, 2>,
+            (const void*)draft_step_kernel<kF32, true, 2>,  (const void*)draft_step_kernel<kF32, false, 2>,
+            (const void*)draft_step_kernel<kBF16, true, 3>, (const void*)draft_step_kernel<kBF16, false, 3>,
+            (const void*)draft_step_kernel<kF32, true, 3>,  (const void*)draft_step_kernel<kF32, false, 3>,
             (const void*)row_stats_kernel<kBF16, 0>,     (const void*)row_stats_kernel<kBF16, 1>,
             (const void*)row_stats_kernel<kF32, 0>,      (const void*)row_stats_kernel<kF32, 1>,
             (const void*)verify_finish_kernel<kBF16>,    (const void*)verify_finish_kernel<kF32>};
@@ -1098,13 +1103,15 @@ int svip_draft_step_masked(svip_ctx* ctx, const void* logits, svip_dtype dtype, 
     a.stop = stop; a.row_stats = row_stats; a.status = ctx->status; a.active = active;
     int S = pick_cluster(ctx, B, V, dtype);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e;
-    if (a.greedy)
-        e = dtype == SVIP_BF16 ? launch_clustered(draft_step_kernel<kBF16, true>, B, S, a, st, kRingBytes)
-                               : launch_clustered(draft_step_kernel<kF32, true>, B, S, a, st, kRingBytes);
+    const bool waves = static_cast<long>(B) * S > 2L * ctx->num_sms;
+    void (*k)(DraftArgs);
+    if (dtype == SVIP_BF16)
+        k = a.greedy ? (waves ? draft_step_kernel<kBF16, true, 3> : draft_step_kernel<kBF16, true, 2>)
+                     : (waves ? draft_step_kernel<kBF16, false, 3> : draft_step_kernel<kBF16, false, 2>);
     else
-        e = dtype == SVIP_BF16 ? launch_clustered(draft_step_kernel<kBF16, false>, B, S, a, st, kRingBytes)
-                               : launch_clustered(draft_step_kernel<kF32, false>, B, S, a, st, kRingBytes);
+        k = a.greedy ? (waves ? draft_step_kernel<kF32, true, 3> : draft_step_kernel<kF32, true, 2>)
+                     : (waves ? draft_step_kernel<kF32, false, 3> : draft_step_kernel<kF32, false, 2>);
+    cudaError_t e = launch_clustered(k, B, S, a, st, kRingBytes);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
     return SVIP_OK;
