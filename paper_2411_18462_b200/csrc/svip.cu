@@ -469,7 +469,7 @@ struct FinishShared {
 };
 
 template <int DT>
-__global__ void __launch_bounds__(kThreads) verify_finish_kernel(FinishArgs a) {
+__global__ void __launch_bounds__(kThreads, 2) verify_finish_kernel(FinishArgs a) {
     using E = ElemTraits<DT>;
     constexpr int EPV = E::kEPV;
     cg::cluster_group cluster = cg::this_cluster();
