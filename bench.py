@@ -31,6 +31,10 @@ from paper_2411_18462_b200 import sharding, workloads  # noqa: E402
 METRIC = "logits GB/s (% of B200 HBM peak) for draft-step+verify; us/step at B=1"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of row_stats_kernel<bf16> per algorithmic byte, from the
+# ncu capture summarised in profiles/row_stats_kernel_bf16_reasoning.md (1056 rows: 337.1 MB for
+# 321.2 MB); traffic grows in proportion to the rows, so a full launch is scaled by its bytes
+ROW_STATS_TRAFFIC_PER_ALGORITHMIC_BYTE = 337.14 / 321.16
 
 
 def describe(w, B=None):
@@ -367,7 +371,9 @@ def run_ours(args):
         "roofline": {"bound": "hbm", "kernel": "row_stats_kernel<bf16> (target rows of svip_verify)",
                      "achieved": achieved, "peak": peak, "peak_kind": "%s copy bandwidth" % peak_kind,
                      "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
-                     "launches_timed": stats_n, "bytes_per_launch": stats_bytes, "traffic": None},
+                     "launches_timed": stats_n, "bytes_per_launch": stats_bytes,
+                     "traffic": ROW_STATS_TRAFFIC_PER_ALGORITHMIC_BYTE * stats_bytes
+                     if w.dtype == "bf16" else None},
         "e2e": {"value": (e2e_bytes / (e2e_ms * 1e-3) / 1e9) if e2e_steps else None, "unit": "GB/s",
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": launches, "clocks": clocks,
