@@ -17,6 +17,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
+#include <mutex>
 #include <new>
 
 #include "svip.h"
@@ -1391,12 +1392,14 @@ struct NoAllocDevice {
     unsigned char* base;   // device address of g_noalloc_scratch on this device
 };
 NoAllocDevice g_noalloc_dev[kNoAllocMaxDevices];
+std::mutex g_noalloc_mutex;   // the per-device set-up may be reached from several host threads
 
 // Once per device, with that device current: the host-side name g_noalloc_scratch is not a device
 // address, so ask the runtime for the address the kernels must be given.
 int noalloc_setup(int device, NoAllocDevice** out) {
     if (device < 0 || device >= kNoAllocMaxDevices) return SVIP_ERR_INVALID_ARG;
     NoAllocDevice* d = &g_noalloc_dev[device];
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
     if (!d->ready) {
         int current = -1;
         if (cudaGetDevice(&current) != cudaSuccess) { cudaGetLastError(); return SVIP_ERR_CUDA; }

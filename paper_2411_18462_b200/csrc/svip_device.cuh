@@ -473,19 +473,31 @@ __device__ __forceinline__ Partial reduce_segment(const RowGeom& g, int seg, flo
             }
             acc_check<kMode>(t, c);
         }
-        // drain: `it` is a multiple of kStages, so the ring position is it & (kStages - 1)
+        // last full ring: same static slots, prefetches only where the segment still has vectors
+        for (; it + kStages <= n; it += kStages) {
+            const uint4* p = src + 32 * it;
+#pragma unroll
+            for (int s = 0; s < kStages; ++s) {
+                cp_async_wait<kStages - 1>();
+                const uint4 raw = lds128(slot0 + s * kSlotStride);
+                if (it + kStages + s < n) cp_async16(slot0 + s * kSlotStride, p + 32 * (kStages + s));
+                cp_async_commit();
+                float x[EPV];
+                ElemTraits<DT>::unpack(raw, x);
+                fold_fast<EPV, kMode, kIdx>(x, vi0 + 32 * (it + s), t);
+            }
+            acc_check<kMode>(t, c);
+        }
+        // fewer than kStages vectors left, all of them already in flight: `it` is a multiple of
+        // kStages, so vector it + k sits in slot k
+        cp_async_wait<0>();
         for (; it < n; ++it) {
-            cp_async_wait<kStages - 1>();
-            const uint32_t sa = slot0 + (it & (kStages - 1)) * kSlotStride;
-            const uint4 raw = lds128(sa);
-            const int nx = it + kStages;
-            if (nx < n) cp_async16(sa, src + 32 * nx);
-            cp_async_commit();
+            const uint4 raw = lds128(slot0 + (it & (kStages - 1)) * kSlotStride);
             float x[EPV];
             ElemTraits<DT>::unpack(raw, x);
             fold_fast<EPV, kMode, kIdx>(x, vi0 + 32 * it, t);
-            acc_check<kMode>(t, c);
         }
+        acc_check<kMode>(t, c);
         if (fold_tail) {
             float x[EPV];
             unpack_edge<DT>(ld_stream(g.base + g.nvec - 1), g.nvec - 1, g, x);
