@@ -223,6 +223,38 @@ int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits
                 const float* uniforms, int32_t* n_accepted, int32_t* next_token, void* stream);
 
 /*
+ * Vocabulary-parallel draft step: the V logits of every row are sharded over G
+ * ranks (a tensor-parallel LM head), rank g holding the V_shard columns that
+ * start at vocab_offset.  The paper's draft step (Algorithm 1 inner loop, Eq. 7)
+ * is unchanged; this is how it is computed when no rank holds a whole row.
+ *
+ *   1. every rank:  svip_vp_partial  -> partial[B][4] fp32 = (largest logit m,
+ *      Z = sum exp((l-m)/T), A = sum exp((l-m)/T)*(l-m)/T in log2 units, global
+ *      index of the first maximum as int bits)        (one pass over the shard)
+ *   2. the ranks all-gather their partials (16 bytes per row and rank) into
+ *      partials[G][B][4], rank-major -- the caller's job (NCCL, any transport)
+ *   3. every rank:  svip_vp_combine  -> entropy[B], stop[B] (identical on all
+ *      ranks), owner[B] = rank whose shard holds the sampled token (-1 when
+ *      greedy), token[B] = the global argmax when T == 0 and -1 otherwise,
+ *      local_target[B] and active[B] = (owner == rank) for step 4
+ *   4. the owner of a row:  svip_vp_locate  -> token[b] for rows with
+ *      active[b] != 0 (others untouched): a second pass over the owner's shard
+ *      of that row only, i.e. 1/G of the logits are read twice.  The ranks then
+ *      share the tokens (max-reduce of token[], which is -1 where not owned).
+ * T == 0 needs steps 1-3 only.  Results equal svip_draft_step on the whole
+ * rows within the same tolerances (the shards are reduced in rank order).
+ * All pointers DEVICE; partial / partials must be 16-byte aligned.
+ */
+int svip_vp_partial(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, int V_shard,
+                    long row_stride, float T, int vocab_offset, float* partial, void* stream);
+int svip_vp_combine(svip_ctx* ctx, const float* partials, int G, int rank, int B, float T, float thresh,
+                    const float* uniforms, float* entropy, uint8_t* stop, int32_t* token,
+                    int32_t* owner, float* local_target, uint8_t* active, void* stream);
+int svip_vp_locate(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, int V_shard,
+                   long row_stride, float T, const float* local_target, const uint8_t* active,
+                   int vocab_offset, int32_t* token, void* stream);
+
+/*
  * The quantities of the paper's analysis for n_pairs (target row, draft row)
  * pairs (Section 2.2: Eq. 1-6; appendix B), with p = softmax(target/T),
  * q = softmax(draft/T), T > 0, all in nats:

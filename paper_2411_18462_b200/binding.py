@@ -77,6 +77,12 @@ def library():
     L.svip_policy_advance.argtypes = [vp, i32, vp, vp, vp, vp, i32, i32, vp, vp]
     L.svip_policy_update.restype = i32
     L.svip_policy_update.argtypes = [vp, i32, vp, vp, vp, vp, i32, i32, vp]
+    L.svip_vp_partial.restype = i32
+    L.svip_vp_partial.argtypes = [vp, vp, i32, i32, i32, lng, f32, i32, vp, vp]
+    L.svip_vp_combine.restype = i32
+    L.svip_vp_combine.argtypes = [vp, vp, i32, i32, i32, f32, f32, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.svip_vp_locate.restype = i32
+    L.svip_vp_locate.argtypes = [vp, vp, i32, i32, i32, lng, f32, vp, vp, i32, vp, vp]
     L.svip_pair_stats.restype = i32
     L.svip_pair_stats.argtypes = [vp, vp, lng, vp, lng, i32, i32, i32, f32, f32, vp, vp]
     L.svip_verify_noalloc.restype = i32
@@ -205,6 +211,22 @@ class Context:
                                      _ptr(target_logits), int(t_row_stride), int(dtype), _ptr(cu_rows),
                                      int(B), int(K), int(n_target_rows), int(V), float(T), _ptr(uniforms),
                                      _ptr(n_accepted), _ptr(next_token), _stream(stream)), self._h)
+
+    def vp_partial(self, logits, dtype, B, V_shard, row_stride, T, vocab_offset, partial, stream=None):
+        _check(library().svip_vp_partial(self._h, _ptr(logits), int(dtype), int(B), int(V_shard), int(row_stride),
+                                         float(T), int(vocab_offset), _ptr(partial), _stream(stream)), self._h)
+
+    def vp_combine(self, partials, G, rank, B, T, thresh, uniforms, entropy, stop, token, owner, local_target,
+                   active, stream=None):
+        _check(library().svip_vp_combine(self._h, _ptr(partials), int(G), int(rank), int(B), float(T), float(thresh),
+                                         _ptr(uniforms), _ptr(entropy), _ptr(stop), _ptr(token), _ptr(owner),
+                                         _ptr(local_target), _ptr(active), _stream(stream)), self._h)
+
+    def vp_locate(self, logits, dtype, B, V_shard, row_stride, T, local_target, active, vocab_offset, token,
+                  stream=None):
+        _check(library().svip_vp_locate(self._h, _ptr(logits), int(dtype), int(B), int(V_shard), int(row_stride),
+                                        float(T), _ptr(local_target), _ptr(active), int(vocab_offset), _ptr(token),
+                                        _stream(stream)), self._h)
 
     def pair_stats(self, q_logits, q_row_stride, target_logits, t_row_stride, dtype, n_pairs, V, T, c_bound, out,
                    stream=None):

@@ -38,7 +38,7 @@ struct SegEntry {
 template <int kMode>
 __device__ __forceinline__ void combine_segments(cg::cluster_group& cluster, SegEntry* seg, int S,
                                                  float c, float u, int lane, Partial& row,
-                                                 SegPick& pick) {
+                                                 SegPick& pick, float abs_target = -1.f) {
     const int nseg = S * kWarps;
     const int per = (nseg + 31) / 32;
     Partial e[kSegPerLane];
@@ -68,7 +68,7 @@ __device__ __forceinline__ void combine_segments(cg::cluster_group& cluster, Seg
     row.m = m;
     row.idx = warp_min_int(idx);
     row.A = warp_sum(asum);
-    pick = pick_segment(mass, per, nseg, u, lane);
+    pick = pick_segment(mass, per, nseg, u, lane, abs_target);
     row.Z = pick.total;
 }
 
@@ -165,6 +165,8 @@ struct DraftArgs {
     float* row_stats;
     unsigned* status;
     const uint8_t* active;   // NULL, or one flag per row: rows with 0 are skipped
+    const float* ext_target; // NULL, or per row the mass to find (units of this row's own Z), see svip_vp_locate
+    int token_offset;        // added to the sampled index (vocabulary shard offset)
 };
 
 template <int DT>
@@ -208,14 +210,17 @@ __global__ void __launch_bounds__(kThreads, kBlocks) draft_step_kernel(DraftArgs
     const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
     pdl_wait();
     if (a.active && !a.active[row]) return;   // the whole cluster leaves together
-    float u = 0.f;
-    if (!kGreedy && warp == 0) u = __ldg(a.uniforms + row);   // fetched now, used after the stream
+    float u = 0.f, ext = -1.f;
+    if (!kGreedy && warp == 0) {   // fetched now, used after the stream
+        if (a.ext_target) ext = fmaxf(__ldg(a.ext_target + row), 0.f);
+        else u = __ldg(a.uniforms + row);
+    }
     Partial t = reduce_segment<DT, 2, kGreedy>(g, rank * kWarps + warp, a.c, lane, slot0);
     if (lane == 0) { seg[warp].m = t.m; seg[warp].idx = t.idx; seg[warp].Z = t.Z; seg[warp].A = t.A; }
     cluster.sync();
     if (warp == 0) {
         Partial r; SegPick p;
-        combine_segments<2>(cluster, seg, S, a.c, u, lane, r, p);
+        combine_segments<2>(cluster, seg, S, a.c, u, lane, r, p, ext);
         if (lane == 0) { res.row = r; res.pick = p; }
     }
     cluster_arrive();   // done with the peers' shared memory
@@ -227,10 +232,10 @@ __global__ void __launch_bounds__(kThreads, kBlocks) draft_step_kernel(DraftArgs
         float H = 0.f;
         if (ok) H = fmaxf(kLn2 * (log2f(R.Z) - R.A / R.Z), 0.f);
         else atomicOr(a.status, SVIP_STATUS_NONFINITE_ROW);
-        a.entropy[row] = H;
-        a.stop[row] = __fsqrt_rn(H) > a.thresh ? 1 : 0;
+        if (a.entropy) a.entropy[row] = H;
+        if (a.stop) a.stop[row] = __fsqrt_rn(H) > a.thresh ? 1 : 0;
         if (a.row_stats) { a.row_stats[2 * row] = R.m; a.row_stats[2 * row + 1] = R.Z; }
-        if (kGreedy || !ok) a.token[row] = (R.idx >= 0 && R.idx < a.V) ? R.idx : 0;
+        if (kGreedy || !ok) a.token[row] = ((R.idx >= 0 && R.idx < a.V) ? R.idx : 0) + a.token_offset;
     }
     if (!kGreedy && ok && P.seg / kWarps == rank) {
         SoftmaxWeights<DT> wf;
@@ -238,7 +243,7 @@ __global__ void __launch_bounds__(kThreads, kBlocks) draft_step_kernel(DraftArgs
         int v_lo, v_hi;
         seg_range(g, P.seg, v_lo, v_hi);
         int virt = fine_scan<EPV>(wf, v_lo, v_hi, P.prefix, P.target, scan, tid, lane, warp);
-        if (tid == 0) a.token[row] = virt >= 0 ? virt - g.pre : 0;
+        if (tid == 0) a.token[row] = (virt >= 0 ? virt - g.pre : 0) + a.token_offset;
     }
     cluster_wait();     // no block leaves while a peer may still read its shared memory
 }
@@ -257,6 +262,8 @@ struct StatsArgs {
     float2* out_stats;       // (m, Z) per row, indexed by target-row number
     int32_t* out_argmax;
     unsigned* status;
+    float4* out_partial;     // kMode 2: (m, Z, A, index of the maximum + idx_offset as int bits)
+    int idx_offset;
 };
 
 template <int DT, int kMode>
@@ -286,16 +293,20 @@ __global__ void __launch_bounds__(kThreads) row_stats_kernel(StatsArgs a) {
                      static_cast<size_t>(in_row) * a.row_stride * ElemTraits<DT>::kBytes;
     const RowGeom g = make_geom<DT>(rp, a.V, S * kWarps);
     const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
-    Partial t = reduce_segment<DT, kMode, kMode == 0>(g, rank * kWarps + warp, a.c, lane, slot0);
-    if (lane == 0) { seg[warp].m = t.m; seg[warp].idx = t.idx; seg[warp].Z = t.Z; seg[warp].A = 0.f; }
+    Partial t = reduce_segment<DT, kMode, kMode != 1>(g, rank * kWarps + warp, a.c, lane, slot0);
+    if (lane == 0) { seg[warp].m = t.m; seg[warp].idx = t.idx; seg[warp].Z = t.Z; seg[warp].A = t.A; }
     cluster.sync();
     if (rank == 0 && warp == 0) {
         Partial r; SegPick p;
         combine_segments<kMode>(cluster, seg, S, a.c, 0.f, lane, r, p);
         if (lane == 0) {
             bool ok = fabsf(r.m) <= kMaxLogit && (kMode == 0 || r.Z > 0.f);
-            if (!ok) atomicOr(a.status, SVIP_STATUS_NONFINITE_ROW);
-            if (kMode >= 1) a.out_stats[out_row] = make_float2(r.m, r.Z);
+            if (!ok && kMode != 2) atomicOr(a.status, SVIP_STATUS_NONFINITE_ROW);   // a shard may be all masked
+            if (kMode == 1) a.out_stats[out_row] = make_float2(r.m, r.Z);
+            if (kMode == 2) {
+                int gi = ((r.idx >= 0 && r.idx < a.V) ? r.idx : 0) + a.idx_offset;
+                a.out_partial[out_row] = make_float4(r.m, ok ? r.Z : 0.f, ok ? r.A : 0.f, __int_as_float(gi));
+            }
             if (a.out_argmax) a.out_argmax[out_row] = (r.idx >= 0 && r.idx < a.V) ? r.idx : 0;
         }
     }
@@ -740,6 +751,82 @@ __global__ void __launch_bounds__(kThreads) verify_greedy_kernel(GreedyArgs a) {
     }
 }
 
+// ------------------------------------------------------------------ vocabulary-parallel draft step
+//
+// The vocabulary is sharded over G ranks (a tensor-parallel LM head).  Each rank reduces its shard of
+// every row to (m, Z, A, argmax); the ranks exchange these 16 bytes per row; then every rank combines
+// them in rank order -- same inputs, same arithmetic, so all ranks agree bit for bit on the entropy,
+// the stop flag, and on which rank's shard holds the sampled token and how far into its mass.
+
+struct VpCombineArgs {
+    const float4* partials;   // [G][B]
+    int G, B, rank;
+    float c, thresh;
+    int greedy;
+    const float* uniforms;
+    float* entropy;
+    uint8_t* stop;
+    int32_t* token;           // greedy: the global argmax; sampling: -1 (the owner fills it in)
+    int32_t* owner;
+    float* ext_target;
+    uint8_t* active;
+    unsigned* status;
+};
+
+__global__ void __launch_bounds__(kPolicyThreads) vp_combine_kernel(VpCombineArgs a) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int b = blockIdx.x * kPolicyThreads + threadIdx.x;
+    if (b >= a.B) return;
+    float m = neg_inf();
+    for (int g = 0; g < a.G; ++g) m = fmaxf(m, a.partials[static_cast<size_t>(g) * a.B + b].x);
+    const float M = __fmul_rn(m, a.c);
+    float Z = 0.f, A = 0.f;
+    int idx = kIntMax;
+    for (int g = 0; g < a.G; ++g) {
+        const float4 p = a.partials[static_cast<size_t>(g) * a.B + b];
+        if (p.x == m) idx = min(idx, __float_as_int(p.w));
+        if (p.y > 0.f) {
+            float d = __fmul_rn(p.x, a.c) - M;
+            float s = ex2_approx(fmaxf(d, kArgFloor));
+            A += s * __fmaf_rn(d, p.y, p.z);
+            Z += s * p.y;
+        }
+    }
+    const bool ok = Z > 0.f && fabsf(m) <= kMaxLogit;
+    float H = 0.f;
+    if (ok) H = fmaxf(kLn2 * (log2f(Z) - A / Z), 0.f);
+    else atomicOr(a.status, SVIP_STATUS_NONFINITE_ROW);
+    a.entropy[b] = H;
+    a.stop[b] = __fsqrt_rn(H) > a.thresh ? 1 : 0;
+    int owner = -1;
+    float local_target = 0.f;
+    if (!a.greedy && ok) {
+        const float target = a.uniforms[b] * Z;
+        float run = 0.f, before = 0.f;
+        int last = -1;
+        for (int g = 0; g < a.G && owner < 0; ++g) {
+            const float4 p = a.partials[static_cast<size_t>(g) * a.B + b];
+            float mass = 0.f;
+            if (p.y > 0.f) mass = p.y * ex2_approx(fmaxf(__fmul_rn(p.x, a.c) - M, kArgFloor));
+            if (mass > 0.f) {
+                last = g; before = run;
+                if (run + mass > target) owner = g;
+            }
+            run += mass;
+        }
+        if (owner < 0) owner = last;   // rounding: the last shard with mass, searched to its end
+        // the owner looks for (target - before) in units of its own Z, i.e. relative to its own maximum
+        const float4 po = a.partials[static_cast<size_t>(owner) * a.B + b];
+        const float up = ex2_approx(fminf(M - __fmul_rn(po.x, a.c), 126.f));
+        local_target = fminf(fmaxf(target - before, 0.f) * up, po.y);
+    }
+    a.token[b] = a.greedy || !ok ? ((idx != kIntMax) ? idx : 0) : -1;
+    a.owner[b] = owner;
+    a.ext_target[b] = local_target;
+    a.active[b] = owner == a.rank ? 1 : 0;
+}
+
 // ------------------------------------------------------------------ draft-length policies
 //
 // Per-sequence drafting state on the device, so that the loop of Algorithm 1 needs no host round
@@ -1014,7 +1101,8 @@ int svip_create(svip_ctx** out, int device, int max_rows) {
             (const void*)draft_step_kernel<kF32, true, 3>,  (const void*)draft_step_kernel<kF32, false, 3>,
             (const void*)row_stats_kernel<kBF16, 0>,     (const void*)row_stats_kernel<kBF16, 1>,
             (const void*)row_stats_kernel<kF32, 0>,      (const void*)row_stats_kernel<kF32, 1>,
-            (const void*)verify_finish_kernel<kBF16>,    (const void*)verify_finish_kernel<kF32>};
+            (const void*)verify_finish_kernel<kBF16>,    (const void*)verify_finish_kernel<kF32>,
+            (const void*)row_stats_kernel<kBF16, 2>,     (const void*)row_stats_kernel<kF32, 2>};
         for (const void* k : ringed)
             if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes) != cudaSuccess)
                 rc = SVIP_ERR_CUDA;
@@ -1102,6 +1190,7 @@ int svip_draft_step_masked(svip_ctx* ctx, const void* logits, svip_dtype dtype, 
     a.logits = logits; a.row_stride = row_stride; a.V = V; a.c = scale_for(T); a.thresh = thresh;
     a.greedy = T > 0.f ? 0 : 1; a.uniforms = uniforms; a.token = token; a.entropy = entropy;
     a.stop = stop; a.row_stats = row_stats; a.status = ctx->status; a.active = active;
+    a.ext_target = nullptr; a.token_offset = 0;
     int S = pick_cluster(ctx, B, V, dtype);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool waves = static_cast<long>(B) * S > 2L * ctx->num_sms;
@@ -1160,6 +1249,7 @@ int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits
     s.logits = target_logits; s.row_stride = t_row_stride; s.V = V; s.c = c; s.draft_rows = 0; s.K = K;
     s.cu = cu_rows; s.q_seq_stride = q_seq_stride; s.q_pos_stride = q_pos_stride;
     s.out_stats = ctx->p_stats; s.out_argmax = sampling ? nullptr : ctx->p_argmax; s.status = ctx->status;
+    s.out_partial = nullptr; s.idx_offset = 0;
     int S = pick_cluster(ctx, n_target_rows, V, dtype);
     const bool timed = ctx->profiling && !ctx->capturing && ctx->prof_used < kProfilePairs;
     if (timed) cudaEventRecord(ctx->prof_start[ctx->prof_used], st);
@@ -1294,6 +1384,69 @@ int svip_policy_update(svip_ctx* ctx, int policy, const int32_t* n_accepted, int
     return SVIP_OK;
 }
 
+int svip_vp_partial(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, int V_shard, long row_stride,
+                    float T, int vocab_offset, float* partial, void* stream) {
+    if (!ctx || !logits || !partial) return SVIP_ERR_INVALID_ARG;
+    if (dtype != SVIP_F32 && dtype != SVIP_BF16) return SVIP_ERR_UNSUPPORTED;
+    if (B < 0 || V_shard < 1 || V_shard > 0x7fffffe0 || row_stride < 0 || vocab_offset < 0) return SVIP_ERR_INVALID_ARG;
+    if (!(T >= 0.f) || std::isinf(T)) return SVIP_ERR_INVALID_ARG;
+    if (!aligned_to(logits, dtype == SVIP_BF16 ? 2 : 4) || !aligned_to(partial, 16)) return SVIP_ERR_INVALID_ARG;
+    if (B == 0) return SVIP_OK;
+    StatsArgs s;
+    s.logits = logits; s.row_stride = row_stride; s.V = V_shard; s.c = scale_for(T); s.draft_rows = 0; s.K = 1;
+    s.cu = nullptr; s.q_seq_stride = 0; s.q_pos_stride = 0; s.out_stats = nullptr; s.out_argmax = nullptr;
+    s.status = ctx->status; s.out_partial = reinterpret_cast<float4*>(partial); s.idx_offset = vocab_offset;
+    const int S = pick_cluster(ctx, B, V_shard, dtype);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 2>, B, S, s, st, kRingBytes)
+                                       : launch_clustered(row_stats_kernel<kF32, 2>, B, S, s, st, kRingBytes);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    return SVIP_OK;
+}
+
+int svip_vp_combine(svip_ctx* ctx, const float* partials, int G, int rank, int B, float T, float thresh,
+                    const float* uniforms, float* entropy, uint8_t* stop, int32_t* token, int32_t* owner,
+                    float* local_target, uint8_t* active, void* stream) {
+    if (!ctx || !partials || !entropy || !stop || !token || !owner || !local_target || !active)
+        return SVIP_ERR_INVALID_ARG;
+    if (G < 1 || rank < 0 || rank >= G || B < 0) return SVIP_ERR_INVALID_ARG;
+    if (!(T >= 0.f) || std::isinf(T) || std::isnan(thresh) || (T > 0.f && !uniforms)) return SVIP_ERR_INVALID_ARG;
+    if (!aligned_to(partials, 16)) return SVIP_ERR_INVALID_ARG;
+    if (B == 0) return SVIP_OK;
+    VpCombineArgs a;
+    a.partials = reinterpret_cast<const float4*>(partials); a.G = G; a.B = B; a.rank = rank; a.c = scale_for(T);
+    a.thresh = thresh; a.greedy = T > 0.f ? 0 : 1; a.uniforms = uniforms; a.entropy = entropy; a.stop = stop;
+    a.token = token; a.owner = owner; a.ext_target = local_target; a.active = active; a.status = ctx->status;
+    cudaError_t e = launch_ex(vp_combine_kernel, static_cast<unsigned>((B + kPolicyThreads - 1) / kPolicyThreads),
+                              kPolicyThreads, 0, 0, static_cast<cudaStream_t>(stream), a);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    return SVIP_OK;
+}
+
+int svip_vp_locate(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, int V_shard, long row_stride,
+                   float T, const float* local_target, const uint8_t* active, int vocab_offset,
+                   int32_t* token, void* stream) {
+    if (!ctx || !logits || !local_target || !active || !token) return SVIP_ERR_INVALID_ARG;
+    if (dtype != SVIP_F32 && dtype != SVIP_BF16) return SVIP_ERR_UNSUPPORTED;
+    if (B < 0 || V_shard < 1 || V_shard > 0x7fffffe0 || row_stride < 0 || vocab_offset < 0) return SVIP_ERR_INVALID_ARG;
+    if (!(T > 0.f) || std::isinf(T)) return SVIP_ERR_INVALID_ARG;
+    if (!aligned_to(logits, dtype == SVIP_BF16 ? 2 : 4)) return SVIP_ERR_INVALID_ARG;
+    if (B == 0) return SVIP_OK;
+    DraftArgs a;
+    a.logits = logits; a.row_stride = row_stride; a.V = V_shard; a.c = scale_for(T); a.thresh = 0.f; a.greedy = 0;
+    a.uniforms = nullptr; a.token = token; a.entropy = nullptr; a.stop = nullptr; a.row_stats = nullptr;
+    a.status = ctx->status; a.active = active; a.ext_target = local_target; a.token_offset = vocab_offset;
+    const int S = pick_cluster(ctx, B, V_shard, dtype);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = dtype == SVIP_BF16 ? launch_clustered(draft_step_kernel<kBF16, false, 2>, B, S, a, st, kRingBytes)
+                                       : launch_clustered(draft_step_kernel<kF32, false, 2>, B, S, a, st, kRingBytes);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    return SVIP_OK;
+}
+
 int svip_pair_stats(svip_ctx* ctx, const void* q_logits, long q_row_stride, const void* target_logits,
                     long t_row_stride, svip_dtype dtype, int n_pairs, int V, float T, float c_bound,
                     float* out, void* stream) {
@@ -1311,6 +1464,7 @@ int svip_pair_stats(svip_ctx* ctx, const void* q_logits, long q_row_stride, cons
     StatsArgs s;
     s.row_stride = t_row_stride; s.V = V; s.c = c; s.draft_rows = 0; s.K = 1; s.cu = nullptr;
     s.q_seq_stride = 0; s.q_pos_stride = 0; s.out_argmax = nullptr; s.status = ctx->status;
+    s.out_partial = nullptr; s.idx_offset = 0;
     for (int side = 0; side < 2; ++side) {
         s.logits = side == 0 ? target_logits : q_logits;
         s.row_stride = side == 0 ? t_row_stride : q_row_stride;

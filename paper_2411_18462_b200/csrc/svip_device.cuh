@@ -594,8 +594,9 @@ struct SegPick {
 };
 
 // `mass[k]` is the mass of segment lane*per + k (0 beyond nseg).  Warp-collective.
+// The mass to find is u * total, or `abs_target` (same units as the masses) when that is >= 0.
 __device__ __forceinline__ SegPick pick_segment(const float (&mass)[kSegPerLane], int per, int nseg,
-                                                float u, int lane) {
+                                                float u, int lane, float abs_target = -1.f) {
     float run[kSegPerLane];
     float acc = 0.f;
 #pragma unroll
@@ -607,7 +608,7 @@ __device__ __forceinline__ SegPick pick_segment(const float (&mass)[kSegPerLane]
     float before = incl - acc;
     SegPick r;
     r.total = __shfl_sync(0xffffffffu, incl, 31);
-    r.target = u * r.total;
+    r.target = abs_target >= 0.f ? abs_target : u * r.total;
     int cand = kIntMax;
     float cpre = 0.f;
 #pragma unroll
