@@ -32,9 +32,9 @@ METRIC = "logits GB/s (% of B200 HBM peak) for draft-step+verify; us/step at B=1
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of row_stats_kernel<bf16> per algorithmic byte, from an
-# ncu capture of a 1056-row launch (337.1 MB moved for 321.2 MB of logits); traffic grows in
+# ncu capture of a 1056-row launch (332.3 MB moved for 321.2 MB of logits); traffic grows in
 # proportion to the rows, so a full launch is scaled by its bytes
-ROW_STATS_TRAFFIC_PER_ALGORITHMIC_BYTE = 337.14 / 321.16
+ROW_STATS_TRAFFIC_PER_ALGORITHMIC_BYTE = 332.34 / 321.16
 
 
 def describe(w, B=None):
