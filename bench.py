@@ -1,15 +1,17 @@
 #!/usr/bin/env python
 """Throughput of one SVIP speculative-decoding round (draft steps + ragged packing + verify).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload ragged] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload stress] [--impl ours|reference]
 
-A step is one whole round over one batch of the `ragged` workload (B = 128 sequences, V = 152064
-bf16 logits, draft lengths K_i in 1..64 set by the entropy stop rule): one svip_draft_step call per
-draft position over the sequences still drafting, one svip_pack_ragged, one svip_verify.  The
-metric is logits GB/s: bytes of logits the round has to read (every draft row once, every target
-row once, plus the draft row of each rejected position) divided by the device time of the step.
-Prints ONE JSON line on rank 0.  With N > 1 (torchrun) every rank runs its own batch on its own GPU
-(weak scaling, no data-path collective); the time is the max over ranks.
+A step is one whole round over one batch of the workload: one svip_draft_step call per draft
+position over the sequences still drafting, one svip_pack_ragged, one svip_verify.  The default
+workload is `stress`, the largest of the five published configurations that fits one GPU (B = 256
+sequences, V = 256000 fp32 logits, K = 8: 4.7 GB of logits per round); `--workload ragged` is the
+long-form configuration with entropy-driven draft lengths.  The metric is logits GB/s: bytes of logits
+the round has to read (every draft row once, every target row once, plus the draft row of each
+rejected position) divided by the device time of the step.  Prints ONE JSON line on rank 0.  With
+N > 1 (torchrun) every rank runs its own batch on its own GPU (weak scaling, no data-path
+collective); the time is the max over ranks.
 """
 from __future__ import annotations
 
@@ -35,6 +37,9 @@ FALLBACK_HBM_GBS = 6650.0
 # ncu capture of a 1056-row launch (332.3 MB moved for 321.2 MB of logits); traffic grows in
 # proportion to the rows, so a full launch is scaled by its bytes
 ROW_STATS_TRAFFIC_PER_ALGORITHMIC_BYTE = 332.34 / 321.16
+# the same for draft_step_kernel<f32, sampling>, from a capture of 128-row launches (132.2 MB read and
+# 7.0 MB written for 131.1 MB of logits)
+DRAFT_F32_TRAFFIC_PER_ALGORITHMIC_BYTE = 139.17 / 131.07
 
 
 def describe(w, B=None):
@@ -193,9 +198,19 @@ class Round:
                               self.d_cu, B, w.K_max, self.Rp, V, w.T, self.d_uv, self.d_nacc, self.d_next, sp))
         self.calls = calls
 
-    def step(self):
-        for c in self.calls:
+    def step(self, draft_events=None):
+        """One round.  draft_events = (before, after): torch events recorded on the launching stream
+        around the draft-step launches of this round."""
+        if draft_events is None:
+            for c in self.calls:
+                c()
+            return
+        draft_events[0].record()
+        for c in self.calls[:-2]:
             c()
+        draft_events[1].record()
+        self.calls[-2]()
+        self.calls[-1]()
 
     def logits_bytes(self):
         """Algorithmic logits bytes of one step (needs the results of a finished step)."""
@@ -263,7 +278,9 @@ def cpu_baseline(w, seconds_budget=20.0):
     """The fp64 oracle, as it stands, on a bounded sample of the same workload, on all host cores."""
     from oracle import svip_oracle as O
     cores = len(os.sched_getaffinity(0))
-    n_seq = min(w.B, 64)
+    # about 4500 rows: 10-20 s of CPU work
+    rows_per_seq = 2.0 * float(w.draft_len.mean()) + 1.0
+    n_seq = min(w.B, max(64, int(round(4500.0 / rows_per_seq))))
     sel = list(range(n_seq))
     rows_q = np.concatenate([np.arange(w.cu_rows[i] - i, w.cu_rows[i] - i + w.draft_len[i]) for i in sel])
     rows_t = np.concatenate([np.arange(w.cu_rows[i], w.cu_rows[i + 1]) for i in sel])
@@ -298,7 +315,8 @@ def run_ours(args):
     if build.is_stale():
         build.build()
     spec = workloads.SPECS[args.workload]
-    w = workloads.make_workload(args.workload, seed=sharding.rank_seed(workloads.BASE_SEED + spec["index"], rank))
+    w = workloads.make_workload(args.workload, seed=sharding.rank_seed(workloads.BASE_SEED + spec["index"], rank),
+                                B=args.batch)
     ctx = Context(dev, max(1 << 14, w.n_target_rows))
     stream = torch.cuda.current_stream()
     rnd = Round(ctx, w, torch, stream.cuda_stream)
@@ -318,13 +336,16 @@ def run_ours(args):
     torch.cuda.synchronize()
     sampler.start()
     launches0 = ctx.launch_count()
+    n_timed = min(args.steps, 1024)
+    draft_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_timed)]
     e0.record(stream)
-    for _ in range(args.steps):
-        rnd.step()
+    for k in range(args.steps):
+        rnd.step(draft_ev[k] if k < n_timed else None)
     e1.record(stream)
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
+    draft_ms = sum(a.elapsed_time(b) for a, b in draft_ev)
     launches = ctx.launch_count() - launches0
     clocks = sampler.stop()
     local_ms = e0.elapsed_time(e1)
@@ -355,8 +376,32 @@ def run_ours(args):
         return
     peak, peak_kind = measured_peak()
     value = total_bytes / (total_ms * 1e-3) / 1e9
+    # the two streaming kernels, each timed live inside the timed region: the row-statistics kernel by
+    # the library's own event pair around its launch, the draft-step kernel as the mean over the
+    # launches of a round (events around the draft launches: launch gaps are inside)
     stats_bytes = w.n_target_rows * w.V * w.elem_bytes
-    achieved = stats_bytes / (stats_ms / max(stats_n, 1) * 1e-3) / 1e9 if stats_n else None
+    stats_gbs = stats_bytes / (stats_ms / max(stats_n, 1) * 1e-3) / 1e9 if stats_n else None
+    n_draft = rnd.K
+    draft_bytes = w.n_draft_rows * w.V * w.elem_bytes / n_draft
+    draft_us = draft_ms * 1e3 / max(n_timed * n_draft, 1)
+    draft_gbs = draft_bytes / (draft_us * 1e-6) / 1e9
+    dt_name = "bf16" if w.dtype == "bf16" else "f32"
+    roof_stats = {"bound": "hbm", "kernel": "row_stats_kernel<%s> (target rows of svip_verify)" % dt_name,
+                  "achieved": stats_gbs, "peak": peak, "peak_kind": "%s copy bandwidth" % peak_kind, "unit": "GB/s",
+                  "frac": (stats_gbs / peak) if stats_gbs else None, "launches_timed": stats_n,
+                  "bytes_per_launch": stats_bytes, "us_per_launch": stats_ms * 1e3 / max(stats_n, 1),
+                  "share_of_step": stats_ms / max(stats_n, 1) / (total_ms / args.steps),
+                  "traffic": ROW_STATS_TRAFFIC_PER_ALGORITHMIC_BYTE * stats_bytes if w.dtype == "bf16" else None}
+    roof_draft = {"bound": "hbm", "kernel": "draft_step_kernel<%s, sampling> (mean over the %d launches of a round)"
+                  % (dt_name, n_draft), "achieved": draft_gbs, "peak": peak,
+                  "peak_kind": "%s copy bandwidth" % peak_kind, "unit": "GB/s", "frac": draft_gbs / peak,
+                  "launches_timed": n_timed * n_draft, "bytes_per_launch": draft_bytes, "us_per_launch": draft_us,
+                  "share_of_step": draft_ms / n_timed / (total_ms / args.steps),
+                  "traffic": DRAFT_F32_TRAFFIC_PER_ALGORITHMIC_BYTE * draft_bytes
+                  if (w.dtype == "f32" and DRAFT_F32_TRAFFIC_PER_ALGORITHMIC_BYTE) else None}
+    # `roofline` is the kernel with the larger share of the step; the other one rides along
+    dominant, other = (roof_draft, roof_stats) if roof_draft["share_of_step"] >= roof_stats["share_of_step"] \
+        else (roof_stats, roof_draft)
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
@@ -365,15 +410,11 @@ def run_ours(args):
                    "target_rows": w.n_target_rows, "rejected_sequences": rejected,
                    "logits_bytes_per_step": step_bytes, "l2": "inputs (%.2f GB per step) larger than L2, no flush" % (step_bytes / 1e9),
                    "launch": "one stream, %d kernels per step" % (launches // max(args.steps, 1)),
-                   "stop_flags_match_draft_lengths": bool(stops_ok), "status_word": status},
+                   "stop_flags_match_draft_lengths": bool(stops_ok) if w.name == "ragged" else None,
+                   "status_word": status},
         "pct_of_hbm_peak_nominal": 100.0 * value / world / NOMINAL_HBM_GBS,
         "pct_of_hbm_peak_measured": 100.0 * value / world / peak,
-        "roofline": {"bound": "hbm", "kernel": "row_stats_kernel<bf16> (target rows of svip_verify)",
-                     "achieved": achieved, "peak": peak, "peak_kind": "%s copy bandwidth" % peak_kind,
-                     "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
-                     "launches_timed": stats_n, "bytes_per_launch": stats_bytes,
-                     "traffic": ROW_STATS_TRAFFIC_PER_ALGORITHMIC_BYTE * stats_bytes
-                     if w.dtype == "bf16" else None},
+        "roofline": dominant, "roofline_other": other,
         "e2e": {"value": (e2e_bytes / (e2e_ms * 1e-3) / 1e9) if e2e_steps else None, "unit": "GB/s",
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": launches, "clocks": clocks,
@@ -434,9 +475,11 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="ragged", choices=sorted(workloads.SPECS))
+    ap.add_argument("--workload", default="stress", choices=sorted(workloads.SPECS))
+    ap.add_argument("--batch", type=int, default=None,
+                    help="sequences per GPU instead of the published batch size (smaller cases for profiling)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--skip-extras", action="store_true",
