@@ -270,6 +270,50 @@ def b1_latency(ctx, torch):
             st.synchronize()
             out[name] = 1000.0 * e0.elapsed_time(e1) / reps
         g.destroy(); one.destroy()
+
+        # the drafting phase as a loop inside the graph (each token: draft step at the sequence's own
+        # position + the policy kernel that also decides the loop), against the same two kernels
+        # driven from the host, which must read the count of drafting sequences back after every token
+        gamma = torch.tensor([K], dtype=torch.int32, device="cuda"); dlen = torch.zeros(1, dtype=torch.int32, device="cuda")
+        act = torch.ones(1, dtype=torch.uint8, device="cuda"); nact = torch.zeros(1, dtype=torch.int32, device="cuda")
+        stop1 = torch.zeros(1, dtype=torch.uint8, device="cuda")
+        st.synchronize()
+        CONSTANT = 1
+        ctx.graph_begin(st)
+        ctx.policy_update(CONSTANT, None, dlen, gamma, act, 1, K, st)
+        body = ctx.graph_loop_begin(st, nact, K)
+        ctx.draft_step_at(dq, 0, 1, V, V, V, dlen, 1, w.T, w.h, ud, act, tok, ent, stop1, stats, body)
+        ctx.policy_advance(CONSTANT, stop1, gamma, dlen, act, 1, K, nact, body)
+        ctx.graph_loop_end()
+        loop = ctx.graph_end(st)
+        for _ in range(20):
+            loop.launch(st)
+        st.synchronize()
+        assert int(dlen.item()) == K
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(st)
+        for _ in range(200):
+            loop.launch(st)
+        e1.record(st)
+        st.synchronize()
+        out["draft_loop_us_per_token"] = 1000.0 * e0.elapsed_time(e1) / 200 / K
+        loop.destroy()
+
+        def host_loop():
+            ctx.policy_update(CONSTANT, None, dlen, gamma, act, 1, K, st)
+            n = 0
+            while True:
+                ctx.draft_step_at(dq, 0, 1, V, V, V, dlen, 1, w.T, w.h, ud, act, tok, ent, stop1, stats, st)
+                ctx.policy_advance(CONSTANT, stop1, gamma, dlen, act, 1, K, nact, st)
+                n += 1
+                if int(nact.item()) == 0:      # device -> host read, once per token
+                    return n
+        for _ in range(5):
+            host_loop()
+        t0 = time.perf_counter()
+        n = sum(host_loop() for _ in range(50))
+        st.synchronize()
+        out["host_loop_us_per_token"] = 1e6 * (time.perf_counter() - t0) / n
     out["kernels_per_round"] = K + 3
     return out
 

@@ -137,6 +137,26 @@ int svip_draft_step_masked(svip_ctx* ctx, const void* logits, svip_dtype dtype, 
                            float* row_stats, void* stream);
 
 /*
+ * svip_draft_step_masked over a buffer that holds the logits of all draft
+ * positions of a round, with the position taken from device memory: sequence b
+ * reads the row that starts at element b*row_stride + pos[b]*pos_stride, takes
+ * its uniform from uniforms[pos[b]*slot_stride + b] and writes token, entropy
+ * and row_stats (two floats) at that same index pos[b]*slot_stride + b; stop[b]
+ * is indexed by sequence alone.  With pos = the draft_len array of
+ * svip_policy_advance, a position-major buffer [K_max][B][V] (pos_stride =
+ * B*V, slot_stride = B) is filled slot by slot as Algorithm 1's inner loop
+ * advances, each sequence at its own length, and svip_verify then reads the
+ * rows, tokens and row_stats with q_seq_stride = 1, q_pos_stride = B.
+ * `pos` is DEVICE [B] int32 (values >= 0; the caller keeps them below the
+ * buffer's positions, e.g. through K_cap of svip_policy_advance); NULL means
+ * position 0 for every sequence, i.e. svip_draft_step_masked.
+ */
+int svip_draft_step_at(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, int V,
+                       long row_stride, long pos_stride, const int32_t* pos, long slot_stride,
+                       float T, float thresh, const float* uniforms, const uint8_t* active,
+                       int32_t* token, float* entropy, uint8_t* stop, float* row_stats, void* stream);
+
+/*
  * Draft-length policies, kept on the device so that the drafting loop needs no
  * host round trip per token.
  *   SVIP_POLICY_ENTROPY    the paper's rule: a sequence stops drafting when the
@@ -305,6 +325,31 @@ int svip_graph_begin(svip_ctx* ctx, void* stream);
 int svip_graph_end(svip_ctx* ctx, void* stream, svip_graph** graph);
 int svip_graph_launch(svip_graph* graph, void* stream);
 int svip_graph_destroy(svip_graph* graph);
+
+/*
+ * The drafting loop of Algorithm 1 ("draft a token, stop when the entropy test
+ * fires") as a loop inside the recorded graph, so that one replay drafts a
+ * whole round without the host reading a stop flag per token.
+ *
+ * svip_graph_loop_begin, between svip_graph_begin and svip_graph_end on the
+ * same `stream`: everything recorded on `stream` so far runs before the loop,
+ * everything recorded on it afterwards runs after the loop.  *body_stream
+ * receives a stream owned by the context; every call issued on it (this
+ * library's, or the caller's own kernels, e.g. the draft model's forward) until
+ * svip_graph_loop_end becomes the loop body.  At replay the body runs once,
+ * then again while *n_active > 0 (DEVICE int32, read after the body: the
+ * counter that svip_policy_advance writes), and in no case more than
+ * `max_iters` times.  If the body holds an svip_policy_advance with this
+ * `n_active`, that kernel takes the decision itself; otherwise
+ * svip_graph_loop_end appends a one-thread kernel that does.
+ * One loop at a time (no nesting); svip_graph_end on a graph whose loop body
+ * was not closed, or could not be recorded, returns SVIP_ERR_STATE and hands
+ * out no graph.  Calls inside the body must come from the thread that opened
+ * it.  The paper has no counterpart beyond the loop of Algorithm 1 itself.
+ */
+int svip_graph_loop_begin(svip_ctx* ctx, void* stream, const int32_t* n_active, int max_iters,
+                          void** body_stream);
+int svip_graph_loop_end(svip_ctx* ctx);
 
 /*
  * svip_verify for callers that must not allocate device memory.

@@ -73,6 +73,12 @@ def library():
     L.svip_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_long)]
     L.svip_draft_step_masked.restype = i32
     L.svip_draft_step_masked.argtypes = [vp, vp, i32, i32, i32, lng, f32, f32, vp, vp, vp, vp, vp, vp, vp]
+    L.svip_draft_step_at.restype = i32
+    L.svip_draft_step_at.argtypes = [vp, vp, i32, i32, i32, lng, lng, vp, lng, f32, f32, vp, vp, vp, vp, vp, vp, vp]
+    L.svip_graph_loop_begin.restype = i32
+    L.svip_graph_loop_begin.argtypes = [vp, vp, vp, i32, C.POINTER(vp)]
+    L.svip_graph_loop_end.restype = i32
+    L.svip_graph_loop_end.argtypes = [vp]
     L.svip_policy_advance.restype = i32
     L.svip_policy_advance.argtypes = [vp, i32, vp, vp, vp, vp, i32, i32, vp, vp]
     L.svip_policy_update.restype = i32
@@ -190,6 +196,13 @@ class Context:
                                                 _ptr(entropy), _ptr(stop), _ptr(row_stats), _stream(stream)),
                self._h)
 
+    def draft_step_at(self, logits, dtype, B, V, row_stride, pos_stride, pos, slot_stride, T, thresh, uniforms,
+                      active, token, entropy, stop, row_stats=None, stream=None):
+        _check(library().svip_draft_step_at(self._h, _ptr(logits), int(dtype), int(B), int(V), int(row_stride),
+                                            int(pos_stride), _ptr(pos), int(slot_stride), float(T), float(thresh),
+                                            _ptr(uniforms), _ptr(active), _ptr(token), _ptr(entropy), _ptr(stop),
+                                            _ptr(row_stats), _stream(stream)), self._h)
+
     def policy_advance(self, policy, stop, gamma, draft_len, active, B, K_cap, n_active=None, stream=None):
         _check(library().svip_policy_advance(self._h, int(policy), _ptr(stop), _ptr(gamma), _ptr(draft_len),
                                              _ptr(active), int(B), int(K_cap), _ptr(n_active), _stream(stream)),
@@ -265,6 +278,16 @@ class Context:
 
     def graph_begin(self, stream):
         _check(library().svip_graph_begin(self._h, _stream(stream)), self._h)
+
+    def graph_loop_begin(self, stream, n_active, max_iters) -> int:
+        """Opens the loop body; returns the raw stream handle on which the body is recorded."""
+        body = C.c_void_p()
+        _check(library().svip_graph_loop_begin(self._h, _stream(stream), _ptr(n_active), int(max_iters),
+                                               C.byref(body)), self._h)
+        return int(body.value)
+
+    def graph_loop_end(self):
+        _check(library().svip_graph_loop_end(self._h), self._h)
 
     def graph_end(self, stream) -> Graph:
         g = C.c_void_p()

@@ -167,6 +167,9 @@ struct DraftArgs {
     const uint8_t* active;   // NULL, or one flag per row: rows with 0 are skipped
     const float* ext_target; // NULL, or per row the mass to find (units of this row's own Z), see svip_vp_locate
     int token_offset;        // added to the sampled index (vocabulary shard offset)
+    const int32_t* pos;      // NULL, or per row the draft position p whose logits are read (svip_draft_step_at)
+    long pos_stride;         // elements between the logits of consecutive positions of a row
+    long slot_stride;        // uniforms / token / entropy / row_stats live at index p * slot_stride + row
 };
 
 template <int DT>
@@ -190,7 +193,8 @@ struct RowShared {
 // kBlocks is the number of blocks the register budget must leave room for on one SM: 2 for
 // launches that fit the GPU in one wave (latency matters, registers are free), 3 for launches of
 // many waves, where a third resident block streams on while another one is in its epilogue.
-template <int DT, bool kGreedy, int kBlocks>
+// kPos compiles the position-indexed form (svip_draft_step_at) in.
+template <int DT, bool kGreedy, int kBlocks, bool kPos = false>
 __global__ void __launch_bounds__(kThreads, kBlocks) draft_step_kernel(DraftArgs a) {
     constexpr int EPV = ElemTraits<DT>::kEPV;
     extern __shared__ uint4 ring[];
@@ -206,14 +210,20 @@ __global__ void __launch_bounds__(kThreads, kBlocks) draft_step_kernel(DraftArgs
     pdl_launch_dependents();
     const char* rp = static_cast<const char*>(a.logits) +
                      static_cast<size_t>(row) * a.row_stride * ElemTraits<DT>::kBytes;
-    const RowGeom g = make_geom<DT>(rp, a.V, S * kWarps);
+    RowGeom g = make_geom<DT>(rp, a.V, S * kWarps);
     const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
     pdl_wait();
     if (a.active && !a.active[row]) return;   // the whole cluster leaves together
+    long p = 0;
+    if (kPos) {
+        p = a.pos[row];
+        rp += p * a.pos_stride * ElemTraits<DT>::kBytes;
+        g = make_geom<DT>(rp, a.V, S * kWarps);
+    }
     float u = 0.f, ext = -1.f;
     if (!kGreedy && warp == 0) {   // fetched now, used after the stream
         if (a.ext_target) ext = fmaxf(__ldg(a.ext_target + row), 0.f);
-        else u = __ldg(a.uniforms + row);
+        else u = __ldg(a.uniforms + (row + p * a.slot_stride));
     }
     Partial t = reduce_segment<DT, 2, kGreedy>(g, rank * kWarps + warp, a.c, lane, slot0);
     if (lane == 0) { seg[warp].m = t.m; seg[warp].idx = t.idx; seg[warp].Z = t.Z; seg[warp].A = t.A; }
@@ -228,14 +238,17 @@ __global__ void __launch_bounds__(kThreads, kBlocks) draft_step_kernel(DraftArgs
     const Partial R = res.row;
     const SegPick P = res.pick;
     const bool ok = (R.Z > 0.f) && (fabsf(R.m) <= kMaxLogit);
+    // where this row's outputs live (the position is read again rather than kept across the stream)
+    long slot = row;
+    if (kPos && tid == 0) slot += a.pos[row] * a.slot_stride;
     if (rank == 0 && tid == 0) {
         float H = 0.f;
         if (ok) H = fmaxf(kLn2 * (log2f(R.Z) - R.A / R.Z), 0.f);
         else atomicOr(a.status, SVIP_STATUS_NONFINITE_ROW);
-        if (a.entropy) a.entropy[row] = H;
+        if (a.entropy) a.entropy[slot] = H;
         if (a.stop) a.stop[row] = __fsqrt_rn(H) > a.thresh ? 1 : 0;
-        if (a.row_stats) { a.row_stats[2 * row] = R.m; a.row_stats[2 * row + 1] = R.Z; }
-        if (kGreedy || !ok) a.token[row] = ((R.idx >= 0 && R.idx < a.V) ? R.idx : 0) + a.token_offset;
+        if (a.row_stats) { a.row_stats[2 * slot] = R.m; a.row_stats[2 * slot + 1] = R.Z; }
+        if (kGreedy || !ok) a.token[slot] = ((R.idx >= 0 && R.idx < a.V) ? R.idx : 0) + a.token_offset;
     }
     if (!kGreedy && ok && P.seg / kWarps == rank) {
         SoftmaxWeights<DT> wf;
@@ -243,7 +256,7 @@ __global__ void __launch_bounds__(kThreads, kBlocks) draft_step_kernel(DraftArgs
         int v_lo, v_hi;
         seg_range(g, P.seg, v_lo, v_hi);
         int virt = fine_scan<EPV>(wf, v_lo, v_hi, P.prefix, P.target, scan, tid, lane, warp);
-        if (tid == 0) a.token[row] = (virt >= 0 ? virt - g.pre : 0) + a.token_offset;
+        if (tid == 0) a.token[slot] = (virt >= 0 ? virt - g.pre : 0) + a.token_offset;
     }
     cluster_wait();     // no block leaves while a peer may still read its shared memory
 }
@@ -833,6 +846,22 @@ __global__ void __launch_bounds__(kPolicyThreads) vp_combine_kernel(VpCombineArg
 // trip per draft token.  ENTROPY is the paper's rule (Eq. 7 flag from the draft step); CONSTANT and
 // HEURISTIC are the two baselines of Section 3.
 
+// Control of a drafting loop recorded as a WHILE node of a CUDA graph.  The kernel that closes an
+// iteration counts it and tells the graph whether the body runs again: only while sequences are
+// still drafting, and never more than `max_iters` times whatever the data say.
+struct LoopCtl {
+    cudaGraphConditionalHandle handle;
+    int* iter;        // iterations done since the loop was entered (NULL: not inside a loop)
+    int max_iters;
+};
+
+__device__ __forceinline__ void loop_decide(const LoopCtl& loop, int n_active) {
+    if (!loop.iter) return;
+    const int it = *loop.iter + 1;
+    *loop.iter = it;
+    cudaGraphSetConditional(loop.handle, (n_active > 0 && it < loop.max_iters) ? 1u : 0u);
+}
+
 struct AdvanceArgs {
     int policy;
     const uint8_t* stop;
@@ -841,6 +870,7 @@ struct AdvanceArgs {
     uint8_t* active;
     int B, K_cap;
     int32_t* n_active;
+    LoopCtl loop;
 };
 
 __global__ void __launch_bounds__(kPolicyThreads) policy_advance_kernel(AdvanceArgs a) {
@@ -862,7 +892,17 @@ __global__ void __launch_bounds__(kPolicyThreads) policy_advance_kernel(AdvanceA
     }
     if (mine) atomicAdd(&count, mine);
     __syncthreads();
-    if (threadIdx.x == 0 && a.n_active) *a.n_active = count;
+    if (threadIdx.x == 0) {
+        if (a.n_active) *a.n_active = count;
+        loop_decide(a.loop, count);
+    }
+}
+
+// Decision of a drafting loop whose body holds no svip_policy_advance on the loop's counter.
+__global__ void loop_decide_kernel(LoopCtl loop, const int32_t* n_active) {
+    pdl_launch_dependents();
+    pdl_wait();
+    if (threadIdx.x == 0) loop_decide(loop, *n_active);
 }
 
 struct UpdateArgs {
@@ -967,6 +1007,13 @@ struct svip_ctx {
     float2* q_stats;
     int32_t* p_argmax;
     unsigned* status;
+    int* loop_iter;            // device: iteration counter of the drafting loop being replayed
+    cudaStream_t loop_stream;  // records the body of a drafting loop
+    int loop_open;             // a loop body is being recorded
+    int loop_decided;          // the body already holds the kernel that decides the loop
+    int loop_failed;           // a loop of the graph being recorded is not closed properly
+    LoopCtl loop;
+    const int32_t* loop_n_active;
     int profiling;
     int prof_used;
     cudaEvent_t* prof_start;
@@ -987,6 +1034,10 @@ const bool g_use_pdl = [] {
     const char* v = std::getenv("SVIP_NO_PDL");
     return !(v && v[0] == '1');
 }();
+
+// Set while the calling thread records the body of a drafting loop: kernels inside a conditional
+// node are launched without the programmatic-serialization attribute.
+thread_local bool t_plain_launches = false;
 
 int cuda_fail(svip_ctx* ctx, cudaError_t e) {
     if (ctx) ctx->last_cuda = static_cast<int>(e);
@@ -1013,7 +1064,7 @@ cudaError_t launch_ex(void (*kernel)(KArgs...), unsigned grid, unsigned block, i
         attr[n].val.clusterDim.z = 1;
         ++n;
     }
-    if (g_use_pdl) {
+    if (g_use_pdl && !t_plain_launches) {
         attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[n].val.programmaticStreamSerializationAllowed = 1;
         ++n;
@@ -1099,6 +1150,8 @@ int svip_create(svip_ctx** out, int device, int max_rows) {
             (const void*)draft_step_kernel<kF32, true, 2>,  (const void*)draft_step_kernel<kF32, false, 2>,
             (const void*)draft_step_kernel<kBF16, true, 3>, (const void*)draft_step_kernel<kBF16, false, 3>,
             (const void*)draft_step_kernel<kF32, true, 3>,  (const void*)draft_step_kernel<kF32, false, 3>,
+            (const void*)draft_step_kernel<kBF16, true, 2, true>, (const void*)draft_step_kernel<kBF16, false, 2, true>,
+            (const void*)draft_step_kernel<kF32, true, 2, true>,  (const void*)draft_step_kernel<kF32, false, 2, true>,
             (const void*)row_stats_kernel<kBF16, 0>,     (const void*)row_stats_kernel<kBF16, 1>,
             (const void*)row_stats_kernel<kF32, 0>,      (const void*)row_stats_kernel<kF32, 1>,
             (const void*)verify_finish_kernel<kBF16>,    (const void*)verify_finish_kernel<kF32>,
@@ -1113,13 +1166,16 @@ int svip_create(svip_ctx** out, int device, int max_rows) {
             cudaMalloc(&c->q_stats, n * sizeof(float2)) != cudaSuccess ||
             cudaMalloc(&c->p_argmax, n * sizeof(int32_t)) != cudaSuccess ||
             cudaMalloc(&c->status, sizeof(unsigned)) != cudaSuccess ||
-            cudaMemset(c->status, 0, sizeof(unsigned)) != cudaSuccess) {
+            cudaMemset(c->status, 0, sizeof(unsigned)) != cudaSuccess ||
+            cudaMalloc(&c->loop_iter, sizeof(int)) != cudaSuccess ||
+            cudaMemset(c->loop_iter, 0, sizeof(int)) != cudaSuccess) {
             rc = SVIP_ERR_CUDA;
         }
     }
     if (rc != SVIP_OK) {
         cudaGetLastError();
         cudaFree(c->p_stats); cudaFree(c->q_stats); cudaFree(c->p_argmax); cudaFree(c->status);
+        cudaFree(c->loop_iter);
         delete c;
     } else {
         *out = c;
@@ -1134,6 +1190,8 @@ int svip_destroy(svip_ctx* ctx) {
     cudaGetDevice(&prev);
     cudaSetDevice(ctx->device);
     cudaFree(ctx->p_stats); cudaFree(ctx->q_stats); cudaFree(ctx->p_argmax); cudaFree(ctx->status);
+    cudaFree(ctx->loop_iter);
+    if (ctx->loop_stream) cudaStreamDestroy(ctx->loop_stream);
     if (ctx->prof_start) {
         for (int k = 0; k < kProfilePairs; ++k) {
             cudaEventDestroy(ctx->prof_start[k]);
@@ -1179,7 +1237,16 @@ int svip_draft_step(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, 
 int svip_draft_step_masked(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, int V, long row_stride,
                            float T, float thresh, const float* uniforms, const uint8_t* active,
                            int32_t* token, float* entropy, uint8_t* stop, float* row_stats, void* stream) {
+    return svip_draft_step_at(ctx, logits, dtype, B, V, row_stride, 0, nullptr, 0, T, thresh, uniforms, active,
+                              token, entropy, stop, row_stats, stream);
+}
+
+int svip_draft_step_at(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, int V, long row_stride,
+                       long pos_stride, const int32_t* pos, long slot_stride, float T, float thresh,
+                       const float* uniforms, const uint8_t* active, int32_t* token, float* entropy,
+                       uint8_t* stop, float* row_stats, void* stream) {
     if (!ctx || !logits || !token || !entropy || !stop) return SVIP_ERR_INVALID_ARG;
+    if (pos_stride < 0 || slot_stride < 0) return SVIP_ERR_INVALID_ARG;
     if (dtype != SVIP_F32 && dtype != SVIP_BF16) return SVIP_ERR_UNSUPPORTED;
     if (B < 0 || V < 1 || V > 0x7fffffe0 || row_stride < 0) return SVIP_ERR_INVALID_ARG;
     if (!(T >= 0.f) || std::isinf(T) || std::isnan(thresh)) return SVIP_ERR_INVALID_ARG;
@@ -1191,6 +1258,7 @@ int svip_draft_step_masked(svip_ctx* ctx, const void* logits, svip_dtype dtype, 
     a.greedy = T > 0.f ? 0 : 1; a.uniforms = uniforms; a.token = token; a.entropy = entropy;
     a.stop = stop; a.row_stats = row_stats; a.status = ctx->status; a.active = active;
     a.ext_target = nullptr; a.token_offset = 0;
+    a.pos = pos; a.pos_stride = pos_stride; a.slot_stride = slot_stride;
     int S = pick_cluster(ctx, B, V, dtype);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool waves = static_cast<long>(B) * S > 2L * ctx->num_sms;
@@ -1201,6 +1269,10 @@ int svip_draft_step_masked(svip_ctx* ctx, const void* logits, svip_dtype dtype, 
     else
         k = a.greedy ? (waves ? draft_step_kernel<kF32, true, 3> : draft_step_kernel<kF32, true, 2>)
                      : (waves ? draft_step_kernel<kF32, false, 3> : draft_step_kernel<kF32, false, 2>);
+    if (pos) {
+        if (dtype == SVIP_BF16) k = a.greedy ? draft_step_kernel<kBF16, true, 2, true> : draft_step_kernel<kBF16, false, 2, true>;
+        else k = a.greedy ? draft_step_kernel<kF32, true, 2, true> : draft_step_kernel<kF32, false, 2, true>;
+    }
     cudaError_t e = launch_clustered(k, B, S, a, st, kRingBytes);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
@@ -1361,8 +1433,13 @@ int svip_policy_advance(svip_ctx* ctx, int policy, const uint8_t* stop, const in
     AdvanceArgs a;
     a.policy = policy; a.stop = stop; a.gamma = gamma; a.draft_len = draft_len; a.active = active;
     a.B = B; a.K_cap = K_cap; a.n_active = n_active;
+    a.loop.iter = nullptr; a.loop.max_iters = 0; a.loop.handle = 0;
+    const bool decides = ctx->loop_open && n_active && n_active == ctx->loop_n_active &&
+                         static_cast<cudaStream_t>(stream) == ctx->loop_stream;
+    if (decides) a.loop = ctx->loop;
     cudaError_t e = launch_ex(policy_advance_kernel, 1, kPolicyThreads, 0, 0, static_cast<cudaStream_t>(stream), a);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
+    if (decides) ctx->loop_decided = 1;
     ctx->launches += 1;
     return SVIP_OK;
 }
@@ -1438,6 +1515,7 @@ int svip_vp_locate(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, i
     a.logits = logits; a.row_stride = row_stride; a.V = V_shard; a.c = scale_for(T); a.thresh = 0.f; a.greedy = 0;
     a.uniforms = nullptr; a.token = token; a.entropy = nullptr; a.stop = nullptr; a.row_stats = nullptr;
     a.status = ctx->status; a.active = active; a.ext_target = local_target; a.token_offset = vocab_offset;
+    a.pos = nullptr; a.pos_stride = 0; a.slot_stride = 0;
     const int S = pick_cluster(ctx, B, V_shard, dtype);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = dtype == SVIP_BF16 ? launch_clustered(draft_step_kernel<kBF16, false, 2>, B, S, a, st, kRingBytes)
@@ -1488,18 +1566,101 @@ int svip_pair_stats(svip_ctx* ctx, const void* q_logits, long q_row_stride, cons
 int svip_graph_begin(svip_ctx* ctx, void* stream) {
     if (!ctx) return SVIP_ERR_INVALID_ARG;
     if (ctx->capturing) return SVIP_ERR_STATE;
-    cudaError_t e = cudaStreamBeginCapture(static_cast<cudaStream_t>(stream), cudaStreamCaptureModeThreadLocal);
+    cudaError_t e = cudaSuccess;
+    if (!ctx->loop_stream) {   // made now: no stream is created while a capture is open
+        e = cudaStreamCreateWithFlags(&ctx->loop_stream, cudaStreamNonBlocking);
+        if (e != cudaSuccess) { ctx->loop_stream = nullptr; return cuda_fail(ctx, e); }
+    }
+    e = cudaStreamBeginCapture(static_cast<cudaStream_t>(stream), cudaStreamCaptureModeThreadLocal);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->capturing = 1;
+    return SVIP_OK;
+}
+
+int svip_graph_loop_begin(svip_ctx* ctx, void* stream, const int32_t* n_active, int max_iters, void** body_stream) {
+    if (!ctx || !n_active || !body_stream || max_iters < 1) return SVIP_ERR_INVALID_ARG;
+    if (!ctx->capturing || ctx->loop_open) return SVIP_ERR_STATE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the iteration counter starts at zero at every replay
+    cudaError_t e = cudaMemsetAsync(ctx->loop_iter, 0, sizeof(int), st);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    cudaStreamCaptureStatus status = cudaStreamCaptureStatusNone;
+    cudaGraph_t graph = nullptr;
+    const cudaGraphNode_t* deps = nullptr;
+    size_t n_deps = 0;
+    e = cudaStreamGetCaptureInfo(st, &status, nullptr, &graph, &deps, &n_deps);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    if (status != cudaStreamCaptureStatusActive || !graph) return SVIP_ERR_STATE;
+    // the body runs once before the first decision (the do-while of Algorithm 1): default value 1
+    cudaGraphConditionalHandle handle;
+    e = cudaGraphConditionalHandleCreate(&handle, graph, 1, cudaGraphCondAssignDefault);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    cudaGraphNodeParams params = {};
+    params.type = cudaGraphNodeTypeConditional;
+    params.conditional.handle = handle;
+    params.conditional.type = cudaGraphCondTypeWhile;
+    params.conditional.size = 1;
+    cudaGraphNode_t node = nullptr;
+    e = cudaGraphAddNode(&node, graph, deps, n_deps, &params);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    cudaGraph_t body = params.conditional.phGraph_out[0];
+    // from here on the graph holds a loop: if its body cannot be recorded, svip_graph_end refuses
+    // to hand the graph out (a loop without a deciding kernel would never end)
+    // what is recorded on `stream` from here on comes after the loop
+    e = cudaStreamUpdateCaptureDependencies(st, &node, 1, cudaStreamSetCaptureDependencies);
+    if (e != cudaSuccess) { ctx->loop_failed = 1; return cuda_fail(ctx, e); }
+    e = cudaStreamBeginCaptureToGraph(ctx->loop_stream, body, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal);
+    if (e != cudaSuccess) { ctx->loop_failed = 1; return cuda_fail(ctx, e); }
+    ctx->loop.handle = handle;
+    ctx->loop.iter = ctx->loop_iter;
+    ctx->loop.max_iters = max_iters;
+    ctx->loop_n_active = n_active;
+    ctx->loop_open = 1;
+    ctx->loop_decided = 0;
+    t_plain_launches = true;
+    *body_stream = ctx->loop_stream;
+    return SVIP_OK;
+}
+
+int svip_graph_loop_end(svip_ctx* ctx) {
+    if (!ctx) return SVIP_ERR_INVALID_ARG;
+    if (!ctx->loop_open) return SVIP_ERR_STATE;
+    cudaError_t e = cudaSuccess;
+    if (!ctx->loop_decided) {   // no svip_policy_advance on the loop's counter in the body: decide here
+        e = launch_ex(loop_decide_kernel, 1, 32, 0, 0, ctx->loop_stream, ctx->loop, ctx->loop_n_active);
+        if (e == cudaSuccess) ctx->launches += 1;
+    }
+    cudaGraph_t body = nullptr;
+    cudaError_t e2 = cudaStreamEndCapture(ctx->loop_stream, &body);
+    ctx->loop_open = 0;
+    t_plain_launches = false;
+    if (e != cudaSuccess) { ctx->loop_failed = 1; return cuda_fail(ctx, e); }
+    if (e2 != cudaSuccess) { ctx->loop_failed = 1; return cuda_fail(ctx, e2); }
     return SVIP_OK;
 }
 
 int svip_graph_end(svip_ctx* ctx, void* stream, svip_graph** graph) {
     if (!ctx || !graph) return SVIP_ERR_INVALID_ARG;
     if (!ctx->capturing) return SVIP_ERR_STATE;
+    // a loop whose body was left open, or whose decision kernel could not be recorded, would
+    // never end at replay: such a graph is not handed out
+    bool broken = ctx->loop_failed != 0;
+    if (ctx->loop_open) {
+        cudaGraph_t body = nullptr;
+        cudaStreamEndCapture(ctx->loop_stream, &body);
+        ctx->loop_open = 0;
+        t_plain_launches = false;
+        broken = true;
+    }
+    ctx->loop_failed = 0;
     ctx->capturing = 0;
     cudaGraph_t g = nullptr;
     cudaError_t e = cudaStreamEndCapture(static_cast<cudaStream_t>(stream), &g);
+    if (broken) {
+        if (g) cudaGraphDestroy(g);
+        cudaGetLastError();
+        return SVIP_ERR_STATE;
+    }
     if (e != cudaSuccess || !g) return cuda_fail(ctx, e);
     cudaGraphExec_t ex = nullptr;
     e = cudaGraphInstantiate(&ex, g, 0);
