@@ -13,6 +13,9 @@
  *   - correction token:  Algorithm 4 (sampling), Algorithm 5 (greedy)
  *   - verify loop, bonus token: Algorithm 1 (outer loop body) / Algorithm 6
  *   - expected acceptance beta, TVD, KL: Eq. 1 - Eq. 4
+ *   - top-k / nucleus truncation (end of this file): not defined by the paper;
+ *     the published definitions, ties kept by threshold, pinned by hand-made
+ *     rows, a brute-force construction and the law of the emitted token
  *
  * Readings of the paper that this file fixes (each is pinned by a CPU test):
  *   - Algorithm 4 prints the residual with draft minus target.  Only
@@ -296,5 +299,70 @@ int svip_oracle_pair_stats(const void *t_row, const void *q_row, int dtype, long
     out[7] = 1.0 - sqrt(c_bound * Hq);
     free(p);
     free(q);
+    return 0;
+}
+
+/* ------------------------------------------------------------------------
+ * Top-k / nucleus (top-p) truncation of a distribution.
+ *
+ * The paper applies its length policy on top of systems that sample from
+ * truncated distributions but does not define the truncation itself; the
+ * definitions here are the published ones (top-k: keep the k most likely
+ * tokens; nucleus: keep the smallest set of most likely tokens whose mass
+ * reaches top_p), made order-independent by a threshold reading of ties:
+ *
+ *   tau_k  = the k-th largest raw logit (1 <= k < V), else the smallest logit
+ *   Z_k    = sum of exp(l_i/T - M) over {l_i >= tau_k},  M = max_i l_i/T
+ *   tau_p  = the largest logit value v with  sum over {l_i >= v} >= top_p*Z_k
+ *            (top_p < 1), else tau_k
+ *   tau    = tau_p (which is >= tau_k); the kept set is {i : l_i >= tau}:
+ *            every token tied with the last kept one is kept too.
+ *
+ * The truncated distribution is softmax(l/T) restricted to the kept set and
+ * renormalised; everything else (sampling, entropy, acceptance, residual) is
+ * the plain definition applied to rows whose dropped logits are -inf.
+ * Sums run over the logits sorted in descending order.
+ * Returns 0, or -1 if scratch memory could not be obtained.
+ */
+static int cmp_desc(const void *a, const void *b)
+{
+    double x = *(const double *)a, y = *(const double *)b;
+    return (x < y) - (x > y);
+}
+
+int svip_oracle_threshold(const void *row, int dtype, long V, double T, long top_k, double top_p,
+                          double *tau, double *Z_topk, double *Z_kept, long *n_kept)
+{
+    double *v = (double *)malloc((size_t)V * sizeof(double));
+    if (!v) return -1;
+    for (long i = 0; i < V; ++i)
+        v[i] = logit_at(row, dtype, i);
+    qsort(v, (size_t)V, sizeof(double), cmp_desc);
+    const double tau_k = (top_k >= 1 && top_k < V) ? v[top_k - 1] : v[V - 1];
+    const double M = v[0] / T;
+    double Zk = 0.0;
+    for (long i = 0; i < V && v[i] >= tau_k; ++i)
+        Zk += (v[i] == -INFINITY) ? 0.0 : exp(v[i] / T - M);
+    double t = tau_k;
+    if (top_p < 1.0) {
+        double c = 0.0;
+        long i = 0;
+        while (i < V && v[i] >= tau_k) {
+            const double val = v[i];
+            while (i < V && v[i] == val) {          /* the whole group of tied logits */
+                c += (val == -INFINITY) ? 0.0 : exp(val / T - M);
+                ++i;
+            }
+            if (c >= top_p * Zk) { t = val; break; }
+        }
+    }
+    double Zt = 0.0;
+    long n = 0;
+    for (long i = 0; i < V && v[i] >= t; ++i) {
+        Zt += (v[i] == -INFINITY) ? 0.0 : exp(v[i] / T - M);
+        ++n;
+    }
+    *tau = t; *Z_topk = Zk; *Z_kept = Zt; *n_kept = n;
+    free(v);
     return 0;
 }

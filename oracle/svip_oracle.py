@@ -63,6 +63,9 @@ def lib():
             f.argtypes = [dp, dp, C.c_long]
         L.svip_oracle_pair_stats.restype = C.c_int
         L.svip_oracle_pair_stats.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_long, C.c_double, C.c_double, dp]
+        L.svip_oracle_threshold.restype = C.c_int
+        L.svip_oracle_threshold.argtypes = [C.c_void_p, C.c_int, C.c_long, C.c_double, C.c_long, C.c_double,
+                                            dp, dp, dp, C.POINTER(C.c_long)]
         L.svip_oracle_residual.restype = C.c_double
         L.svip_oracle_residual.argtypes = [dp, dp, C.c_long, dp]
         _lib = L
@@ -253,3 +256,54 @@ def pack_ragged(draft_len):
         cu.append(cu[-1] + int(K) + 1)
     return (np.array(cu, dtype=np.int64), np.array(row_seq, dtype=np.int64),
             np.array(row_pos, dtype=np.int64))
+
+
+# ---------------------------------------------------------------- top-k / nucleus truncation
+
+def threshold(logits: np.ndarray, T: float, top_k: int, top_p: float, threads: int = 1):
+    """Per row: (tau, Z_topk, Z_kept, n_kept) of the truncation (see svip_oracle_threshold): the kept set is
+    {i : l_i >= tau}; masses are relative to the row maximum."""
+    logits = _rows2d(logits)
+    n, V = logits.shape
+    code = _dtype_code(logits)
+    tau = np.empty(n); Zk = np.empty(n); Zt = np.empty(n); kept = np.empty(n, dtype=np.int64)
+    L = lib()
+
+    def one(r):
+        a = C.c_double(); b = C.c_double(); c = C.c_double(); k = C.c_long()
+        rc = L.svip_oracle_threshold(logits.ctypes.data + r * logits.strides[0], code, V, float(T), int(top_k),
+                                     float(top_p), C.byref(a), C.byref(b), C.byref(c), C.byref(k))
+        if rc != 0:
+            raise MemoryError("oracle threshold")
+        tau[r] = a.value; Zk[r] = b.value; Zt[r] = c.value; kept[r] = k.value
+
+    _pmap(one, n, threads)
+    return tau, Zk, Zt, kept
+
+
+def mask_below(logits: np.ndarray, tau: np.ndarray) -> np.ndarray:
+    """Copy of the rows with every logit below its row's tau replaced by -inf (dropped tokens)."""
+    logits = _rows2d(logits)
+    tau = np.asarray(tau, dtype=np.float64).reshape(-1, 1)
+    if logits.dtype == np.float32:
+        return np.where(logits.astype(np.float64) >= tau, logits, np.float32(-np.inf)).astype(np.float32)
+    vals = (logits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    return np.where(vals >= tau, logits, np.uint16(0xFF80)).astype(np.uint16)
+
+
+def truncate(logits: np.ndarray, T: float, top_k: int, top_p: float, threads: int = 1) -> np.ndarray:
+    tau, _, _, _ = threshold(logits, T, top_k, top_p, threads)
+    return mask_below(logits, tau)
+
+
+def draft_step_filtered(logits, T, h, uniforms, top_k, top_p, threads: int = 1):
+    """The draft step on the truncated distribution: token ~ q~, H = H(q~), stop = sqrt(H) > h."""
+    return draft_step(truncate(logits, T, top_k, top_p, threads), T, h, uniforms, threads)
+
+
+def verify_filtered(draft_tokens, q_logits, target_logits, cu_rows, T, uniforms, top_k, top_p, q_row_of=None,
+                    want_accept_prob=False, threads: int = 1):
+    """The verification round with both models' distributions truncated the same way."""
+    return verify(draft_tokens, truncate(q_logits, T, top_k, top_p, threads),
+                  truncate(target_logits, T, top_k, top_p, threads), cu_rows, T, uniforms, q_row_of=q_row_of,
+                  want_accept_prob=want_accept_prob, threads=threads)
