@@ -157,6 +157,28 @@ int svip_draft_step_at(svip_ctx* ctx, const void* logits, svip_dtype dtype, int 
                        int32_t* token, float* entropy, uint8_t* stop, float* row_stats, void* stream);
 
 /*
+ * Truncation threshold of every row for top-k and nucleus (top-p) sampling.
+ * The paper runs its policy on top of samplers that truncate the distribution
+ * but does not define the truncation; this library uses the published
+ * definitions with ties kept by value:
+ *   tau_k = the k-th largest logit of the row (top_k in 1..V-1; 0 or >= V: off)
+ *   tau   = the largest logit value v for which the mass of {l >= v} reaches
+ *           top_p times the mass of {l >= tau_k} (top_p in (0,1); >= 1: off,
+ *           tau = tau_k), masses being those of softmax(l / T)
+ * thr[r] receives tau of row r as a logit value (-inf when nothing is
+ * dropped): the kept tokens are exactly those with logit >= thr[r], so tokens
+ * tied with the last kept one stay.  tau_k is exact; the nucleus compares fp32
+ * masses (summed as 2^-40 fixed point, so the result does not depend on the
+ * order of summation) and may differ from an fp64 evaluation where the running
+ * mass comes within about 1e-6 of top_p.  T > 0.  NaN logits count as -inf.
+ * Every row is read once per radix pass: 2 (bf16) or 4 (fp32) passes for top-k,
+ * as many again for the nucleus (+1 for the nucleus alone).
+ *   logits  DEVICE, row r starts at element r*row_stride;  thr  DEVICE [n_rows] fp32 out
+ */
+int svip_row_threshold(svip_ctx* ctx, const void* logits, svip_dtype dtype, int n_rows, int V,
+                       long row_stride, float T, int top_k, float top_p, float* thr, void* stream);
+
+/*
  * Draft-length policies, kept on the device so that the drafting loop needs no
  * host round trip per token.
  *   SVIP_POLICY_ENTROPY    the paper's rule: a sequence stops drafting when the

@@ -79,6 +79,8 @@ def library():
     L.svip_graph_loop_begin.argtypes = [vp, vp, vp, i32, C.POINTER(vp)]
     L.svip_graph_loop_end.restype = i32
     L.svip_graph_loop_end.argtypes = [vp]
+    L.svip_row_threshold.restype = i32
+    L.svip_row_threshold.argtypes = [vp, vp, i32, i32, i32, lng, f32, i32, f32, vp, vp]
     L.svip_policy_advance.restype = i32
     L.svip_policy_advance.argtypes = [vp, i32, vp, vp, vp, vp, i32, i32, vp, vp]
     L.svip_policy_update.restype = i32
@@ -202,6 +204,10 @@ class Context:
                                             int(pos_stride), _ptr(pos), int(slot_stride), float(T), float(thresh),
                                             _ptr(uniforms), _ptr(active), _ptr(token), _ptr(entropy), _ptr(stop),
                                             _ptr(row_stats), _stream(stream)), self._h)
+
+    def row_threshold(self, logits, dtype, n_rows, V, row_stride, T, top_k, top_p, thr, stream=None):
+        _check(library().svip_row_threshold(self._h, _ptr(logits), int(dtype), int(n_rows), int(V), int(row_stride),
+                                            float(T), int(top_k), float(top_p), _ptr(thr), _stream(stream)), self._h)
 
     def policy_advance(self, policy, stop, gamma, draft_len, active, B, K_cap, n_active=None, stream=None):
         _check(library().svip_policy_advance(self._h, int(policy), _ptr(stop), _ptr(gamma), _ptr(draft_len),

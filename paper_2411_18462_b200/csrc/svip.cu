@@ -991,6 +991,8 @@ __global__ void __launch_bounds__(kPackThreads) pack_ragged_kernel(const int32_t
 
 }  // namespace svip
 
+#include "svip_select.cuh"
+
 // ==================================================================== host side / C ABI
 
 using namespace svip;
@@ -1155,7 +1157,8 @@ int svip_create(svip_ctx** out, int device, int max_rows) {
             (const void*)row_stats_kernel<kBF16, 0>,     (const void*)row_stats_kernel<kBF16, 1>,
             (const void*)row_stats_kernel<kF32, 0>,      (const void*)row_stats_kernel<kF32, 1>,
             (const void*)verify_finish_kernel<kBF16>,    (const void*)verify_finish_kernel<kF32>,
-            (const void*)row_stats_kernel<kBF16, 2>,     (const void*)row_stats_kernel<kF32, 2>};
+            (const void*)row_stats_kernel<kBF16, 2>,     (const void*)row_stats_kernel<kF32, 2>,
+            (const void*)row_threshold_kernel<kBF16>,    (const void*)row_threshold_kernel<kF32>};
         for (const void* k : ringed)
             if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes) != cudaSuccess)
                 rc = SVIP_ERR_CUDA;
@@ -1274,6 +1277,26 @@ int svip_draft_step_at(svip_ctx* ctx, const void* logits, svip_dtype dtype, int 
         else k = a.greedy ? draft_step_kernel<kF32, true, 2, true> : draft_step_kernel<kF32, false, 2, true>;
     }
     cudaError_t e = launch_clustered(k, B, S, a, st, kRingBytes);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    return SVIP_OK;
+}
+
+int svip_row_threshold(svip_ctx* ctx, const void* logits, svip_dtype dtype, int n_rows, int V, long row_stride,
+                       float T, int top_k, float top_p, float* thr, void* stream) {
+    if (!ctx || !logits || !thr) return SVIP_ERR_INVALID_ARG;
+    if (dtype != SVIP_F32 && dtype != SVIP_BF16) return SVIP_ERR_UNSUPPORTED;
+    if (n_rows < 0 || V < 1 || V > 0x7fffffe0 || row_stride < 0 || top_k < 0) return SVIP_ERR_INVALID_ARG;
+    if (!(T > 0.f) || std::isinf(T) || !(top_p > 0.f)) return SVIP_ERR_INVALID_ARG;
+    if (!aligned_to(logits, dtype == SVIP_BF16 ? 2 : 4)) return SVIP_ERR_INVALID_ARG;
+    if (n_rows == 0) return SVIP_OK;
+    ThresholdArgs a;
+    a.logits = logits; a.row_stride = row_stride; a.V = V; a.c = scale_for(T);
+    a.top_k = (top_k >= 1 && top_k < V) ? top_k : 0; a.top_p = top_p; a.thr = thr;
+    const int S = pick_cluster(ctx, n_rows, V, dtype);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = dtype == SVIP_BF16 ? launch_clustered(row_threshold_kernel<kBF16>, n_rows, S, a, st, kRingBytes)
+                                       : launch_clustered(row_threshold_kernel<kF32>, n_rows, S, a, st, kRingBytes);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
     return SVIP_OK;

@@ -1,0 +1,363 @@
+// Truncation threshold of a logits row (top-k and nucleus / top-p).
+//
+// The kept set of a row is {i : l_i >= tau}: tau_k is the k-th largest logit, and inside that set
+// tau is the largest logit value v for which the mass of {l_i >= v} reaches top_p of the mass of
+// {l_i >= tau_k}; tokens tied with the last kept one are all kept.  The paper applies its length
+// policy on top of samplers that truncate but does not define the truncation; these are the
+// published definitions (top-k, nucleus sampling) read with a threshold so that the result does not
+// depend on the order of equal logits.
+//
+// One cluster per row.  The value is found by a radix descent over an order-preserving integer
+// image of the logits, 8 bits per pass: every pass streams the row once (cp.async ring, as the other
+// kernels), histograms the digit of the elements that match the digits already fixed (counts, and
+// for the nucleus the masses 2^(l*c - M) in 2^-40 fixed point, so that every sum is an integer and
+// the result is the same whatever the order of the additions), the blocks add their histograms up
+// through distributed shared memory, and every block takes the same decision from the same sums.
+// bf16 rows need two passes per descent, fp32 rows four.
+#pragma once
+
+#include "svip_device.cuh"
+
+namespace svip {
+
+constexpr int kHistCopies = 8;           // private histograms per block (one per pair of warps)
+constexpr float kMassScale = 1099511627776.0f;   // 2^40
+
+struct ThresholdArgs {
+    const void* logits;
+    long row_stride;
+    int V;
+    float c;        // log2(e) / T
+    int top_k;      // 1 .. V-1, or 0 when off
+    float top_p;    // (0, 1), or >= 1 when off
+    float* thr;     // [rows] out: tau as a logit value (-inf: nothing is dropped)
+};
+
+// Monotone image of a float: a < b  <=>  key(a) < key(b).  NaN counts as -inf.
+__device__ __forceinline__ uint32_t order_key(float x) {
+    if (!(x == x)) x = neg_inf();
+    if (x == 0.f) x = 0.f;          // -0 and +0 are one value
+    const uint32_t u = __float_as_uint(x);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__device__ __forceinline__ float key_value(uint32_t key) {
+    return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
+}
+
+// Streams segment `seg` of the row with the calling warp and hands every vector to f(x, vi), with
+// the elements outside the row set to -inf.
+template <int DT, class F>
+__device__ __forceinline__ void stream_segment(const RowGeom& g, int seg, int lane, uint32_t slot0, F&& f) {
+    constexpr int EPV = ElemTraits<DT>::kEPV;
+    constexpr uint32_t kSlotStride = kThreads * 16;
+    int v_lo, v_hi;
+    seg_range(g, seg, v_lo, v_hi);
+    const int vi0 = v_lo + lane;
+    const int n = v_hi > vi0 ? (v_hi - vi0 + 31) >> 5 : 0;
+    const uint4* src = g.base + vi0;
+#pragma unroll
+    for (int s = 0; s < kStages; ++s) {
+        if (s < n) cp_async16(slot0 + s * kSlotStride, src + 32 * s);
+        cp_async_commit();
+    }
+    for (int it = 0; it < n; ++it) {
+        cp_async_wait<kStages - 1>();
+        const uint32_t slot = slot0 + (it & (kStages - 1)) * kSlotStride;
+        const uint4 raw = lds128(slot);
+        if (it + kStages < n) cp_async16(slot, src + 32 * (it + kStages));
+        cp_async_commit();
+        float x[EPV];
+        unpack_masked<DT>(raw, vi0 + 32 * it, g, x);
+        f(x, vi0 + 32 * it);
+    }
+    cp_async_wait<0>();
+}
+
+struct SelectShared {
+    uint32_t priv[kHistCopies][3][256];   // per copy: count, mass low word, mass high word
+    uint32_t blk_cnt[256];                // this block's histogram, read by the peers
+    unsigned long long blk_mass[256];
+    uint32_t tot_cnt[256];                // the cluster's histogram
+    unsigned long long tot_mass[256];
+    float blk_max;                        // this block's largest logit
+    unsigned long long blk_above;         // this block's mass of the elements >= tau_k
+    float warp_max[kWarps];
+    unsigned long long warp_above[kWarps];
+    // decision of a pass (written by warp 0)
+    int bin;
+    uint32_t cnt_above;
+    unsigned long long mass_above;
+    unsigned long long mass_total;
+    unsigned long long mass_bin;
+};
+
+__device__ __forceinline__ unsigned long long shfl_up_u64(unsigned long long v, int o) {
+    uint32_t lo = __shfl_up_sync(0xffffffffu, static_cast<uint32_t>(v), o);
+    uint32_t hi = __shfl_up_sync(0xffffffffu, static_cast<uint32_t>(v >> 32), o);
+    return (static_cast<unsigned long long>(hi) << 32) | lo;
+}
+
+// One pass: histogram of digit (key >> shift) & 255 over the elements whose higher digits equal
+// those of `prefix` (all elements when first).  kMass adds the masses; kMax also finds the largest
+// logit; `key_k` (with kAbove) sums the mass of the elements with key >= key_k.  On return every
+// block of the cluster holds the cluster-wide histogram in sh.tot_*.
+template <int DT, bool kMass, bool kMax, bool kAbove>
+__device__ __forceinline__ void histogram_pass(cg::cluster_group& cluster, const RowGeom& g, int S, int rank,
+                                               int tid, uint32_t slot0, uint32_t prefix, int shift, bool first,
+                                               float c, float M, uint32_t key_k, SelectShared& sh,
+                                               float& row_max, unsigned long long& above) {
+    constexpr int EPV = ElemTraits<DT>::kEPV;
+    const int lane = tid & 31, warp = tid >> 5;
+    for (int i = tid; i < kHistCopies * 3 * 256; i += kThreads) (&sh.priv[0][0][0])[i] = 0;
+    __syncthreads();
+    uint32_t* h_cnt = sh.priv[warp >> 1][0];
+    uint32_t* h_lo = sh.priv[warp >> 1][1];
+    uint32_t* h_hi = sh.priv[warp >> 1][2];
+    float mx = neg_inf();
+    unsigned long long ab = 0;
+    const uint32_t want = first ? 0u : (prefix >> (shift + 8));
+    stream_segment<DT>(g, rank * kWarps + warp, lane, slot0, [&](const float (&x)[EPV], int) {
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) {
+            const uint32_t key = order_key(x[j]);
+            if (kMax) mx = fmaxf(mx, x[j]);
+            unsigned long long wq = 0;
+            if (kMass) {
+                const float w = ex2_approx(fmaxf(__fmaf_rn(x[j], c, -M), kArgFloor));
+                wq = __float2ull_rz(w * kMassScale);
+                if (kAbove && key >= key_k) ab += wq;
+            }
+            if (first || (key >> (shift + 8)) == want) {
+                const uint32_t bin = (key >> shift) & 255u;
+                atomicAdd(h_cnt + bin, 1u);
+                if (kMass && wq) {
+                    const uint32_t lo = static_cast<uint32_t>(wq);
+                    const uint32_t old = atomicAdd(h_lo + bin, lo);
+                    const uint32_t carry = (old + lo < old) ? 1u : 0u;
+                    const uint32_t hi = static_cast<uint32_t>(wq >> 32) + carry;
+                    if (hi) atomicAdd(h_hi + bin, hi);
+                }
+            }
+        }
+    });
+    if (kMax) {
+        mx = warp_max(mx);
+        if (lane == 0) sh.warp_max[warp] = mx;
+    }
+    if (kAbove) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            uint32_t lo = __shfl_xor_sync(0xffffffffu, static_cast<uint32_t>(ab), o);
+            uint32_t hi = __shfl_xor_sync(0xffffffffu, static_cast<uint32_t>(ab >> 32), o);
+            ab += (static_cast<unsigned long long>(hi) << 32) | lo;
+        }
+        if (lane == 0) sh.warp_above[warp] = ab;
+    }
+    __syncthreads();
+    if (tid < 256) {
+        uint32_t cn = 0;
+        unsigned long long ms = 0;
+#pragma unroll
+        for (int k = 0; k < kHistCopies; ++k) {
+            cn += sh.priv[k][0][tid];
+            if (kMass) ms += (static_cast<unsigned long long>(sh.priv[k][2][tid]) << 32) + sh.priv[k][1][tid];
+        }
+        sh.blk_cnt[tid] = cn;
+        sh.blk_mass[tid] = ms;
+    }
+    if (tid == 0) {
+        float m = neg_inf();
+        unsigned long long s = 0;
+        for (int w = 0; w < kWarps; ++w) {
+            if (kMax) m = fmaxf(m, sh.warp_max[w]);
+            if (kAbove) s += sh.warp_above[w];
+        }
+        sh.blk_max = m;
+        sh.blk_above = s;
+    }
+    cluster.sync();
+    if (tid < 256) {
+        uint32_t cn = 0;
+        unsigned long long ms = 0;
+        for (int r = 0; r < S; ++r) {
+            const SelectShared* peer = cluster.map_shared_rank(&sh, r);
+            cn += peer->blk_cnt[tid];
+            if (kMass) ms += peer->blk_mass[tid];
+        }
+        sh.tot_cnt[tid] = cn;
+        sh.tot_mass[tid] = ms;
+    }
+    if (kMax || kAbove) {
+        float m = neg_inf();
+        unsigned long long s = 0;
+        for (int r = 0; r < S; ++r) {
+            const SelectShared* peer = cluster.map_shared_rank(&sh, r);
+            if (kMax) m = fmaxf(m, peer->blk_max);
+            if (kAbove) s += peer->blk_above;
+        }
+        if (kMax) row_max = m;
+        if (kAbove) above = s;
+    }
+    cluster.sync();   // every peer has read this block's histogram; tot_* is visible block-wide
+}
+
+// Warp 0: walks the cluster histogram from the highest digit down and finds the digit at which
+// the running count reaches `k_rem` (kByMass false) or the running mass reaches `p_rem`.
+template <bool kByMass>
+__device__ __forceinline__ void decide(SelectShared& sh, int lane, uint32_t k_rem, unsigned long long p_rem) {
+    // lane l owns the digits 255 - 8l ... 248 - 8l, highest first
+    uint32_t cn[8];
+    unsigned long long ms[8];
+    uint32_t csum = 0;
+    unsigned long long msum = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int bin = 255 - 8 * lane - j;
+        cn[j] = sh.tot_cnt[bin];
+        ms[j] = sh.tot_mass[bin];
+        csum += cn[j];
+        msum += ms[j];
+    }
+    uint32_t cinc = csum;
+    unsigned long long minc = msum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t cu = __shfl_up_sync(0xffffffffu, cinc, o);
+        const unsigned long long mu = shfl_up_u64(minc, o);
+        if (lane >= o) { cinc += cu; minc += mu; }
+    }
+    uint32_t cbefore = cinc - csum;              // digits above this lane's
+    unsigned long long mbefore = minc - msum;
+    int hit = -1;
+    uint32_t c_at = 0;
+    unsigned long long m_at = 0, m_bin = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const bool reached = kByMass ? (mbefore + ms[j] >= p_rem) : (cbefore + cn[j] >= k_rem);
+        if (hit < 0 && reached && (kByMass ? ms[j] > 0 : cn[j] > 0)) {
+            hit = 255 - 8 * lane - j;
+            c_at = cbefore;
+            m_at = mbefore;
+            m_bin = ms[j];
+        }
+        cbefore += cn[j];
+        mbefore += ms[j];
+    }
+    const unsigned who = __ballot_sync(0xffffffffu, hit >= 0);
+    const unsigned long long total = __shfl_sync(0xffffffffu, static_cast<uint32_t>(minc), 31) |
+        (static_cast<unsigned long long>(__shfl_sync(0xffffffffu, static_cast<uint32_t>(minc >> 32), 31)) << 32);
+    if (who == 0) {
+        // nothing reaches the target (an empty histogram): stay at the lowest digit
+        if (lane == 0) { sh.bin = 0; sh.cnt_above = 0; sh.mass_above = 0; sh.mass_total = total; sh.mass_bin = 0; }
+    } else if (lane == __ffs(who) - 1) {
+        sh.bin = hit; sh.cnt_above = c_at; sh.mass_above = m_at; sh.mass_total = total; sh.mass_bin = m_bin;
+    }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads, 2) row_threshold_kernel(ThresholdArgs a) {
+    constexpr int kLevels = DT == kBF16 ? 2 : 4;   // the low 16 bits of a bf16 logit carry nothing
+    extern __shared__ uint4 ring[];
+    __shared__ SelectShared sh;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int S = cluster.dim_blocks().x;
+    const int rank = cluster.block_rank();
+    const int row = blockIdx.x / S;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    pdl_launch_dependents();
+    const char* rp = static_cast<const char*>(a.logits) +
+                     static_cast<size_t>(row) * a.row_stride * ElemTraits<DT>::kBytes;
+    const RowGeom g = make_geom<DT>(rp, a.V, S * kWarps);
+    const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
+    pdl_wait();
+
+    const bool use_k = a.top_k >= 1 && a.top_k < a.V;
+    const bool use_p = a.top_p < 1.0f;
+    float row_max = neg_inf();
+    unsigned long long above = 0;
+    bool have_max = false;
+    uint32_t key_k = 0;       // key of tau_k (0: below every key, nothing dropped)
+
+    if (use_k) {
+        uint32_t prefix = 0, k_rem = static_cast<uint32_t>(a.top_k);
+        for (int level = 0; level < kLevels; ++level) {
+            const int shift = 24 - 8 * level;
+            if (level == 0)
+                histogram_pass<DT, false, true, false>(cluster, g, S, rank, tid, slot0, prefix, shift, true, a.c, 0.f,
+                                                       0u, sh, row_max, above);
+            else
+                histogram_pass<DT, false, false, false>(cluster, g, S, rank, tid, slot0, prefix, shift, false, a.c,
+                                                        0.f, 0u, sh, row_max, above);
+            if (warp == 0) decide<false>(sh, lane, k_rem, 0ull);
+            __syncthreads();
+            prefix |= static_cast<uint32_t>(sh.bin) << shift;
+            k_rem -= sh.cnt_above;
+            __syncthreads();   // the decision is read before the next pass overwrites it
+        }
+        have_max = true;
+        // digits below the ones examined: a bf16 logit has them all zero, which the key stores as
+        // ones for negative values
+        key_k = prefix;
+        if (DT == kBF16 && !(prefix & 0x80000000u)) key_k |= 0xffffu;
+    }
+
+    uint32_t key_t = key_k;
+    if (use_p) {
+        if (!have_max) {
+            // the masses are taken relative to the largest logit: find it first
+            float mx = neg_inf();
+            stream_segment<DT>(g, rank * kWarps + warp, lane, slot0,
+                               [&](const float (&x)[ElemTraits<DT>::kEPV], int) {
+#pragma unroll
+                for (int j = 0; j < ElemTraits<DT>::kEPV; ++j) mx = fmaxf(mx, x[j]);
+            });
+            mx = warp_max(mx);
+            if (lane == 0) sh.warp_max[warp] = mx;
+            __syncthreads();
+            if (tid == 0) {
+                float m = neg_inf();
+                for (int w = 0; w < kWarps; ++w) m = fmaxf(m, sh.warp_max[w]);
+                sh.blk_max = m;
+            }
+            cluster.sync();
+            float m = neg_inf();
+            for (int r = 0; r < S; ++r) m = fmaxf(m, cluster.map_shared_rank(&sh, r)->blk_max);
+            row_max = m;
+            cluster.sync();
+        }
+        const bool finite = fabsf(row_max) <= kMaxLogit;
+        const float M = finite ? __fmul_rn(row_max, a.c) : 0.f;
+        uint32_t prefix = 0;
+        unsigned long long p_rem = 0;
+        for (int level = 0; level < kLevels; ++level) {
+            const int shift = 24 - 8 * level;
+            if (level == 0)
+                histogram_pass<DT, true, false, true>(cluster, g, S, rank, tid, slot0, prefix, shift, true, a.c, M,
+                                                      key_k, sh, row_max, above);
+            else
+                histogram_pass<DT, true, false, false>(cluster, g, S, rank, tid, slot0, prefix, shift, false, a.c, M,
+                                                       key_k, sh, row_max, above);
+            if (level == 0) {
+                // target mass: top_p of the mass of the top-k set (the whole row without top-k)
+                const double want = ceil(static_cast<double>(a.top_p) * static_cast<double>(above));
+                p_rem = static_cast<unsigned long long>(want);
+                if (p_rem < 1) p_rem = 1;
+                if (p_rem > above) p_rem = above;
+            }
+            if (warp == 0) decide<true>(sh, lane, 0u, p_rem);
+            __syncthreads();
+            prefix |= static_cast<uint32_t>(sh.bin) << shift;
+            p_rem -= sh.mass_above;
+            __syncthreads();
+        }
+        uint32_t key_p = prefix;
+        if (DT == kBF16 && !(prefix & 0x80000000u)) key_p |= 0xffffu;
+        if (above == 0 || !finite) key_p = 0;   // a row without mass: the nucleus drops nothing
+        key_t = key_p > key_k ? key_p : key_k;
+    }
+    if (rank == 0 && tid == 0) a.thr[row] = key_t ? key_value(key_t) : neg_inf();
+    // the last pass ended with a cluster barrier after all remote reads: blocks may leave
+}
+
+}  // namespace svip

@@ -1,0 +1,154 @@
+"""svip_row_threshold (top-k / nucleus cut of every row) against the oracle's sorted-row definition."""
+import numpy as np
+import pytest
+
+import svip_testlib as tl
+from paper_2411_18462_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+NUCLEUS_TOL = 1e-5      # in units of the top-k mass, like the CDF tolerance of sampled tokens
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2411_18462_b200 import Context, build
+    build.build()
+    c = Context(0, 1 << 12)
+    yield c
+    c.destroy()
+
+
+def values_of(rows):
+    return W.bf16_bits_to_f32(rows).astype(np.float64) if rows.dtype == np.uint16 else rows.astype(np.float64)
+
+
+def gpu_threshold(ctx, rows, T, k, p, pad_elems=0, row_stride=None):
+    import torch
+    n, V = rows.shape
+    stride = V if row_stride is None else row_stride
+    buf = np.zeros(pad_elems + n * stride + 16, dtype=rows.dtype)
+    buf[:] = np.nan if rows.dtype == np.float32 else 0x7FC0      # poison between the rows
+    for r in range(n):
+        buf[pad_elems + r * stride: pad_elems + r * stride + V] = rows[r]
+    d = tl.to_device(buf)
+    thr = torch.full((n,), 123.0, device="cuda")
+    ctx.row_threshold(d.data_ptr() + pad_elems * rows.itemsize, tl.dtype_code(rows), n, V, stride, T, k, p, thr)
+    torch.cuda.synchronize()
+    return thr.cpu().numpy()
+
+
+def check(oracle, rows, T, k, p, got, label=""):
+    """tau_k is exact.  The nucleus cut is exact unless the running mass comes within NUCLEUS_TOL of top_p at
+    the oracle's cut; then the GPU's cut must still satisfy the definition within that tolerance."""
+    tau, Zk, _, _ = oracle.threshold(rows, T, k, p, threads=8)
+    vals = values_of(rows)
+    n_soft = 0
+    for r in range(rows.shape[0]):
+        v = vals[r]
+        want = tau[r] if np.isfinite(tau[r]) else -np.inf
+        if (v >= want).all():
+            assert (v >= got[r]).all(), "%s row %d: nothing is dropped, got thr %r" % (label, r, got[r])
+            continue
+        if got[r] == np.float32(want):
+            continue
+        assert p < 1.0, "%s row %d: top-k cut must be exact: %r vs %r" % (label, r, got[r], want)
+        finite = v[np.isfinite(v)]
+        w = np.where(np.isfinite(v), np.exp((v - finite.max()) / T), 0.0)
+        g = float(got[r])
+        assert (v == g).any(), "%s row %d: thr %r is not a logit of the row" % (label, r, g)
+        tau_k = np.sort(v)[::-1][k - 1] if 1 <= k < v.size else v.min()
+        assert g >= tau_k
+        assert w[v >= g].sum() >= (p - NUCLEUS_TOL) * Zk[r], (label, r)
+        assert w[v > g].sum() < (p + NUCLEUS_TOL) * Zk[r], (label, r)
+        n_soft += 1
+    return n_soft
+
+
+CASES = [(0, 0.9), (50, 1.0), (50, 0.8), (1, 1.0), (0, 0.5), (1000, 0.95), (0, 0.999)]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("V", [777, 32000, 152064])
+def test_threshold_matches_the_oracle(ctx, oracle, dtype, V):
+    rng = np.random.default_rng(V + (dtype == "bf16"))
+    n = 12
+    x = (rng.standard_normal((n, V)) * rng.uniform(0.3, 6.0, size=(n, 1))).astype(np.float32)
+    x[3, rng.integers(0, V)] += 25.0            # a peaked row
+    x[4] = 0.0                                  # all equal: one group of ties
+    x[5, ::3] = -np.inf                         # dropped tokens in the input
+    rows = W.to_bf16_bits(x) if dtype == "bf16" else x
+    soft = 0
+    for k, p in CASES:
+        kk = min(k, V - 1) if k else 0
+        got = gpu_threshold(ctx, rows, 1.0, kk, p)
+        soft += check(oracle, rows, 1.0, kk, p, got, "V=%d %s k=%d p=%g" % (V, dtype, kk, p))
+    assert soft <= 2, "cuts decided inside the tolerance band should be rare: %d" % soft
+
+
+@pytest.mark.parametrize("S", [1, 2, 3, 5, 8])
+def test_every_cluster_size_and_unaligned_rows(ctx, oracle, S):
+    rng = np.random.default_rng(40 + S)
+    V = 40013
+    for dtype in ("f32", "bf16"):
+        x = (rng.standard_normal((5, V)) * 2.5).astype(np.float32)
+        rows = W.to_bf16_bits(x) if dtype == "bf16" else x
+        ctx.set_cluster_size(S)
+        try:
+            for pad, stride in ((0, V), (3, V + 5), (1, V + 1)):
+                got = gpu_threshold(ctx, rows, 0.7, 300, 0.9, pad_elems=pad, row_stride=stride)
+                check(oracle, rows, 0.7, 300, 0.9, got, "S=%d %s pad=%d" % (S, dtype, pad))
+        finally:
+            ctx.set_cluster_size(0)
+
+
+def test_small_and_degenerate_rows(ctx, oracle):
+    rng = np.random.default_rng(9)
+    for V in (1, 2, 5, 17, 33, 300):
+        x = (rng.standard_normal((4, V)) * 2).astype(np.float32)
+        x[1] = x[1, 0]                                  # all tied
+        for k, p in ((0, 0.7), (1, 1.0), (2, 0.6), (V - 1, 1.0), (V, 0.9), (V + 5, 1.0)):
+            got = gpu_threshold(ctx, x, 1.0, k, p)
+            check(oracle, x, 1.0, k, p, got, "V=%d k=%d p=%g" % (V, k, p))
+    # signed zeros are one value; NaN counts as a dropped token
+    x = np.array([[0.0, -0.0, 1.0, -1.0, np.nan, 0.0, -2.0, 0.5]], dtype=np.float32)
+    got = gpu_threshold(ctx, x, 1.0, 3, 1.0)
+    assert got[0] == 0.0                                # third largest is a zero; every zero is kept
+    y = np.where(np.isnan(x), -np.inf, x).astype(np.float32)
+    for k, p in ((2, 1.0), (0, 0.8), (5, 0.9)):
+        assert np.array_equal(gpu_threshold(ctx, x, 1.0, k, p), gpu_threshold(ctx, y, 1.0, k, p))
+        check(oracle, y, 1.0, k, p, gpu_threshold(ctx, y, 1.0, k, p), "nan row")
+    # a row of dropped tokens only: nothing to cut
+    z = np.full((1, 64), -np.inf, dtype=np.float32)
+    assert gpu_threshold(ctx, z, 1.0, 4, 0.9)[0] == -np.inf
+
+
+def test_both_off_drops_nothing(ctx):
+    rng = np.random.default_rng(1)
+    x = (rng.standard_normal((3, 5000)) * 2).astype(np.float32)
+    got = gpu_threshold(ctx, x, 1.0, 0, 1.0)
+    assert np.all(got == -np.inf)
+
+
+def test_published_shapes(ctx, oracle):
+    """Rows of the ragged (bf16, heavy-tailed scales, planted tokens) and stress (fp32 Zipf) recipes."""
+    w = W.make_workload("ragged", B=8)
+    rows = np.ascontiguousarray(w.q_logits[:40])
+    for k, p in ((0, 0.9), (64, 0.95)):
+        check(oracle, rows, w.T, k, p, gpu_threshold(ctx, rows, w.T, k, p), "ragged")
+    w = W.make_workload("stress", B=4)
+    rows = np.ascontiguousarray(w.q_logits[:16])
+    for k, p in ((0, 0.9), (100, 1.0), (4000, 0.99)):
+        check(oracle, rows, w.T, k, p, gpu_threshold(ctx, rows, w.T, k, p), "stress")
+
+
+def test_threshold_bad_arguments(ctx):
+    import torch
+    from paper_2411_18462_b200 import SvipError
+    x = torch.zeros(4, 64, device="cuda"); t = torch.zeros(4, device="cuda")
+    for bad in (dict(T=0.0), dict(top_p=0.0), dict(top_k=-1), dict(V=0)):
+        a = dict(T=1.0, top_k=3, top_p=0.9, V=64)
+        a.update(bad)
+        with pytest.raises(SvipError):
+            ctx.row_threshold(x, 0, 4, a["V"], 64, a["T"], a["top_k"], a["top_p"], t)
+    ctx.row_threshold(x, 0, 0, 64, 64, 1.0, 3, 0.9, t)      # no rows
