@@ -179,6 +179,31 @@ int svip_row_threshold(svip_ctx* ctx, const void* logits, svip_dtype dtype, int 
                        long row_stride, float T, int top_k, float top_p, float* thr, void* stream);
 
 /*
+ * The draft step and the verification round on truncated distributions: every
+ * distribution is softmax(l / T) restricted to the tokens whose logit is >= the
+ * row's threshold (from svip_row_threshold) and renormalised.  Sampling,
+ * entropy and stop test (Algorithm 1, Eq. 7), acceptance (Algorithm 2) and the
+ * residual (Algorithm 4) are those of svip_draft_step_masked / svip_verify
+ * applied to these distributions; a draft token that the target's truncation
+ * dropped has target probability zero and is rejected.  T > 0 only.
+ *   thr     DEVICE [B] fp32: threshold of each draft row of this step
+ *   q_thr   DEVICE fp32, indexed like draft_tokens / q_stats (by draft row)
+ *   p_thr   DEVICE [n_target_rows] fp32
+ * row_stats / q_stats hold (m, Z) of the truncated distribution.  Other
+ * arguments as for svip_draft_step_masked and svip_verify.
+ */
+int svip_draft_step_filtered(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, int V,
+                             long row_stride, float T, float thresh, const float* uniforms,
+                             const uint8_t* active, const float* thr, int32_t* token, float* entropy,
+                             uint8_t* stop, float* row_stats, void* stream);
+int svip_verify_filtered(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits,
+                         long q_row_stride, const float* q_stats, const float* q_thr,
+                         long q_seq_stride, long q_pos_stride, const void* target_logits,
+                         long t_row_stride, const float* p_thr, svip_dtype dtype,
+                         const int32_t* cu_rows, int B, int K, int n_target_rows, int V, float T,
+                         const float* uniforms, int32_t* n_accepted, int32_t* next_token, void* stream);
+
+/*
  * Draft-length policies, kept on the device so that the drafting loop needs no
  * host round trip per token.
  *   SVIP_POLICY_ENTROPY    the paper's rule: a sequence stops drafting when the

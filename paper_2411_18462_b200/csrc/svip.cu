@@ -170,18 +170,21 @@ struct DraftArgs {
     const int32_t* pos;      // NULL, or per row the draft position p whose logits are read (svip_draft_step_at)
     long pos_stride;         // elements between the logits of consecutive positions of a row
     long slot_stride;        // uniforms / token / entropy / row_stats live at index p * slot_stride + row
+    const float* thr;        // NULL, or per row the truncation threshold: only logits >= thr[row] count
 };
 
 template <int DT>
 struct SoftmaxWeights {
     RowGeom g;
     float c, M;
+    float thr = -INFINITY;   // logits below it carry no weight (truncated distributions)
     __device__ __forceinline__ void operator()(int vi, float (&w)[ElemTraits<DT>::kEPV]) const {
         constexpr int EPV = ElemTraits<DT>::kEPV;
         float x[EPV];
         unpack_masked<DT>(g.base[vi], vi, g, x);
 #pragma unroll
-        for (int j = 0; j < EPV; ++j) w[j] = ex2_approx(fmaxf(__fmaf_rn(x[j], c, -M), kArgFloor));
+        for (int j = 0; j < EPV; ++j)
+            w[j] = x[j] >= thr ? ex2_approx(fmaxf(__fmaf_rn(x[j], c, -M), kArgFloor)) : 0.f;
     }
 };
 
@@ -193,8 +196,9 @@ struct RowShared {
 // kBlocks is the number of blocks the register budget must leave room for on one SM: 2 for
 // launches that fit the GPU in one wave (latency matters, registers are free), 3 for launches of
 // many waves, where a third resident block streams on while another one is in its epilogue.
-// kPos compiles the position-indexed form (svip_draft_step_at) in.
-template <int DT, bool kGreedy, int kBlocks, bool kPos = false>
+// kPos compiles the position-indexed form (svip_draft_step_at) in, kThr the truncated form
+// (svip_draft_step_filtered).
+template <int DT, bool kGreedy, int kBlocks, bool kPos = false, bool kThr = false>
 __global__ void __launch_bounds__(kThreads, kBlocks) draft_step_kernel(DraftArgs a) {
     constexpr int EPV = ElemTraits<DT>::kEPV;
     extern __shared__ uint4 ring[];
@@ -225,7 +229,8 @@ __global__ void __launch_bounds__(kThreads, kBlocks) draft_step_kernel(DraftArgs
         if (a.ext_target) ext = fmaxf(__ldg(a.ext_target + row), 0.f);
         else u = __ldg(a.uniforms + (row + p * a.slot_stride));
     }
-    Partial t = reduce_segment<DT, 2, kGreedy>(g, rank * kWarps + warp, a.c, lane, slot0);
+    const float thr = kThr ? a.thr[row] : neg_inf();
+    Partial t = reduce_segment<DT, 2, kGreedy, kThr>(g, rank * kWarps + warp, a.c, lane, slot0, thr);
     if (lane == 0) { seg[warp].m = t.m; seg[warp].idx = t.idx; seg[warp].Z = t.Z; seg[warp].A = t.A; }
     cluster.sync();
     if (warp == 0) {
@@ -252,7 +257,7 @@ __global__ void __launch_bounds__(kThreads, kBlocks) draft_step_kernel(DraftArgs
     }
     if (!kGreedy && ok && P.seg / kWarps == rank) {
         SoftmaxWeights<DT> wf;
-        wf.g = g; wf.c = a.c; wf.M = __fmul_rn(R.m, a.c);
+        wf.g = g; wf.c = a.c; wf.M = __fmul_rn(R.m, a.c); wf.thr = thr;
         int v_lo, v_hi;
         seg_range(g, P.seg, v_lo, v_hi);
         int virt = fine_scan<EPV>(wf, v_lo, v_hi, P.prefix, P.target, scan, tid, lane, warp);
@@ -277,9 +282,10 @@ struct StatsArgs {
     unsigned* status;
     float4* out_partial;     // kMode 2: (m, Z, A, index of the maximum + idx_offset as int bits)
     int idx_offset;
+    const float* thr;        // kThr: truncation threshold per row (target rows: by target row; draft rows: by draft row)
 };
 
-template <int DT, int kMode>
+template <int DT, int kMode, bool kThr = false>
 __global__ void __launch_bounds__(kThreads) row_stats_kernel(StatsArgs a) {
     cg::cluster_group cluster = cg::this_cluster();
     const int S = cluster.dim_blocks().x;
@@ -306,7 +312,8 @@ __global__ void __launch_bounds__(kThreads) row_stats_kernel(StatsArgs a) {
                      static_cast<size_t>(in_row) * a.row_stride * ElemTraits<DT>::kBytes;
     const RowGeom g = make_geom<DT>(rp, a.V, S * kWarps);
     const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
-    Partial t = reduce_segment<DT, kMode, kMode != 1>(g, rank * kWarps + warp, a.c, lane, slot0);
+    const float thr = kThr ? a.thr[in_row] : neg_inf();
+    Partial t = reduce_segment<DT, kMode, kMode != 1, kThr>(g, rank * kWarps + warp, a.c, lane, slot0, thr);
     if (lane == 0) { seg[warp].m = t.m; seg[warp].idx = t.idx; seg[warp].Z = t.Z; seg[warp].A = t.A; }
     cluster.sync();
     if (rank == 0 && warp == 0) {
@@ -345,6 +352,8 @@ struct FinishArgs {
     int32_t* n_accepted;
     int32_t* next_token;
     unsigned* status;
+    const float* p_thr;           // kThr: truncation threshold of every target row
+    const float* q_thr;           // kThr: ... of every draft row (indexed like the draft tokens)
 };
 
 // Weights max(0, p - q) of Algorithm 4 (or p alone for the bonus token) for one vector.
@@ -354,13 +363,14 @@ struct ResidualWeights {
     const void* qrow;
     float c, Mp, rZp, Mq, rZq;
     int bonus;
+    float thr_p = -INFINITY, thr_q = -INFINITY;   // truncated distributions: logits below carry nothing
     __device__ __forceinline__ void operator()(int vi, float (&w)[ElemTraits<DT>::kEPV]) const {
         constexpr int EPV = ElemTraits<DT>::kEPV;
         float x[EPV];
         unpack_masked<DT>(__ldg(gt.base + vi), vi, gt, x);
 #pragma unroll
         for (int j = 0; j < EPV; ++j)
-            w[j] = ex2_approx(fmaxf(__fmaf_rn(x[j], c, -Mp), kArgFloor)) * rZp;
+            w[j] = x[j] >= thr_p ? ex2_approx(fmaxf(__fmaf_rn(x[j], c, -Mp), kArgFloor)) * rZp : 0.f;
         if (bonus) return;
         float d[EPV];
         if (gq.pre == gt.pre) {
@@ -375,7 +385,7 @@ struct ResidualWeights {
         }
 #pragma unroll
         for (int j = 0; j < EPV; ++j) {
-            float q = ex2_approx(fmaxf(__fmaf_rn(d[j], c, -Mq), kArgFloor)) * rZq;
+            float q = d[j] >= thr_q ? ex2_approx(fmaxf(__fmaf_rn(d[j], c, -Mq), kArgFloor)) * rZq : 0.f;
             w[j] = fmaxf(w[j] - q, 0.f);
         }
     }
@@ -385,7 +395,7 @@ struct ResidualWeights {
 // four stages for the target row and four for the draft row.  Same arithmetic as
 // ResidualWeights::weights (packed), without its masking: vectors that stick out of the row, and
 // rows whose draft row has another 16-byte phase, go through the functor instead.
-template <int DT>
+template <int DT, bool kThr>
 __device__ __forceinline__ float residual_segment_sum(const ResidualWeights<DT>& wf, int seg, int lane,
                                                       uint32_t slot0) {
     constexpr int EPV = ElemTraits<DT>::kEPV;
@@ -441,6 +451,10 @@ __device__ __forceinline__ float residual_segment_sum(const ResidualWeights<DT>&
         float x[EPV], d[EPV];
         ElemTraits<DT>::unpack(rt, x);
         ElemTraits<DT>::unpack(rq, d);
+        if (kThr) {
+            drop_below<EPV>(x, wf.thr_p);
+            drop_below<EPV>(d, wf.thr_q);
+        }
 #pragma unroll
         for (int j = 0; j < EPV; j += 2) {
             float a0, a1;
@@ -493,7 +507,7 @@ struct FinishShared {
     SegPick pick;
 };
 
-template <int DT>
+template <int DT, bool kThr = false>
 __global__ void __launch_bounds__(kThreads, 2) verify_finish_kernel(FinishArgs a) {
     using E = ElemTraits<DT>;
     constexpr int EPV = E::kEPV;
@@ -536,6 +550,10 @@ __global__ void __launch_bounds__(kThreads, 2) verify_finish_kernel(FinishArgs a
                     float eq = exp2f(fmaxf(__fmaf_rn(dv, a.c, -__fmul_rn(qs.x, a.c)), kArgFloor));
                     if (!(tv > neg_inf())) ep = 0.f;
                     if (!(dv > neg_inf())) eq = 0.f;
+                    if (kThr) {   // tokens that the truncation dropped have probability zero
+                        if (!(tv >= a.p_thr[row0 + j])) ep = 0.f;
+                        if (!(dv >= a.q_thr[dr])) eq = 0.f;
+                    }
                     // r < min(1, (ep/Zp)/(eq/Zq)) without the division: a ratio >= 1 accepts every
                     // r in [0,1); p(x) == 0 accepts none; q(x) == 0 < p(x) is a ratio of +inf
                     float r = a.uniforms[row0 + j];
@@ -561,6 +579,7 @@ __global__ void __launch_bounds__(kThreads, 2) verify_finish_kernel(FinishArgs a
         float2 ps = a.p_stats[row0 + n_acc];
         wf.Mp = __fmul_rn(ps.x, a.c);
         wf.rZp = 1.0f / ps.y;
+        if (kThr) wf.thr_p = a.p_thr[row0 + n_acc];
     }
     wf.bonus = n_acc >= Ki;
     wf.qrow = nullptr; wf.gq = wf.gt; wf.Mq = 0.f; wf.rZq = 0.f;
@@ -571,13 +590,14 @@ __global__ void __launch_bounds__(kThreads, 2) verify_finish_kernel(FinishArgs a
         float2 qs = a.q_stats_user ? a.q_stats_user[dr] : a.q_stats_ws[row0 + n_acc];
         wf.Mq = __fmul_rn(qs.x, a.c);
         wf.rZq = 1.0f / qs.y;
+        if (kThr) wf.thr_q = a.q_thr[dr];
     }
 
     int token = -1;
     for (int pass = 0; pass < 2; ++pass) {
         // mass of this warp's segment
         int v_lo, v_hi;
-        float acc = residual_segment_sum<DT>(wf, rank * kWarps + warp, lane, slot0);
+        float acc = residual_segment_sum<DT, kThr>(wf, rank * kWarps + warp, lane, slot0);
         acc = warp_sum(acc);
         if (lane == 0) { seg[warp].m = 0.f; seg[warp].idx = 0; seg[warp].Z = acc; seg[warp].A = 0.f; }
         cluster.sync();
@@ -1158,7 +1178,10 @@ int svip_create(svip_ctx** out, int device, int max_rows) {
             (const void*)row_stats_kernel<kF32, 0>,      (const void*)row_stats_kernel<kF32, 1>,
             (const void*)verify_finish_kernel<kBF16>,    (const void*)verify_finish_kernel<kF32>,
             (const void*)row_stats_kernel<kBF16, 2>,     (const void*)row_stats_kernel<kF32, 2>,
-            (const void*)row_threshold_kernel<kBF16>,    (const void*)row_threshold_kernel<kF32>};
+            (const void*)row_threshold_kernel<kBF16>,    (const void*)row_threshold_kernel<kF32>,
+            (const void*)draft_step_kernel<kBF16, false, 2, false, true>, (const void*)draft_step_kernel<kF32, false, 2, false, true>,
+            (const void*)row_stats_kernel<kBF16, 1, true>, (const void*)row_stats_kernel<kF32, 1, true>,
+            (const void*)verify_finish_kernel<kBF16, true>, (const void*)verify_finish_kernel<kF32, true>};
         for (const void* k : ringed)
             if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes) != cudaSuccess)
                 rc = SVIP_ERR_CUDA;
@@ -1230,6 +1253,11 @@ int svip_read_status(svip_ctx* ctx, unsigned* flags, void* stream) {
     return SVIP_OK;
 }
 
+static int draft_impl(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, int V, long row_stride,
+                      long pos_stride, const int32_t* pos, long slot_stride, float T, float thresh,
+                      const float* uniforms, const uint8_t* active, const float* thr, int32_t* token,
+                      float* entropy, uint8_t* stop, float* row_stats, void* stream);
+
 int svip_draft_step(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, int V, long row_stride,
                     float T, float thresh, const float* uniforms, int32_t* token, float* entropy,
                     uint8_t* stop, float* row_stats, void* stream) {
@@ -1248,6 +1276,22 @@ int svip_draft_step_at(svip_ctx* ctx, const void* logits, svip_dtype dtype, int 
                        long pos_stride, const int32_t* pos, long slot_stride, float T, float thresh,
                        const float* uniforms, const uint8_t* active, int32_t* token, float* entropy,
                        uint8_t* stop, float* row_stats, void* stream) {
+    return draft_impl(ctx, logits, dtype, B, V, row_stride, pos_stride, pos, slot_stride, T, thresh, uniforms, active,
+                      nullptr, token, entropy, stop, row_stats, stream);
+}
+
+int svip_draft_step_filtered(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, int V, long row_stride,
+                             float T, float thresh, const float* uniforms, const uint8_t* active, const float* thr,
+                             int32_t* token, float* entropy, uint8_t* stop, float* row_stats, void* stream) {
+    if (!thr || !(T > 0.f)) return SVIP_ERR_INVALID_ARG;
+    return draft_impl(ctx, logits, dtype, B, V, row_stride, 0, nullptr, 0, T, thresh, uniforms, active, thr, token,
+                      entropy, stop, row_stats, stream);
+}
+
+static int draft_impl(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, int V, long row_stride,
+                      long pos_stride, const int32_t* pos, long slot_stride, float T, float thresh,
+                      const float* uniforms, const uint8_t* active, const float* thr, int32_t* token,
+                      float* entropy, uint8_t* stop, float* row_stats, void* stream) {
     if (!ctx || !logits || !token || !entropy || !stop) return SVIP_ERR_INVALID_ARG;
     if (pos_stride < 0 || slot_stride < 0) return SVIP_ERR_INVALID_ARG;
     if (dtype != SVIP_F32 && dtype != SVIP_BF16) return SVIP_ERR_UNSUPPORTED;
@@ -1261,7 +1305,7 @@ int svip_draft_step_at(svip_ctx* ctx, const void* logits, svip_dtype dtype, int 
     a.greedy = T > 0.f ? 0 : 1; a.uniforms = uniforms; a.token = token; a.entropy = entropy;
     a.stop = stop; a.row_stats = row_stats; a.status = ctx->status; a.active = active;
     a.ext_target = nullptr; a.token_offset = 0;
-    a.pos = pos; a.pos_stride = pos_stride; a.slot_stride = slot_stride;
+    a.pos = pos; a.pos_stride = pos_stride; a.slot_stride = slot_stride; a.thr = thr;
     int S = pick_cluster(ctx, B, V, dtype);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool waves = static_cast<long>(B) * S > 2L * ctx->num_sms;
@@ -1276,6 +1320,7 @@ int svip_draft_step_at(svip_ctx* ctx, const void* logits, svip_dtype dtype, int 
         if (dtype == SVIP_BF16) k = a.greedy ? draft_step_kernel<kBF16, true, 2, true> : draft_step_kernel<kBF16, false, 2, true>;
         else k = a.greedy ? draft_step_kernel<kF32, true, 2, true> : draft_step_kernel<kF32, false, 2, true>;
     }
+    if (thr) k = dtype == SVIP_BF16 ? draft_step_kernel<kBF16, false, 2, false, true> : draft_step_kernel<kF32, false, 2, false, true>;
     cudaError_t e = launch_clustered(k, B, S, a, st, kRingBytes);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
@@ -1315,12 +1360,15 @@ int svip_pack_ragged(svip_ctx* ctx, const int32_t* draft_len, int B, int K_max, 
     return SVIP_OK;
 }
 
-int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits, long q_row_stride,
-                const float* q_stats, long q_seq_stride, long q_pos_stride, const void* target_logits,
-                long t_row_stride, svip_dtype dtype, const int32_t* cu_rows, int B, int K,
-                int n_target_rows, int V, float T, const float* uniforms, int32_t* n_accepted,
-                int32_t* next_token, void* stream) {
+// The verification round; q_thr / p_thr are both NULL (plain distributions) or both given
+// (distributions truncated at those per-row thresholds).
+static int verify_impl(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits, long q_row_stride,
+                       const float* q_stats, long q_seq_stride, long q_pos_stride, const void* target_logits,
+                       long t_row_stride, svip_dtype dtype, const int32_t* cu_rows, int B, int K,
+                       int n_target_rows, int V, float T, const float* uniforms, int32_t* n_accepted,
+                       int32_t* next_token, void* stream, const float* q_thr, const float* p_thr) {
     if (!ctx || !draft_tokens || !target_logits || !n_accepted || !next_token) return SVIP_ERR_INVALID_ARG;
+    const bool truncated = q_thr != nullptr;
     if (dtype != SVIP_F32 && dtype != SVIP_BF16) return SVIP_ERR_UNSUPPORTED;
     if (B < 0 || K < 1 || V < 1 || V > 0x7fffffe0 || t_row_stride < 0 || q_row_stride < 0) return SVIP_ERR_INVALID_ARG;
     if (!(T >= 0.f) || std::isinf(T)) return SVIP_ERR_INVALID_ARG;
@@ -1344,11 +1392,14 @@ int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits
     s.logits = target_logits; s.row_stride = t_row_stride; s.V = V; s.c = c; s.draft_rows = 0; s.K = K;
     s.cu = cu_rows; s.q_seq_stride = q_seq_stride; s.q_pos_stride = q_pos_stride;
     s.out_stats = ctx->p_stats; s.out_argmax = sampling ? nullptr : ctx->p_argmax; s.status = ctx->status;
-    s.out_partial = nullptr; s.idx_offset = 0;
+    s.out_partial = nullptr; s.idx_offset = 0; s.thr = p_thr;
     int S = pick_cluster(ctx, n_target_rows, V, dtype);
     const bool timed = ctx->profiling && !ctx->capturing && ctx->prof_used < kProfilePairs;
     if (timed) cudaEventRecord(ctx->prof_start[ctx->prof_used], st);
-    if (sampling)
+    if (truncated)
+        e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 1, true>, n_target_rows, S, s, st, kRingBytes)
+                               : launch_clustered(row_stats_kernel<kF32, 1, true>, n_target_rows, S, s, st, kRingBytes);
+    else if (sampling)
         e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 1>, n_target_rows, S, s, st, kRingBytes)
                                : launch_clustered(row_stats_kernel<kF32, 1>, n_target_rows, S, s, st, kRingBytes);
     else
@@ -1372,11 +1423,15 @@ int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits
     if (!q_stats) {
         StatsArgs d = s;
         d.logits = q_logits; d.row_stride = q_row_stride; d.draft_rows = 1;
-        d.out_stats = ctx->q_stats; d.out_argmax = nullptr;
+        d.out_stats = ctx->q_stats; d.out_argmax = nullptr; d.thr = q_thr;
         long units = static_cast<long>(B) * K;
         int Sd = pick_cluster(ctx, n_target_rows - B, V, dtype);
-        e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 1>, units, Sd, d, st, kRingBytes)
-                               : launch_clustered(row_stats_kernel<kF32, 1>, units, Sd, d, st, kRingBytes);
+        if (truncated)
+            e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 1, true>, units, Sd, d, st, kRingBytes)
+                                   : launch_clustered(row_stats_kernel<kF32, 1, true>, units, Sd, d, st, kRingBytes);
+        else
+            e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 1>, units, Sd, d, st, kRingBytes)
+                                   : launch_clustered(row_stats_kernel<kF32, 1>, units, Sd, d, st, kRingBytes);
         if (e != cudaSuccess) return cuda_fail(ctx, e);
         ctx->launches += 1;
     }
@@ -1387,6 +1442,7 @@ int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits
     f.q_seq_stride = q_seq_stride; f.q_pos_stride = q_pos_stride; f.t_logits = target_logits;
     f.t_row_stride = t_row_stride; f.p_stats = ctx->p_stats; f.cu = cu_rows; f.K = K; f.V = V; f.c = c;
     f.uniforms = uniforms; f.n_accepted = n_accepted; f.next_token = next_token; f.status = ctx->status;
+    f.p_thr = p_thr; f.q_thr = q_thr;
     // up to two rows per sequence are streamed: long rows are cut finer than the one-wave policy
     // asks for (this kernel runs for many microseconds, so several waves are fine)
     int Sf = pick_cluster(ctx, B, V, dtype);
@@ -1395,11 +1451,36 @@ int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits
         while (Sf < kMaxCluster && 2 * row_bytes / Sf > (512L << 10)) Sf *= 2;
         if (Sf > kMaxCluster) Sf = kMaxCluster;
     }
-    e = dtype == SVIP_BF16 ? launch_clustered(verify_finish_kernel<kBF16>, B, Sf, f, st, kRingBytes)
-                           : launch_clustered(verify_finish_kernel<kF32>, B, Sf, f, st, kRingBytes);
+    if (truncated)
+        e = dtype == SVIP_BF16 ? launch_clustered(verify_finish_kernel<kBF16, true>, B, Sf, f, st, kRingBytes)
+                               : launch_clustered(verify_finish_kernel<kF32, true>, B, Sf, f, st, kRingBytes);
+    else
+        e = dtype == SVIP_BF16 ? launch_clustered(verify_finish_kernel<kBF16>, B, Sf, f, st, kRingBytes)
+                               : launch_clustered(verify_finish_kernel<kF32>, B, Sf, f, st, kRingBytes);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
     return SVIP_OK;
+}
+
+int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits, long q_row_stride,
+                const float* q_stats, long q_seq_stride, long q_pos_stride, const void* target_logits,
+                long t_row_stride, svip_dtype dtype, const int32_t* cu_rows, int B, int K,
+                int n_target_rows, int V, float T, const float* uniforms, int32_t* n_accepted,
+                int32_t* next_token, void* stream) {
+    return verify_impl(ctx, draft_tokens, q_logits, q_row_stride, q_stats, q_seq_stride, q_pos_stride,
+                       target_logits, t_row_stride, dtype, cu_rows, B, K, n_target_rows, V, T, uniforms,
+                       n_accepted, next_token, stream, nullptr, nullptr);
+}
+
+int svip_verify_filtered(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits, long q_row_stride,
+                         const float* q_stats, const float* q_thr, long q_seq_stride, long q_pos_stride,
+                         const void* target_logits, long t_row_stride, const float* p_thr, svip_dtype dtype,
+                         const int32_t* cu_rows, int B, int K, int n_target_rows, int V, float T,
+                         const float* uniforms, int32_t* n_accepted, int32_t* next_token, void* stream) {
+    if (!q_thr || !p_thr || !(T > 0.f)) return SVIP_ERR_INVALID_ARG;
+    return verify_impl(ctx, draft_tokens, q_logits, q_row_stride, q_stats, q_seq_stride, q_pos_stride,
+                       target_logits, t_row_stride, dtype, cu_rows, B, K, n_target_rows, V, T, uniforms,
+                       n_accepted, next_token, stream, q_thr, p_thr);
 }
 
 int svip_profile_enable(svip_ctx* ctx, int on) {
@@ -1538,7 +1619,7 @@ int svip_vp_locate(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, i
     a.logits = logits; a.row_stride = row_stride; a.V = V_shard; a.c = scale_for(T); a.thresh = 0.f; a.greedy = 0;
     a.uniforms = nullptr; a.token = token; a.entropy = nullptr; a.stop = nullptr; a.row_stats = nullptr;
     a.status = ctx->status; a.active = active; a.ext_target = local_target; a.token_offset = vocab_offset;
-    a.pos = nullptr; a.pos_stride = 0; a.slot_stride = 0;
+    a.pos = nullptr; a.pos_stride = 0; a.slot_stride = 0; a.thr = nullptr;
     const int S = pick_cluster(ctx, B, V_shard, dtype);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = dtype == SVIP_BF16 ? launch_clustered(draft_step_kernel<kBF16, false, 2>, B, S, a, st, kRingBytes)

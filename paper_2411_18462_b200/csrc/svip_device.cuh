@@ -163,10 +163,13 @@ __device__ __forceinline__ float vec_max(const float (&x)[EPV]) {
 // 1 = max + Z, 2 = max + Z + A.
 template <int DT, int kMode>
 __device__ __forceinline__ void fold_vector(const uint4& raw, int vi, const RowGeom& g, float c,
-                                            Partial& t, float& M) {
+                                            Partial& t, float& M, float thr = -INFINITY) {
     constexpr int EPV = ElemTraits<DT>::kEPV;
     float x[EPV];
     unpack_masked<DT>(raw, vi, g, x);
+#pragma unroll
+    for (int j = 0; j < EPV; ++j)
+        if (!(x[j] >= thr)) x[j] = neg_inf();   // below the truncation threshold (or NaN): dropped
     float tmax = vec_max<EPV>(x);
     if (tmax > t.m) {
         float Mn = __fmul_rn(tmax, c);
@@ -198,7 +201,8 @@ __device__ __forceinline__ void fold_vector(const uint4& raw, int vi, const RowG
 // Slow path: streams segment `seg` with plain loads, an exact per-lane running maximum and
 // masking of -inf / NaN logits to zero mass.
 template <int DT, int kMode>
-__device__ __noinline__ Partial reduce_segment_slow(const RowGeom& g, int seg, float c, int lane) {
+__device__ __noinline__ Partial reduce_segment_slow(const RowGeom& g, int seg, float c, int lane,
+                                                    float thr = -INFINITY) {
     Partial t;
     t.m = neg_inf(); t.idx = kIntMax; t.Z = 0.f; t.A = 0.f;
     float M = neg_inf();
@@ -206,7 +210,7 @@ __device__ __noinline__ Partial reduce_segment_slow(const RowGeom& g, int seg, f
     seg_range(g, seg, v_lo, v_hi);
     for (int vi = v_lo + lane; vi < v_hi; vi += 32) {
         uint4 r0 = ld_stream(g.base + vi);
-        fold_vector<DT, kMode>(r0, vi, g, c, t, M);
+        fold_vector<DT, kMode>(r0, vi, g, c, t, M, thr);
     }
     return t;
 }
@@ -401,9 +405,18 @@ __device__ __forceinline__ Partial warp_merge(Partial t, float c) {
 // Streams segment `seg` of the row with the calling warp and returns the warp's merged partial
 // (all lanes hold it).  `slot0` is the shared-memory address of this thread's first ring slot;
 // slot s lives kThreads * 16 bytes further.  kIdx asks for the index of the maximum.
-template <int DT, int kMode, bool kIdx>
+// Logits below the truncation threshold get the stand-in that carries no mass.
+template <int EPV>
+__device__ __forceinline__ void drop_below(float (&x)[EPV], float thr) {
+#pragma unroll
+    for (int j = 0; j < EPV; ++j) x[j] = x[j] >= thr ? x[j] : kMasked;
+}
+
+// kThr: only logits >= thr count (truncated distributions); the reference of the exponentials is
+// still taken from the raw logits, so a segment without a kept logit simply sums to zero.
+template <int DT, int kMode, bool kIdx, bool kThr = false>
 __device__ __forceinline__ Partial reduce_segment(const RowGeom& g, int seg, float c, int lane,
-                                                  uint32_t slot0) {
+                                                  uint32_t slot0, float thr = -INFINITY) {
     constexpr int EPV = ElemTraits<DT>::kEPV;
     constexpr uint32_t kSlotStride = kThreads * 16;
     int v_lo, v_hi;
@@ -455,6 +468,7 @@ __device__ __forceinline__ Partial reduce_segment(const RowGeom& g, int seg, flo
         if (fold_head) {
             float x[EPV];
             unpack_edge<DT>(ld_stream(g.base), 0, g, x);
+            if (kThr) drop_below<EPV>(x, thr);
             fold_fast<EPV, kMode, kIdx>(x, 0, t);
         }
         int it = 0;
@@ -469,6 +483,7 @@ __device__ __forceinline__ Partial reduce_segment(const RowGeom& g, int seg, flo
                 cp_async_commit();
                 float x[EPV];
                 ElemTraits<DT>::unpack(raw, x);
+                if (kThr) drop_below<EPV>(x, thr);
                 fold_fast<EPV, kMode, kIdx>(x, vi0 + 32 * (it + s), t);
             }
             acc_check<kMode>(t, c);
@@ -484,6 +499,7 @@ __device__ __forceinline__ Partial reduce_segment(const RowGeom& g, int seg, flo
                 cp_async_commit();
                 float x[EPV];
                 ElemTraits<DT>::unpack(raw, x);
+                if (kThr) drop_below<EPV>(x, thr);
                 fold_fast<EPV, kMode, kIdx>(x, vi0 + 32 * (it + s), t);
             }
             acc_check<kMode>(t, c);
@@ -495,12 +511,14 @@ __device__ __forceinline__ Partial reduce_segment(const RowGeom& g, int seg, flo
             const uint4 raw = lds128(slot0 + (it & (kStages - 1)) * kSlotStride);
             float x[EPV];
             ElemTraits<DT>::unpack(raw, x);
+            if (kThr) drop_below<EPV>(x, thr);
             fold_fast<EPV, kMode, kIdx>(x, vi0 + 32 * it, t);
         }
         acc_check<kMode>(t, c);
         if (fold_tail) {
             float x[EPV];
             unpack_edge<DT>(ld_stream(g.base + g.nvec - 1), g.nvec - 1, g, x);
+            if (kThr) drop_below<EPV>(x, thr);
             fold_fast<EPV, kMode, kIdx>(x, g.nvec - 1, t);
             acc_check<kMode>(t, c);
         }
@@ -514,7 +532,7 @@ __device__ __forceinline__ Partial reduce_segment(const RowGeom& g, int seg, flo
     // +inf, NaN (from -inf or NaN logits, or an overflow between two checks): redo the segment
     if (kMode >= 1) bad = bad || !(fabsf(Z) <= 3.0e38f) || !(fabsf(A) <= 3.0e38f);
     if (__any_sync(0xffffffffu, bad)) {
-        Partial p = reduce_segment_slow<DT, kMode>(g, seg, c, lane);
+        Partial p = reduce_segment_slow<DT, kMode>(g, seg, c, lane, kThr ? thr : -INFINITY);
         return warp_merge<kMode>(p, c);
     }
     Partial r;

@@ -152,3 +152,98 @@ def test_threshold_bad_arguments(ctx):
         with pytest.raises(SvipError):
             ctx.row_threshold(x, 0, 4, a["V"], 64, a["T"], a["top_k"], a["top_p"], t)
     ctx.row_threshold(x, 0, 0, 64, 64, 1.0, 3, 0.9, t)      # no rows
+
+
+# ------------------------------------------------------------------ truncated draft step and verify
+
+def gpu_thresholds(ctx, rows, T, k, p):
+    import torch
+    d = tl.to_device(rows)
+    thr = torch.empty(rows.shape[0], device="cuda")
+    ctx.row_threshold(d, tl.dtype_code(rows), rows.shape[0], rows.shape[1], rows.shape[1], T, k, p, thr)
+    torch.cuda.synchronize()
+    return d, thr
+
+
+@pytest.mark.parametrize("dtype,V", [("bf16", 32000), ("f32", 50021), ("bf16", 152064)])
+@pytest.mark.parametrize("k,p", [(50, 1.0), (0, 0.9), (200, 0.8)])
+def test_filtered_draft_step_matches_the_oracle_on_the_kept_set(ctx, oracle, dtype, V, k, p):
+    import torch
+    rng = np.random.default_rng(V + k)
+    B, T, h = 24, 0.8, 0.3
+    x = (rng.standard_normal((B, V)) * rng.uniform(0.3, 5.0, size=(B, 1))).astype(np.float32)
+    x[2, rng.integers(0, V)] += 20.0
+    rows = W.to_bf16_bits(x) if dtype == "bf16" else x
+    u = rng.random(B).astype(np.float32)
+    d_rows, thr = gpu_thresholds(ctx, rows, T, k, p)
+    check(oracle, rows, T, k, p, thr.cpu().numpy(), "draft rows")
+    masked = oracle.mask_below(rows, thr.cpu().numpy().astype(np.float64))     # the kept set the GPU was given
+    for S in (0, 1, 3, 8):
+        ctx.set_cluster_size(S)
+        try:
+            tok = torch.full((B,), -7, dtype=torch.int32, device="cuda"); ent = torch.zeros(B, device="cuda")
+            stop = torch.zeros(B, dtype=torch.uint8, device="cuda"); stats = torch.zeros(B, 2, device="cuda")
+            ctx.draft_step_filtered(d_rows, tl.dtype_code(rows), B, V, V, T, h, tl.to_device(u), None, thr, tok, ent,
+                                    stop, stats)
+            torch.cuda.synchronize()
+        finally:
+            ctx.set_cluster_size(0)
+        got = (tok.cpu().numpy(), ent.cpu().numpy(), stop.cpu().numpy(), None)
+        tl.check_draft_against_oracle(oracle, masked, T, h, u, got, "filtered draft S=%d" % S)
+        vals = values_of(rows)
+        assert np.all(vals[np.arange(B), got[0]] >= thr.cpu().numpy()), "a sampled token lies outside the kept set"
+        # (m, Z) of the truncated distribution
+        st = stats.cpu().numpy()
+        for b in range(0, B, 5):
+            keep = vals[b] >= float(thr[b])
+            Z = np.exp((vals[b][keep] - vals[b].max()) / T).sum()
+            assert st[b, 0] == np.float32(vals[b].max()) and abs(st[b, 1] - Z) <= 1e-5 * Z
+    assert ctx.read_status() == 0
+
+
+@pytest.mark.parametrize("name,give_stats", [("chat", True), ("chat", False), ("tiny", True)])
+@pytest.mark.parametrize("k,p", [(40, 1.0), (0, 0.85), (300, 0.9)])
+def test_filtered_verify_matches_the_oracle(ctx, oracle, name, give_stats, k, p):
+    import torch
+    w = W.make_workload(name, B=8 if name == "chat" else None, K_max=6 if name == "chat" else None)
+    B, V, K, T = w.B, w.V, w.K_max, w.T
+    dt = tl.dtype_code(w.q_logits)
+    d_q, q_thr = gpu_thresholds(ctx, w.q_logits, T, k, p)
+    d_t, p_thr = gpu_thresholds(ctx, w.target_logits, T, k, p)
+    qm = oracle.mask_below(w.q_logits, q_thr.cpu().numpy().astype(np.float64))
+    tm = oracle.mask_below(w.target_logits, p_thr.cpu().numpy().astype(np.float64))
+    # draft tokens from the truncated draft distributions (GPU), with their normalisers
+    Rq = w.q_logits.shape[0]
+    tok = torch.zeros(Rq, dtype=torch.int32, device="cuda"); ent = torch.zeros(Rq, device="cuda")
+    stop = torch.zeros(Rq, dtype=torch.uint8, device="cuda"); stats = torch.zeros(Rq, 2, device="cuda")
+    ctx.draft_step_filtered(d_q, dt, Rq, V, V, T, w.h, tl.to_device(w.draft_uniforms.astype(np.float32)), None, q_thr,
+                            tok, ent, stop, stats)
+    torch.cuda.synchronize()
+    tokens = tok.cpu().numpy()
+    uv, moved = tl.guard_accept_uniforms(oracle, tokens, qm, tm, w.cu_rows, T, w.verify_uniforms, threads=8)
+    n_acc = torch.full((B,), -7, dtype=torch.int32, device="cuda"); nxt = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+    ctx.verify_filtered(tok, d_q, V, stats if give_stats else None, q_thr, -1, 0, d_t, V, p_thr, dt,
+                        tl.to_device(w.cu_rows.astype(np.int32)), B, K, w.n_target_rows, V, T, tl.to_device(uv), n_acc, nxt)
+    torch.cuda.synchronize()
+    got = (n_acc.cpu().numpy(), nxt.cpu().numpy())
+    c = tl.check_verify_against_oracle(oracle, tokens, qm, tm, w.cu_rows, T, uv, got, "filtered verify %s" % name)
+    # the emitted token is never one that the target's truncation dropped
+    tv = values_of(w.target_logits)
+    for i in range(B):
+        r = int(w.cu_rows[i]) + int(got[0][i])
+        assert tv[r, got[1][i]] >= float(p_thr[r])
+    assert 0 <= c["mean_accepted"] <= K
+    assert ctx.read_status() == 0
+
+
+def test_filtered_entry_points_reject_bad_arguments(ctx):
+    import torch
+    from paper_2411_18462_b200 import SvipError
+    x = torch.zeros(4, 64, device="cuda"); f = torch.zeros(8, device="cuda")
+    i = torch.zeros(8, dtype=torch.int32, device="cuda"); b = torch.zeros(8, dtype=torch.uint8, device="cuda")
+    with pytest.raises(SvipError):
+        ctx.draft_step_filtered(x, 0, 4, 64, 64, 1.0, 0.3, f, None, None, i, f, b)       # no thresholds
+    with pytest.raises(SvipError):
+        ctx.draft_step_filtered(x, 0, 4, 64, 64, 0.0, 0.3, f, None, f, i, f, b)          # greedy has nothing to truncate
+    with pytest.raises(SvipError):
+        ctx.verify_filtered(i, x, 64, None, None, -1, 0, x, 64, f, 0, None, 1, 1, 2, 64, 1.0, f, i, i)
