@@ -318,6 +318,58 @@ def b1_latency(ctx, torch):
     return out
 
 
+def truncated_round(ctx, torch, rnd, top_k=50, top_p=0.9, reps=10):
+    """The same round with top-k / nucleus truncated distributions, on the resident buffers of `rnd`:
+    thresholds of the draft rows of every step and of all target rows, truncated draft steps, truncated
+    verify.  Returns us per part and the logits GB/s of the whole truncated round."""
+    w, B, V, K = rnd.w, rnd.B, rnd.V, rnd.K
+    if not w.T > 0:
+        return None
+    sp = rnd.stream
+    dev = rnd.d_q.device
+    q_thr = torch.zeros(K * B, device=dev); p_thr = torch.zeros(rnd.Rp, device=dev)
+    q, ud, tok, ent = rnd.d_q.data_ptr(), rnd.d_ud.data_ptr(), rnd.d_tok.data_ptr(), rnd.d_ent.data_ptr()
+    stop, stats = rnd.d_stop.data_ptr(), rnd.d_stats.data_ptr()
+    thr_calls, draft_calls = [], []
+    for j in range(K):
+        o = j * B
+        a = int(rnd.active[j])
+        thr_calls.append(ctx.bind("row_threshold", q + o * V * rnd.esz, rnd.dt, a, V, V, w.T, top_k, top_p,
+                                  q_thr.data_ptr() + 4 * o, sp))
+        draft_calls.append(ctx.bind("draft_step_filtered", q + o * V * rnd.esz, rnd.dt, a, V, V, w.T, w.h, ud + 4 * o,
+                                    None, q_thr.data_ptr() + 4 * o, tok + 4 * o, ent + 4 * o, stop + o,
+                                    stats + 8 * o, sp))
+    t_thr = ctx.bind("row_threshold", rnd.d_t, rnd.dt, rnd.Rp, V, V, w.T, top_k, top_p, p_thr, sp)
+    pack = ctx.bind("pack_ragged", rnd.d_len, B, w.K_max, rnd.d_cu, None, None, sp)
+    ver = ctx.bind("verify_filtered", rnd.d_tok, rnd.d_q, V, rnd.d_stats, q_thr, 1, B, rnd.d_t, V, p_thr, rnd.dt,
+                   rnd.d_cu, B, w.K_max, rnd.Rp, V, w.T, rnd.d_uv, rnd.d_nacc, rnd.d_next, sp)
+
+    def timed(calls):
+        for c in calls:
+            c()
+        torch.cuda.synchronize()
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            for c in calls:
+                c()
+        e1.record()
+        torch.cuda.synchronize()
+        return 1000.0 * e0.elapsed_time(e1) / reps
+
+    out = {"top_k": top_k, "top_p": top_p,
+           "draft_thresholds_us": timed(thr_calls), "draft_steps_us": timed(draft_calls),
+           "target_thresholds_us": timed([t_thr]), "verify_us": timed([pack, ver])}
+    whole = [c for pair in zip(thr_calls, draft_calls) for c in pair] + [t_thr, pack, ver]
+    out["round_us"] = timed(whole)
+    nbytes, _ = rnd.logits_bytes()
+    out["logits_GBps"] = nbytes / (out["round_us"] * 1e-6) / 1e9
+    passes = (2 if w.dtype == "bf16" else 4) * ((1 if top_k else 0) + (1 if top_p < 1 else 0)) + \
+        (1 if (top_p < 1 and not top_k) else 0)
+    out["threshold_passes_per_row"] = passes
+    return out
+
+
 def cpu_baseline(w, seconds_budget=20.0):
     """The fp64 oracle, as it stands, on a bounded sample of the same workload, on all host cores."""
     from oracle import svip_oracle as O
@@ -468,6 +520,10 @@ def run_ours(args):
             line["b1"] = b1_latency(ctx, torch)
         except Exception as exc:   # the headline number does not depend on the latency probe
             line["b1"] = {"error": repr(exc)}
+        try:
+            line["truncated"] = truncated_round(ctx, torch, rnd)
+        except Exception as exc:
+            line["truncated"] = {"error": repr(exc)}
     if not args.no_cpu_baseline and not args.skip_extras:
         line["cpu_baseline"] = cpu_baseline(w)
     line["paper_context"] = ("end-to-end speedups over fixed draft length reported by the paper: up to 17% "

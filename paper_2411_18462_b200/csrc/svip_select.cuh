@@ -20,7 +20,8 @@
 
 namespace svip {
 
-constexpr int kHistCopies = 8;           // private histograms per block (one per pair of warps)
+constexpr int kHistCopies = 8;           // interleaved copies of the histogram: lane l adds into copy l % 8, so
+                                         // lanes that meet in one bin mostly hit different words and banks
 constexpr float kMassScale = 1099511627776.0f;   // 2^40
 
 struct ThresholdArgs {
@@ -75,7 +76,7 @@ __device__ __forceinline__ void stream_segment(const RowGeom& g, int seg, int la
 }
 
 struct SelectShared {
-    uint32_t priv[kHistCopies][3][256];   // per copy: count, mass low word, mass high word
+    uint32_t priv[3][256][kHistCopies];   // count, mass low word, mass high word; per digit, per copy
     uint32_t blk_cnt[256];                // this block's histogram, read by the peers
     unsigned long long blk_mass[256];
     uint32_t tot_cnt[256];                // the cluster's histogram
@@ -111,9 +112,9 @@ __device__ __forceinline__ void histogram_pass(cg::cluster_group& cluster, const
     const int lane = tid & 31, warp = tid >> 5;
     for (int i = tid; i < kHistCopies * 3 * 256; i += kThreads) (&sh.priv[0][0][0])[i] = 0;
     __syncthreads();
-    uint32_t* h_cnt = sh.priv[warp >> 1][0];
-    uint32_t* h_lo = sh.priv[warp >> 1][1];
-    uint32_t* h_hi = sh.priv[warp >> 1][2];
+    uint32_t* h_cnt = &sh.priv[0][0][lane % kHistCopies];
+    uint32_t* h_lo = &sh.priv[1][0][lane % kHistCopies];
+    uint32_t* h_hi = &sh.priv[2][0][lane % kHistCopies];
     float mx = neg_inf();
     unsigned long long ab = 0;
     const uint32_t want = first ? 0u : (prefix >> (shift + 8));
@@ -128,10 +129,12 @@ __device__ __forceinline__ void histogram_pass(cg::cluster_group& cluster, const
                 wq = __float2ull_rz(w * kMassScale);
                 if (kAbove && key >= key_k) ab += wq;
             }
-            if (first || (key >> (shift + 8)) == want) {
-                const uint32_t bin = (key >> shift) & 255u;
-                atomicAdd(h_cnt + bin, 1u);
-                if (kMass && wq) {
+            // the nucleus descent is decided by the masses alone, the top-k descent by the counts
+            if ((first || (key >> (shift + 8)) == want) && (!kMass || wq)) {
+                const uint32_t bin = ((key >> shift) & 255u) * kHistCopies;
+                if (!kMass) {
+                    atomicAdd(h_cnt + bin, 1u);
+                } else {
                     const uint32_t lo = static_cast<uint32_t>(wq);
                     const uint32_t old = atomicAdd(h_lo + bin, lo);
                     const uint32_t carry = (old + lo < old) ? 1u : 0u;
@@ -160,8 +163,8 @@ __device__ __forceinline__ void histogram_pass(cg::cluster_group& cluster, const
         unsigned long long ms = 0;
 #pragma unroll
         for (int k = 0; k < kHistCopies; ++k) {
-            cn += sh.priv[k][0][tid];
-            if (kMass) ms += (static_cast<unsigned long long>(sh.priv[k][2][tid]) << 32) + sh.priv[k][1][tid];
+            cn += sh.priv[0][tid][k];
+            if (kMass) ms += (static_cast<unsigned long long>(sh.priv[2][tid][k]) << 32) + sh.priv[1][tid][k];
         }
         sh.blk_cnt[tid] = cn;
         sh.blk_mass[tid] = ms;
