@@ -23,6 +23,8 @@ namespace svip {
 constexpr int kHistCopies = 8;           // interleaved copies of the histogram: lane l adds into copy l % 8, so
                                          // lanes that meet in one bin mostly hit different words and banks
 constexpr float kMassScale = 1099511627776.0f;   // 2^40
+constexpr int kCandPerBlock = 1024;      // candidate keys a block may collect
+constexpr int kPoolCap = 4096;           // candidate keys of the whole cluster (lives in the histogram copies)
 
 struct ThresholdArgs {
     const void* logits;
@@ -85,6 +87,10 @@ struct SelectShared {
     unsigned long long blk_above;         // this block's mass of the elements >= tau_k
     float warp_max[kWarps];
     unsigned long long warp_above[kWarps];
+    // candidate path (top-k with a small k)
+    uint32_t lane_key[kThreads];          // key of the largest logit each thread saw
+    uint32_t cand[kCandPerBlock];         // keys of this block's elements >= the lower bound
+    uint32_t cand_n;                      // how many there are (may exceed the capacity: then the path is left)
     // decision of a pass (written by warp 0)
     int bin;
     uint32_t cnt_above;
@@ -258,6 +264,151 @@ __device__ __forceinline__ void decide(SelectShared& sh, int lane, uint32_t k_re
     }
 }
 
+__device__ __forceinline__ unsigned long long mass_of_key(uint32_t key, float c, float M) {
+    const float w = ex2_approx(fmaxf(__fmaf_rn(key_value(key), c, -M), kArgFloor));
+    return __float2ull_rz(w * kMassScale);
+}
+
+// Radix descent over `n` keys held in shared memory, the same in every block of the cluster, so
+// no exchange is needed: the k_rem-th largest key (by counts), or the key at which the running mass
+// from the top reaches p_rem.  Block-collective.
+template <int kLevels, bool kByMass>
+__device__ __forceinline__ uint32_t pool_select(SelectShared& sh, const uint32_t* pool, int n, uint32_t k_rem,
+                                                unsigned long long p_rem, float c, float M, int tid) {
+    const int lane = tid & 31, warp = tid >> 5;
+    uint32_t prefix = 0;
+    for (int level = 0; level < kLevels; ++level) {
+        const int shift = 24 - 8 * level;
+        if (tid < 256) { sh.tot_cnt[tid] = 0; sh.tot_mass[tid] = 0; }
+        __syncthreads();
+        for (int i = tid; i < n; i += kThreads) {
+            const uint32_t key = pool[i];
+            if (level == 0 || (key >> (shift + 8)) == (prefix >> (shift + 8))) {
+                const uint32_t bin = (key >> shift) & 255u;
+                if (!kByMass) {
+                    atomicAdd(&sh.tot_cnt[bin], 1u);
+                } else {
+                    const unsigned long long wq = mass_of_key(key, c, M);
+                    if (wq) atomicAdd(&sh.tot_mass[bin], wq);
+                }
+            }
+        }
+        __syncthreads();
+        if (warp == 0) decide<kByMass>(sh, lane, k_rem, p_rem);
+        __syncthreads();
+        prefix |= static_cast<uint32_t>(sh.bin) << shift;
+        k_rem -= sh.cnt_above;
+        p_rem -= sh.mass_above;
+        __syncthreads();
+    }
+    if (kLevels == 2 && !(prefix & 0x80000000u)) prefix |= 0xffffu;
+    return prefix;
+}
+
+// Top-k (and the nucleus inside it) for a small k, in two passes over the row.  Pass 1 leaves the
+// largest logit of every thread; the k-th largest of these S * 512 values is a lower bound t0 of
+// tau_k (they are k distinct elements of the row).  Pass 2 collects every element >= t0 -- a few more
+// than k when k is small against the number of threads.  tau_k, the mass of the top-k set and the
+// nucleus cut then come from these candidates alone, which every block of the cluster holds in
+// full.  Returns false (for the whole cluster alike) when the candidates do not fit; nothing has
+// been written then and the caller takes the radix descent over the full row.
+template <int DT>
+__device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const RowGeom& g, int S, int rank, int tid,
+                                               uint32_t slot0, const ThresholdArgs& a, bool use_p, SelectShared& sh,
+                                               uint32_t& key_out) {
+    constexpr int EPV = ElemTraits<DT>::kEPV;
+    constexpr int kLevels = DT == kBF16 ? 2 : 4;
+    const int lane = tid & 31, warp = tid >> 5;
+    uint32_t* pool = &sh.priv[0][0][0];
+    static_assert(sizeof(sh.priv) >= kPoolCap * sizeof(uint32_t), "the pool lives in the histogram copies");
+    // pass 1: the largest key of every thread
+    uint32_t best = 0;
+    stream_segment<DT>(g, rank * kWarps + warp, lane, slot0, [&](const float (&x)[EPV], int) {
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) best = max(best, order_key(x[j]));
+    });
+    sh.lane_key[tid] = best;
+    if (tid == 0) sh.cand_n = 0;
+    cluster.sync();
+    const int n_lane = S * kThreads;
+    for (int r = 0; r < S; ++r) pool[r * kThreads + tid] = cluster.map_shared_rank(&sh, r)->lane_key[tid];
+    __syncthreads();
+    const uint32_t t0 = pool_select<kLevels, false>(sh, pool, n_lane, static_cast<uint32_t>(a.top_k), 0ull, 0.f, 0.f, tid);
+    // pass 2: every element at or above the lower bound
+    stream_segment<DT>(g, rank * kWarps + warp, lane, slot0, [&](const float (&x)[EPV], int) {
+#pragma unroll
+        for (int j = 0; j < EPV; ++j) {
+            const uint32_t key = order_key(x[j]);
+            if (key >= t0) {
+                const uint32_t pos = atomicAdd(&sh.cand_n, 1u);
+                if (pos < kCandPerBlock) sh.cand[pos] = key;
+            }
+        }
+    });
+    cluster.sync();     // every block's candidates are complete (and nobody still reads lane_key)
+    int total = 0, mine_at = 0;
+    bool fits = true;
+    for (int r = 0; r < S; ++r) {
+        const uint32_t nr = cluster.map_shared_rank(&sh, r)->cand_n;
+        if (nr > kCandPerBlock) fits = false;
+        if (r < rank) mine_at += static_cast<int>(min(nr, static_cast<uint32_t>(kCandPerBlock)));
+        total += static_cast<int>(min(nr, static_cast<uint32_t>(kCandPerBlock)));
+    }
+    if (total > kPoolCap) fits = false;
+    if (fits) {
+        int at = 0;
+        for (int r = 0; r < S; ++r) {
+            const SelectShared* peer = cluster.map_shared_rank(&sh, r);
+            const int nr = static_cast<int>(peer->cand_n);
+            for (int i = tid; i < nr; i += kThreads) pool[at + i] = peer->cand[i];
+            at += nr;
+        }
+    }
+    (void)mine_at;
+    cluster.sync();     // the peers have read this block's candidates
+    if (!fits) return false;
+    uint32_t key_k = pool_select<kLevels, false>(sh, pool, total, static_cast<uint32_t>(a.top_k), 0ull, 0.f, 0.f, tid);
+    uint32_t key_t = key_k;
+    if (use_p) {
+        // the largest candidate is the largest logit of the row
+        uint32_t top = 0;
+        for (int i = tid; i < total; i += kThreads) top = max(top, pool[i]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) top = max(top, __shfl_xor_sync(0xffffffffu, top, o));
+        if (lane == 0) sh.warp_max[warp] = __uint_as_float(top);
+        __syncthreads();
+        top = 0;
+        for (int w = 0; w < kWarps; ++w) top = max(top, __float_as_uint(sh.warp_max[w]));
+        const float row_max = key_value(top);
+        const bool finite = fabsf(row_max) <= kMaxLogit;
+        const float M = finite ? __fmul_rn(row_max, a.c) : 0.f;
+        unsigned long long zk = 0;
+        for (int i = tid; i < total; i += kThreads)
+            if (pool[i] >= key_k) zk += mass_of_key(pool[i], a.c, M);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            uint32_t lo = __shfl_xor_sync(0xffffffffu, static_cast<uint32_t>(zk), o);
+            uint32_t hi = __shfl_xor_sync(0xffffffffu, static_cast<uint32_t>(zk >> 32), o);
+            zk += (static_cast<unsigned long long>(hi) << 32) | lo;
+        }
+        __syncthreads();   // warp_max has been read
+        if (lane == 0) sh.warp_above[warp] = zk;
+        __syncthreads();
+        zk = 0;
+        for (int w = 0; w < kWarps; ++w) zk += sh.warp_above[w];
+        if (finite && zk > 0) {
+            const double want = ceil(static_cast<double>(a.top_p) * static_cast<double>(zk));
+            unsigned long long p_rem = static_cast<unsigned long long>(want);
+            if (p_rem < 1) p_rem = 1;
+            if (p_rem > zk) p_rem = zk;
+            const uint32_t key_p = pool_select<kLevels, true>(sh, pool, total, 0u, p_rem, a.c, M, tid);
+            if (key_p > key_t) key_t = key_p;
+        }
+    }
+    key_out = key_t;
+    return true;
+}
+
 template <int DT>
 __global__ void __launch_bounds__(kThreads, 2) row_threshold_kernel(ThresholdArgs a) {
     constexpr int kLevels = DT == kBF16 ? 2 : 4;   // the low 16 bits of a bf16 logit carry nothing
@@ -281,6 +432,15 @@ __global__ void __launch_bounds__(kThreads, 2) row_threshold_kernel(ThresholdArg
     unsigned long long above = 0;
     bool have_max = false;
     uint32_t key_k = 0;       // key of tau_k (0: below every key, nothing dropped)
+
+    // a small k against the number of threads of the cluster: two passes and a handful of candidates
+    if (use_k && a.top_k <= (S * kThreads) / 4) {
+        uint32_t key_t = 0;
+        if (candidate_path<DT>(cluster, g, S, rank, tid, slot0, a, use_p, sh, key_t)) {
+            if (rank == 0 && tid == 0) a.thr[row] = key_t ? key_value(key_t) : neg_inf();
+            return;
+        }
+    }
 
     if (use_k) {
         uint32_t prefix = 0, k_rem = static_cast<uint32_t>(a.top_k);
