@@ -171,8 +171,10 @@ int svip_draft_step_at(svip_ctx* ctx, const void* logits, svip_dtype dtype, int 
  * masses (summed as 2^-40 fixed point, so the result does not depend on the
  * order of summation) and may differ from an fp64 evaluation where the running
  * mass comes within about 1e-6 of top_p.  T > 0.  NaN logits count as -inf.
- * Every row is read once per radix pass: 2 (bf16) or 4 (fp32) passes for top-k,
- * as many again for the nucleus (+1 for the nucleus alone).
+ * Cost: with a small top_k (at most a quarter of the threads that share a row,
+ * i.e. 128 .. 1024) every row is read twice, with or without top_p; otherwise
+ * once per radix pass: 2 (bf16) or 4 (fp32) passes for top-k, as many again
+ * for the nucleus (+1 for the nucleus alone).
  *   logits  DEVICE, row r starts at element r*row_stride;  thr  DEVICE [n_rows] fp32 out
  */
 int svip_row_threshold(svip_ctx* ctx, const void* logits, svip_dtype dtype, int n_rows, int V,
@@ -282,6 +284,10 @@ int svip_pack_ragged(svip_ctx* ctx, const int32_t* draft_len, int B, int K_max,
  *   n_accepted     DEVICE [B] int32 out, in [0, K_i]
  *   next_token     DEVICE [B] int32 out
  * Needs n_target_rows <= max_rows of svip_create (else SVIP_ERR_WORKSPACE).
+ * Probabilities are fp32: where p and q of the rejected position agree to
+ * within about 1e-6 in total (a rejection there has that probability), the
+ * residual is at rounding level and next_token is only approximately
+ * distributed as Algorithm 4 asks.
  */
 int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits,
                 long q_row_stride, const float* q_stats, long q_seq_stride, long q_pos_stride,

@@ -546,19 +546,21 @@ __global__ void __launch_bounds__(kThreads, 2) verify_finish_kernel(FinishArgs a
                     float dv = E::load_one(ql + static_cast<size_t>(dr) * a.q_row_stride * E::kBytes, x);
                     float2 ps = a.p_stats[row0 + j];
                     float2 qs = a.q_stats_user ? a.q_stats_user[dr] : a.q_stats_ws[row0 + j];
-                    float ep = exp2f(fmaxf(__fmaf_rn(tv, a.c, -__fmul_rn(ps.x, a.c)), kArgFloor));
-                    float eq = exp2f(fmaxf(__fmaf_rn(dv, a.c, -__fmul_rn(qs.x, a.c)), kArgFloor));
-                    if (!(tv > neg_inf())) ep = 0.f;
-                    if (!(dv > neg_inf())) eq = 0.f;
+                    // p(x)/q(x) = 2^(ap - aq) * Zq / Zp, from the difference of the two log2 arguments, so
+                    // that a token however unlikely under both models keeps its ratio (no underflow)
+                    const float ap = __fmaf_rn(tv, a.c, -__fmul_rn(ps.x, a.c));
+                    const float aq = __fmaf_rn(dv, a.c, -__fmul_rn(qs.x, a.c));
+                    bool p_zero = !(tv > neg_inf()), q_zero = !(dv > neg_inf());   // NaN counts as -inf
                     if (kThr) {   // tokens that the truncation dropped have probability zero
-                        if (!(tv >= a.p_thr[row0 + j])) ep = 0.f;
-                        if (!(dv >= a.q_thr[dr])) eq = 0.f;
+                        p_zero = p_zero || !(tv >= a.p_thr[row0 + j]);
+                        q_zero = q_zero || !(dv >= a.q_thr[dr]);
                     }
-                    // r < min(1, (ep/Zp)/(eq/Zq)) without the division: a ratio >= 1 accepts every
-                    // r in [0,1); p(x) == 0 accepts none; q(x) == 0 < p(x) is a ratio of +inf
-                    float r = a.uniforms[row0 + j];
-                    float lhs = __fmul_rn(eq, ps.y), rhs = __fmul_rn(ep, qs.y);
-                    acc = ep > 0.f && (rhs >= lhs || __fmul_rn(r, lhs) < rhs);
+                    // r < min(1, ratio) without the division: a ratio >= 1 accepts every r in [0,1);
+                    // p(x) == 0 accepts none; q(x) == 0 < p(x) is a ratio of +inf
+                    const float r = a.uniforms[row0 + j];
+                    const float d = fminf(fmaxf(ap - aq, -126.f), 126.f);
+                    const float num = __fmul_rn(exp2f(d), qs.y);
+                    acc = !p_zero && (q_zero || num >= ps.y || __fmul_rn(r, ps.y) < num);
                 }
                 rej = !acc;
             }

@@ -7,7 +7,8 @@
 // published definitions (top-k, nucleus sampling) read with a threshold so that the result does not
 // depend on the order of equal logits.
 //
-// One cluster per row.  The value is found by a radix descent over an order-preserving integer
+// One cluster per row.  Top-k with a small k takes two passes and a handful of candidates (see
+// candidate_path below).  Otherwise the value is found by a radix descent over an order-preserving integer
 // image of the logits, 8 bits per pass: every pass streams the row once (cp.async ring, as the other
 // kernels), histograms the digit of the elements that match the digits already fixed (counts, and
 // for the nucleus the masses 2^(l*c - M) in 2^-40 fixed point, so that every sum is an integer and
@@ -346,12 +347,11 @@ __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const
         }
     });
     cluster.sync();     // every block's candidates are complete (and nobody still reads lane_key)
-    int total = 0, mine_at = 0;
+    int total = 0;
     bool fits = true;
     for (int r = 0; r < S; ++r) {
         const uint32_t nr = cluster.map_shared_rank(&sh, r)->cand_n;
         if (nr > kCandPerBlock) fits = false;
-        if (r < rank) mine_at += static_cast<int>(min(nr, static_cast<uint32_t>(kCandPerBlock)));
         total += static_cast<int>(min(nr, static_cast<uint32_t>(kCandPerBlock)));
     }
     if (total > kPoolCap) fits = false;
@@ -364,7 +364,6 @@ __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const
             at += nr;
         }
     }
-    (void)mine_at;
     cluster.sync();     // the peers have read this block's candidates
     if (!fits) return false;
     uint32_t key_k = pool_select<kLevels, false>(sh, pool, total, static_cast<uint32_t>(a.top_k), 0ull, 0.f, 0.f, tid);

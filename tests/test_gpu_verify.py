@@ -205,3 +205,34 @@ def test_published_configs(ctx, oracle, name):
         tl.check_verify_against_oracle(oracle, tok.astype(np.int32), w.q_logits, t2, w.cu_rows, 1.0,
                                        w.verify_uniforms, got, "tiny all-accept")
     assert ctx.read_status() == 0
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_accept_ratio_of_very_unlikely_tokens(ctx, oracle, bf16):
+    """Draft tokens that both models find almost impossible (probabilities far below the smallest fp32
+    number) still have a well-defined ratio p(x)/q(x); the accept count must follow it (Algorithm 2), not
+    the ratio of two underflowed exponentials.  Only the accept counts are compared: at such positions
+    p and q may agree so closely that the residual of Algorithm 4 is below fp32 resolution."""
+    rng = np.random.default_rng(31)
+    B, V, K, T = 48, 20011, 1, 0.5
+    base = (rng.standard_normal((B, V)) * 8.0).astype(np.float32)          # margins of ~60 logits, /T -> 120
+    tgt_first = base + (rng.standard_normal((B, V)) * 1.5).astype(np.float32)
+    tgt = np.empty((2 * B, V), np.float32)
+    tgt[0::2] = tgt_first
+    tgt[1::2] = base                                                       # the bonus row, unused here
+    q = base.copy()
+    if bf16:
+        q = W.to_bf16_bits(q); tgt = W.to_bf16_bits(tgt)
+    qv = W.bf16_bits_to_f32(q) if bf16 else q
+    tok = qv.argmin(axis=1).astype(np.int32)                               # the least likely token of each row
+    margin = (qv.max(axis=1) - qv[np.arange(B), tok]) / T * 1.4427
+    assert margin.min() > 127                                              # below 2^-127 under the draft model
+    cu = (np.arange(B + 1) * 2).astype(np.int64)
+    uv = rng.random(2 * B).astype(np.float32)
+    uv, _ = tl.guard_accept_uniforms(oracle, tok, q, tgt, cu, T, uv, threads=8)
+    n_g, _ = tl.gpu_verify(ctx, tok, q, tgt, cu, K, T, uv)
+    n_o, _, ap = oracle.verify(tok, q, tgt, cu, T, uv.astype(np.float64), want_accept_prob=True, threads=8)
+    assert np.array_equal(n_g.astype(np.int64), n_o)
+    probs = np.array([a[0] for a in ap])
+    assert (probs < 0.9).sum() > 5 and (probs >= 1.0).sum() > 5            # both outcomes are exercised
+    assert 0 < n_o.sum() < B
