@@ -39,10 +39,10 @@ struct ThresholdArgs {
 
 // Monotone image of a float: a < b  <=>  key(a) < key(b).  NaN counts as -inf.
 __device__ __forceinline__ uint32_t order_key(float x) {
-    if (!(x == x)) x = neg_inf();
-    if (x == 0.f) x = 0.f;          // -0 and +0 are one value
+    x = fmaxf(x, neg_inf());        // NaN -> -inf (the maximum of a NaN and a number is the number)
+    x = x + 0.f;                    // -0 -> +0: the two zeros are one value
     const uint32_t u = __float_as_uint(x);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    return u ^ (static_cast<uint32_t>(static_cast<int32_t>(u) >> 31) | 0x80000000u);
 }
 
 __device__ __forceinline__ float key_value(uint32_t key) {
@@ -322,27 +322,31 @@ __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const
     const int lane = tid & 31, warp = tid >> 5;
     uint32_t* pool = &sh.priv[0][0][0];
     static_assert(sizeof(sh.priv) >= kPoolCap * sizeof(uint32_t), "the pool lives in the histogram copies");
-    // pass 1: the largest key of every thread
-    uint32_t best = 0;
+    // pass 1: the largest logit of every thread (fmaxf skips NaN); threads without elements keep key 0
+    float best = neg_inf();
+    bool any = false;
     stream_segment<DT>(g, rank * kWarps + warp, lane, slot0, [&](const float (&x)[EPV], int) {
+        any = true;
 #pragma unroll
-        for (int j = 0; j < EPV; ++j) best = max(best, order_key(x[j]));
+        for (int j = 0; j < EPV; ++j) best = fmaxf(best, x[j]);
     });
-    sh.lane_key[tid] = best;
+    sh.lane_key[tid] = any ? order_key(best) : 0u;
     if (tid == 0) sh.cand_n = 0;
     cluster.sync();
     const int n_lane = S * kThreads;
     for (int r = 0; r < S; ++r) pool[r * kThreads + tid] = cluster.map_shared_rank(&sh, r)->lane_key[tid];
     __syncthreads();
     const uint32_t t0 = pool_select<kLevels, false>(sh, pool, n_lane, static_cast<uint32_t>(a.top_k), 0ull, 0.f, 0.f, tid);
-    // pass 2: every element at or above the lower bound
+    // pass 2: every element at or above the lower bound.  Comparing the logits is comparing the keys,
+    // except for NaN, which counts as -inf and so belongs to the candidates only when the bound is that low.
+    const float t0v = t0 ? key_value(t0) : neg_inf();
+    const bool lowest = !(t0v > neg_inf());
     stream_segment<DT>(g, rank * kWarps + warp, lane, slot0, [&](const float (&x)[EPV], int) {
 #pragma unroll
         for (int j = 0; j < EPV; ++j) {
-            const uint32_t key = order_key(x[j]);
-            if (key >= t0) {
+            if (x[j] >= t0v || (lowest && !(x[j] == x[j]))) {
                 const uint32_t pos = atomicAdd(&sh.cand_n, 1u);
-                if (pos < kCandPerBlock) sh.cand[pos] = key;
+                if (pos < kCandPerBlock) sh.cand[pos] = order_key(x[j]);
             }
         }
     });
@@ -365,7 +369,7 @@ __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const
         }
     }
     cluster.sync();     // the peers have read this block's candidates
-    if (!fits) return false;
+    if (!fits || total < a.top_k) return false;
     uint32_t key_k = pool_select<kLevels, false>(sh, pool, total, static_cast<uint32_t>(a.top_k), 0ull, 0.f, 0.f, tid);
     uint32_t key_t = key_k;
     if (use_p) {
