@@ -328,6 +328,7 @@ def truncated_round(ctx, torch, rnd, top_k=50, top_p=0.9, reps=10):
     sp = rnd.stream
     dev = rnd.d_q.device
     q_thr = torch.zeros(K * B, device=dev); p_thr = torch.zeros(rnd.Rp, device=dev)
+    p_stats = torch.zeros(rnd.Rp, 2, device=dev)
     q, ud, tok, ent = rnd.d_q.data_ptr(), rnd.d_ud.data_ptr(), rnd.d_tok.data_ptr(), rnd.d_ent.data_ptr()
     stop, stats = rnd.d_stop.data_ptr(), rnd.d_stats.data_ptr()
     thr_calls, draft_calls = [], []
@@ -335,13 +336,13 @@ def truncated_round(ctx, torch, rnd, top_k=50, top_p=0.9, reps=10):
         o = j * B
         a = int(rnd.active[j])
         thr_calls.append(ctx.bind("row_threshold", q + o * V * rnd.esz, rnd.dt, a, V, V, w.T, top_k, top_p,
-                                  q_thr.data_ptr() + 4 * o, sp))
+                                  q_thr.data_ptr() + 4 * o, None, sp))
         draft_calls.append(ctx.bind("draft_step_filtered", q + o * V * rnd.esz, rnd.dt, a, V, V, w.T, w.h, ud + 4 * o,
                                     None, q_thr.data_ptr() + 4 * o, tok + 4 * o, ent + 4 * o, stop + o,
                                     stats + 8 * o, sp))
-    t_thr = ctx.bind("row_threshold", rnd.d_t, rnd.dt, rnd.Rp, V, V, w.T, top_k, top_p, p_thr, sp)
+    t_thr = ctx.bind("row_threshold", rnd.d_t, rnd.dt, rnd.Rp, V, V, w.T, top_k, top_p, p_thr, p_stats, sp)
     pack = ctx.bind("pack_ragged", rnd.d_len, B, w.K_max, rnd.d_cu, None, None, sp)
-    ver = ctx.bind("verify_filtered", rnd.d_tok, rnd.d_q, V, rnd.d_stats, q_thr, 1, B, rnd.d_t, V, p_thr, rnd.dt,
+    ver = ctx.bind("verify_filtered", rnd.d_tok, rnd.d_q, V, rnd.d_stats, q_thr, 1, B, rnd.d_t, V, p_thr, p_stats, rnd.dt,
                    rnd.d_cu, B, w.K_max, rnd.Rp, V, w.T, rnd.d_uv, rnd.d_nacc, rnd.d_next, sp)
 
     def timed(calls):

@@ -176,9 +176,15 @@ int svip_draft_step_at(svip_ctx* ctx, const void* logits, svip_dtype dtype, int 
  * once per radix pass: 2 (bf16) or 4 (fp32) passes for top-k, as many again
  * for the nucleus (+1 for the nucleus alone).
  *   logits  DEVICE, row r starts at element r*row_stride;  thr  DEVICE [n_rows] fp32 out
+ *   stats   DEVICE [n_rows][2] fp32 out, or NULL: (m, Z) of the truncated
+ *           distribution in the convention of svip_draft_step's row_stats (m the
+ *           largest logit, Z the mass of the kept set relative to it), 8-byte
+ *           aligned; svip_verify_filtered takes them as p_stats.  Free with a
+ *           small top_k; one more pass over the row otherwise.
  */
 int svip_row_threshold(svip_ctx* ctx, const void* logits, svip_dtype dtype, int n_rows, int V,
-                       long row_stride, float T, int top_k, float top_p, float* thr, void* stream);
+                       long row_stride, float T, int top_k, float top_p, float* thr, float* stats,
+                       void* stream);
 
 /*
  * The draft step and the verification round on truncated distributions: every
@@ -191,6 +197,8 @@ int svip_row_threshold(svip_ctx* ctx, const void* logits, svip_dtype dtype, int 
  *   thr     DEVICE [B] fp32: threshold of each draft row of this step
  *   q_thr   DEVICE fp32, indexed like draft_tokens / q_stats (by draft row)
  *   p_thr   DEVICE [n_target_rows] fp32
+ *   p_stats DEVICE [n_target_rows][2] fp32 from svip_row_threshold, or NULL
+ *           (then one more pass over the target rows computes them)
  * row_stats / q_stats hold (m, Z) of the truncated distribution.  Other
  * arguments as for svip_draft_step_masked and svip_verify.
  */
@@ -201,9 +209,10 @@ int svip_draft_step_filtered(svip_ctx* ctx, const void* logits, svip_dtype dtype
 int svip_verify_filtered(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits,
                          long q_row_stride, const float* q_stats, const float* q_thr,
                          long q_seq_stride, long q_pos_stride, const void* target_logits,
-                         long t_row_stride, const float* p_thr, svip_dtype dtype,
-                         const int32_t* cu_rows, int B, int K, int n_target_rows, int V, float T,
-                         const float* uniforms, int32_t* n_accepted, int32_t* next_token, void* stream);
+                         long t_row_stride, const float* p_thr, const float* p_stats,
+                         svip_dtype dtype, const int32_t* cu_rows, int B, int K, int n_target_rows,
+                         int V, float T, const float* uniforms, int32_t* n_accepted,
+                         int32_t* next_token, void* stream);
 
 /*
  * Draft-length policies, kept on the device so that the drafting loop needs no

@@ -80,12 +80,12 @@ def library():
     L.svip_graph_loop_end.restype = i32
     L.svip_graph_loop_end.argtypes = [vp]
     L.svip_row_threshold.restype = i32
-    L.svip_row_threshold.argtypes = [vp, vp, i32, i32, i32, lng, f32, i32, f32, vp, vp]
+    L.svip_row_threshold.argtypes = [vp, vp, i32, i32, i32, lng, f32, i32, f32, vp, vp, vp]
     L.svip_draft_step_filtered.restype = i32
     L.svip_draft_step_filtered.argtypes = [vp, vp, i32, i32, i32, lng, f32, f32, vp, vp, vp, vp, vp, vp, vp, vp]
     L.svip_verify_filtered.restype = i32
-    L.svip_verify_filtered.argtypes = [vp, vp, vp, lng, vp, vp, lng, lng, vp, lng, vp, i32, vp, i32, i32, i32, i32,
-                                       f32, vp, vp, vp, vp]
+    L.svip_verify_filtered.argtypes = [vp, vp, vp, lng, vp, vp, lng, lng, vp, lng, vp, vp, i32, vp, i32, i32, i32,
+                                       i32, f32, vp, vp, vp, vp]
     L.svip_policy_advance.restype = i32
     L.svip_policy_advance.argtypes = [vp, i32, vp, vp, vp, vp, i32, i32, vp, vp]
     L.svip_policy_update.restype = i32
@@ -210,9 +210,10 @@ class Context:
                                             _ptr(uniforms), _ptr(active), _ptr(token), _ptr(entropy), _ptr(stop),
                                             _ptr(row_stats), _stream(stream)), self._h)
 
-    def row_threshold(self, logits, dtype, n_rows, V, row_stride, T, top_k, top_p, thr, stream=None):
+    def row_threshold(self, logits, dtype, n_rows, V, row_stride, T, top_k, top_p, thr, stats=None, stream=None):
         _check(library().svip_row_threshold(self._h, _ptr(logits), int(dtype), int(n_rows), int(V), int(row_stride),
-                                            float(T), int(top_k), float(top_p), _ptr(thr), _stream(stream)), self._h)
+                                            float(T), int(top_k), float(top_p), _ptr(thr), _ptr(stats),
+                                            _stream(stream)), self._h)
 
     def draft_step_filtered(self, logits, dtype, B, V, row_stride, T, thresh, uniforms, active, thr, token, entropy,
                             stop, row_stats=None, stream=None):
@@ -223,10 +224,11 @@ class Context:
 
     def verify_filtered(self, draft_tokens, q_logits, q_row_stride, q_stats, q_thr, q_seq_stride, q_pos_stride,
                         target_logits, t_row_stride, p_thr, dtype, cu_rows, B, K, n_target_rows, V, T, uniforms,
-                        n_accepted, next_token, stream=None):
+                        n_accepted, next_token, p_stats=None, stream=None):
         _check(library().svip_verify_filtered(
             self._h, _ptr(draft_tokens), _ptr(q_logits), int(q_row_stride), _ptr(q_stats), _ptr(q_thr),
-            int(q_seq_stride), int(q_pos_stride), _ptr(target_logits), int(t_row_stride), _ptr(p_thr), int(dtype),
+            int(q_seq_stride), int(q_pos_stride), _ptr(target_logits), int(t_row_stride), _ptr(p_thr),
+            _ptr(p_stats), int(dtype),
             _ptr(cu_rows), int(B), int(K), int(n_target_rows), int(V), float(T), _ptr(uniforms), _ptr(n_accepted),
             _ptr(next_token), _stream(stream)), self._h)
 

@@ -1330,7 +1330,7 @@ static int draft_impl(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B
 }
 
 int svip_row_threshold(svip_ctx* ctx, const void* logits, svip_dtype dtype, int n_rows, int V, long row_stride,
-                       float T, int top_k, float top_p, float* thr, void* stream) {
+                       float T, int top_k, float top_p, float* thr, float* stats, void* stream) {
     if (!ctx || !logits || !thr) return SVIP_ERR_INVALID_ARG;
     if (dtype != SVIP_F32 && dtype != SVIP_BF16) return SVIP_ERR_UNSUPPORTED;
     if (n_rows < 0 || V < 1 || V > 0x7fffffe0 || row_stride < 0 || top_k < 0) return SVIP_ERR_INVALID_ARG;
@@ -1340,6 +1340,8 @@ int svip_row_threshold(svip_ctx* ctx, const void* logits, svip_dtype dtype, int 
     ThresholdArgs a;
     a.logits = logits; a.row_stride = row_stride; a.V = V; a.c = scale_for(T);
     a.top_k = (top_k >= 1 && top_k < V) ? top_k : 0; a.top_p = top_p; a.thr = thr;
+    a.stats = reinterpret_cast<float2*>(stats);
+    if (stats && !aligned_to(stats, 8)) return SVIP_ERR_INVALID_ARG;
     const int S = pick_cluster(ctx, n_rows, V, dtype);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = dtype == SVIP_BF16 ? launch_clustered(row_threshold_kernel<kBF16>, n_rows, S, a, st, kRingBytes)
@@ -1368,7 +1370,8 @@ static int verify_impl(svip_ctx* ctx, const int32_t* draft_tokens, const void* q
                        const float* q_stats, long q_seq_stride, long q_pos_stride, const void* target_logits,
                        long t_row_stride, svip_dtype dtype, const int32_t* cu_rows, int B, int K,
                        int n_target_rows, int V, float T, const float* uniforms, int32_t* n_accepted,
-                       int32_t* next_token, void* stream, const float* q_thr, const float* p_thr) {
+                       int32_t* next_token, void* stream, const float* q_thr, const float* p_thr,
+                       const float* p_stats_user) {
     if (!ctx || !draft_tokens || !target_logits || !n_accepted || !next_token) return SVIP_ERR_INVALID_ARG;
     const bool truncated = q_thr != nullptr;
     if (dtype != SVIP_F32 && dtype != SVIP_BF16) return SVIP_ERR_UNSUPPORTED;
@@ -1398,7 +1401,9 @@ static int verify_impl(svip_ctx* ctx, const int32_t* draft_tokens, const void* q
     int S = pick_cluster(ctx, n_target_rows, V, dtype);
     const bool timed = ctx->profiling && !ctx->capturing && ctx->prof_used < kProfilePairs;
     if (timed) cudaEventRecord(ctx->prof_start[ctx->prof_used], st);
-    if (truncated)
+    if (p_stats_user)
+        e = cudaSuccess;   // the caller already holds (m, Z) of every target row
+    else if (truncated)
         e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 1, true>, n_target_rows, S, s, st, kRingBytes)
                                : launch_clustered(row_stats_kernel<kF32, 1, true>, n_target_rows, S, s, st, kRingBytes);
     else if (sampling)
@@ -1408,7 +1413,7 @@ static int verify_impl(svip_ctx* ctx, const int32_t* draft_tokens, const void* q
         e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 0>, n_target_rows, S, s, st, kRingBytes)
                                : launch_clustered(row_stats_kernel<kF32, 0>, n_target_rows, S, s, st, kRingBytes);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
-    ctx->launches += 1;
+    if (!p_stats_user) ctx->launches += 1;
     if (timed) cudaEventRecord(ctx->prof_stop[ctx->prof_used++], st);
 
     if (!sampling) {
@@ -1442,7 +1447,9 @@ static int verify_impl(svip_ctx* ctx, const int32_t* draft_tokens, const void* q
     f.draft_tokens = draft_tokens; f.q_logits = q_logits; f.q_row_stride = q_row_stride;
     f.q_stats_user = reinterpret_cast<const float2*>(q_stats); f.q_stats_ws = ctx->q_stats;
     f.q_seq_stride = q_seq_stride; f.q_pos_stride = q_pos_stride; f.t_logits = target_logits;
-    f.t_row_stride = t_row_stride; f.p_stats = ctx->p_stats; f.cu = cu_rows; f.K = K; f.V = V; f.c = c;
+    f.t_row_stride = t_row_stride;
+    f.p_stats = p_stats_user ? reinterpret_cast<const float2*>(p_stats_user) : ctx->p_stats;
+    f.cu = cu_rows; f.K = K; f.V = V; f.c = c;
     f.uniforms = uniforms; f.n_accepted = n_accepted; f.next_token = next_token; f.status = ctx->status;
     f.p_thr = p_thr; f.q_thr = q_thr;
     // up to two rows per sequence are streamed: long rows are cut finer than the one-wave policy
@@ -1471,18 +1478,19 @@ int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits
                 int32_t* next_token, void* stream) {
     return verify_impl(ctx, draft_tokens, q_logits, q_row_stride, q_stats, q_seq_stride, q_pos_stride,
                        target_logits, t_row_stride, dtype, cu_rows, B, K, n_target_rows, V, T, uniforms,
-                       n_accepted, next_token, stream, nullptr, nullptr);
+                       n_accepted, next_token, stream, nullptr, nullptr, nullptr);
 }
 
 int svip_verify_filtered(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits, long q_row_stride,
                          const float* q_stats, const float* q_thr, long q_seq_stride, long q_pos_stride,
-                         const void* target_logits, long t_row_stride, const float* p_thr, svip_dtype dtype,
-                         const int32_t* cu_rows, int B, int K, int n_target_rows, int V, float T,
+                         const void* target_logits, long t_row_stride, const float* p_thr, const float* p_stats,
+                         svip_dtype dtype, const int32_t* cu_rows, int B, int K, int n_target_rows, int V, float T,
                          const float* uniforms, int32_t* n_accepted, int32_t* next_token, void* stream) {
     if (!q_thr || !p_thr || !(T > 0.f)) return SVIP_ERR_INVALID_ARG;
+    if (p_stats && !aligned_to(p_stats, 8)) return SVIP_ERR_INVALID_ARG;
     return verify_impl(ctx, draft_tokens, q_logits, q_row_stride, q_stats, q_seq_stride, q_pos_stride,
                        target_logits, t_row_stride, dtype, cu_rows, B, K, n_target_rows, V, T, uniforms,
-                       n_accepted, next_token, stream, q_thr, p_thr);
+                       n_accepted, next_token, stream, q_thr, p_thr, p_stats);
 }
 
 int svip_profile_enable(svip_ctx* ctx, int on) {

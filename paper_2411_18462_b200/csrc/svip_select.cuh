@@ -35,6 +35,7 @@ struct ThresholdArgs {
     int top_k;      // 1 .. V-1, or 0 when off
     float top_p;    // (0, 1), or >= 1 when off
     float* thr;     // [rows] out: tau as a logit value (-inf: nothing is dropped)
+    float2* stats;  // [rows] out or NULL: (largest logit, mass of the kept set relative to it)
 };
 
 // Monotone image of a float: a < b  <=>  key(a) < key(b).  NaN counts as -inf.
@@ -265,6 +266,28 @@ __device__ __forceinline__ void decide(SelectShared& sh, int lane, uint32_t k_re
     }
 }
 
+// Sum of one 64-bit integer per thread over the block (every thread gets it).  Two barriers.
+__device__ __forceinline__ unsigned long long block_sum_u64(SelectShared& sh, unsigned long long v, int tid) {
+    const int lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        uint32_t lo = __shfl_xor_sync(0xffffffffu, static_cast<uint32_t>(v), o);
+        uint32_t hi = __shfl_xor_sync(0xffffffffu, static_cast<uint32_t>(v >> 32), o);
+        v += (static_cast<unsigned long long>(hi) << 32) | lo;
+    }
+    __syncthreads();   // warp_above may still be read from an earlier use
+    if (lane == 0) sh.warp_above[warp] = v;
+    __syncthreads();
+    v = 0;
+    for (int w = 0; w < kWarps; ++w) v += sh.warp_above[w];
+    return v;
+}
+
+// What the statistics output holds for a row: (m, Z~) in the convention of the draft step's row_stats.
+__device__ __forceinline__ float2 kept_stats(float row_max, unsigned long long kept_mass, bool finite) {
+    return make_float2(row_max, finite ? static_cast<float>(static_cast<double>(kept_mass) / 1099511627776.0) : 0.f);
+}
+
 __device__ __forceinline__ unsigned long long mass_of_key(uint32_t key, float c, float M) {
     const float w = ex2_approx(fmaxf(__fmaf_rn(key_value(key), c, -M), kArgFloor));
     return __float2ull_rz(w * kMassScale);
@@ -372,7 +395,10 @@ __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const
     if (!fits || total < a.top_k) return false;
     uint32_t key_k = pool_select<kLevels, false>(sh, pool, total, static_cast<uint32_t>(a.top_k), 0ull, 0.f, 0.f, tid);
     uint32_t key_t = key_k;
-    if (use_p) {
+    float row_max = neg_inf();
+    bool finite = false;
+    float M = 0.f;
+    if (use_p || a.stats) {
         // the largest candidate is the largest logit of the row
         uint32_t top = 0;
         for (int i = tid; i < total; i += kThreads) top = max(top, pool[i]);
@@ -382,23 +408,15 @@ __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const
         __syncthreads();
         top = 0;
         for (int w = 0; w < kWarps; ++w) top = max(top, __float_as_uint(sh.warp_max[w]));
-        const float row_max = key_value(top);
-        const bool finite = fabsf(row_max) <= kMaxLogit;
-        const float M = finite ? __fmul_rn(row_max, a.c) : 0.f;
+        row_max = key_value(top);
+        finite = fabsf(row_max) <= kMaxLogit;
+        M = finite ? __fmul_rn(row_max, a.c) : 0.f;
+    }
+    if (use_p) {
         unsigned long long zk = 0;
         for (int i = tid; i < total; i += kThreads)
             if (pool[i] >= key_k) zk += mass_of_key(pool[i], a.c, M);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            uint32_t lo = __shfl_xor_sync(0xffffffffu, static_cast<uint32_t>(zk), o);
-            uint32_t hi = __shfl_xor_sync(0xffffffffu, static_cast<uint32_t>(zk >> 32), o);
-            zk += (static_cast<unsigned long long>(hi) << 32) | lo;
-        }
-        __syncthreads();   // warp_max has been read
-        if (lane == 0) sh.warp_above[warp] = zk;
-        __syncthreads();
-        zk = 0;
-        for (int w = 0; w < kWarps; ++w) zk += sh.warp_above[w];
+        zk = block_sum_u64(sh, zk, tid);
         if (finite && zk > 0) {
             const double want = ceil(static_cast<double>(a.top_p) * static_cast<double>(zk));
             unsigned long long p_rem = static_cast<unsigned long long>(want);
@@ -407,6 +425,13 @@ __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const
             const uint32_t key_p = pool_select<kLevels, true>(sh, pool, total, 0u, p_rem, a.c, M, tid);
             if (key_p > key_t) key_t = key_p;
         }
+    }
+    if (a.stats) {
+        unsigned long long zt = 0;
+        for (int i = tid; i < total; i += kThreads)
+            if (pool[i] >= key_t) zt += mass_of_key(pool[i], a.c, M);
+        zt = block_sum_u64(sh, zt, tid);
+        if (rank == 0 && tid == 0) a.stats[blockIdx.x / S] = kept_stats(row_max, zt, finite);
     }
     key_out = key_t;
     return true;
@@ -469,7 +494,7 @@ __global__ void __launch_bounds__(kThreads, 2) row_threshold_kernel(ThresholdArg
     }
 
     uint32_t key_t = key_k;
-    if (use_p) {
+    if (use_p || a.stats) {
         if (!have_max) {
             // the masses are taken relative to the largest logit: find it first
             float mx = neg_inf();
@@ -492,6 +517,8 @@ __global__ void __launch_bounds__(kThreads, 2) row_threshold_kernel(ThresholdArg
             row_max = m;
             cluster.sync();
         }
+    }
+    if (use_p) {
         const bool finite = fabsf(row_max) <= kMaxLogit;
         const float M = finite ? __fmul_rn(row_max, a.c) : 0.f;
         uint32_t prefix = 0;
@@ -523,7 +550,29 @@ __global__ void __launch_bounds__(kThreads, 2) row_threshold_kernel(ThresholdArg
         key_t = key_p > key_k ? key_p : key_k;
     }
     if (rank == 0 && tid == 0) a.thr[row] = key_t ? key_value(key_t) : neg_inf();
-    // the last pass ended with a cluster barrier after all remote reads: blocks may leave
+    if (a.stats) {
+        // the mass of the kept set: one more pass (the descents above know it only in part)
+        const bool finite = fabsf(row_max) <= kMaxLogit;
+        const float M = finite ? __fmul_rn(row_max, a.c) : 0.f;
+        unsigned long long kept = 0;
+        stream_segment<DT>(g, rank * kWarps + warp, lane, slot0, [&](const float (&x)[ElemTraits<DT>::kEPV], int) {
+#pragma unroll
+            for (int j = 0; j < ElemTraits<DT>::kEPV; ++j) {
+                if (order_key(x[j]) >= key_t) {
+                    const float w = ex2_approx(fmaxf(__fmaf_rn(x[j], a.c, -M), kArgFloor));
+                    kept += __float2ull_rz(w * kMassScale);
+                }
+            }
+        });
+        kept = block_sum_u64(sh, kept, tid);
+        if (tid == 0) sh.blk_above = kept;
+        cluster.sync();
+        unsigned long long all = 0;
+        for (int r = 0; r < S; ++r) all += cluster.map_shared_rank(&sh, r)->blk_above;
+        if (rank == 0 && tid == 0) a.stats[row] = kept_stats(row_max, all, finite);
+        cluster.sync();   // the peers have read this block's sum
+    }
+    // every pass ended with a cluster barrier after all remote reads: blocks may leave
 }
 
 }  // namespace svip

@@ -128,6 +128,13 @@ def test_both_off_drops_nothing(ctx):
     x = (rng.standard_normal((3, 5000)) * 2).astype(np.float32)
     got = gpu_threshold(ctx, x, 1.0, 0, 1.0)
     assert np.all(got == -np.inf)
+    # the statistics are then those of the whole row
+    import torch
+    st = torch.zeros(3, 2, device="cuda"); thr = torch.zeros(3, device="cuda")
+    ctx.row_threshold(tl.to_device(x), 0, 3, 5000, 5000, 1.0, 0, 1.0, thr, st)
+    torch.cuda.synchronize()
+    Z = np.exp(x.astype(np.float64) - x.max(axis=1, keepdims=True)).sum(axis=1)
+    assert np.array_equal(st.cpu().numpy()[:, 0], x.max(axis=1)) and np.allclose(st.cpu().numpy()[:, 1], Z, rtol=1e-5)
 
 
 def test_published_shapes(ctx, oracle):
@@ -156,11 +163,11 @@ def test_threshold_bad_arguments(ctx):
 
 # ------------------------------------------------------------------ truncated draft step and verify
 
-def gpu_thresholds(ctx, rows, T, k, p):
+def gpu_thresholds(ctx, rows, T, k, p, stats=None):
     import torch
     d = tl.to_device(rows)
     thr = torch.empty(rows.shape[0], device="cuda")
-    ctx.row_threshold(d, tl.dtype_code(rows), rows.shape[0], rows.shape[1], rows.shape[1], T, k, p, thr)
+    ctx.row_threshold(d, tl.dtype_code(rows), rows.shape[0], rows.shape[1], rows.shape[1], T, k, p, thr, stats)
     torch.cuda.synchronize()
     return d, thr
 
@@ -202,14 +209,23 @@ def test_filtered_draft_step_matches_the_oracle_on_the_kept_set(ctx, oracle, dty
 
 
 @pytest.mark.parametrize("name,give_stats", [("chat", True), ("chat", False), ("tiny", True)])
-@pytest.mark.parametrize("k,p", [(40, 1.0), (0, 0.85), (300, 0.9)])
+@pytest.mark.parametrize("k,p", [(40, 1.0), (0, 0.85), (300, 0.9), (2000, 0.95)])
 def test_filtered_verify_matches_the_oracle(ctx, oracle, name, give_stats, k, p):
     import torch
     w = W.make_workload(name, B=8 if name == "chat" else None, K_max=6 if name == "chat" else None)
     B, V, K, T = w.B, w.V, w.K_max, w.T
     dt = tl.dtype_code(w.q_logits)
     d_q, q_thr = gpu_thresholds(ctx, w.q_logits, T, k, p)
-    d_t, p_thr = gpu_thresholds(ctx, w.target_logits, T, k, p)
+    # with give_stats the normalisers of the target rows come from the threshold kernel as well
+    p_stats = torch.full((w.n_target_rows, 2), -5.0, device="cuda") if give_stats else None
+    d_t, p_thr = gpu_thresholds(ctx, w.target_logits, T, k, p, p_stats)
+    if give_stats:
+        tv_all = values_of(w.target_logits)
+        ps = p_stats.cpu().numpy()
+        for r in range(0, w.n_target_rows, 7):
+            keep = tv_all[r] >= float(p_thr[r])
+            Z = np.exp((tv_all[r][keep] - tv_all[r].max()) / T).sum()
+            assert ps[r, 0] == np.float32(tv_all[r].max()) and abs(ps[r, 1] - Z) <= 1e-5 * Z, (r, ps[r], Z)
     qm = oracle.mask_below(w.q_logits, q_thr.cpu().numpy().astype(np.float64))
     tm = oracle.mask_below(w.target_logits, p_thr.cpu().numpy().astype(np.float64))
     # draft tokens from the truncated draft distributions (GPU), with their normalisers
@@ -222,8 +238,11 @@ def test_filtered_verify_matches_the_oracle(ctx, oracle, name, give_stats, k, p)
     tokens = tok.cpu().numpy()
     uv, moved = tl.guard_accept_uniforms(oracle, tokens, qm, tm, w.cu_rows, T, w.verify_uniforms, threads=8)
     n_acc = torch.full((B,), -7, dtype=torch.int32, device="cuda"); nxt = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+    launches = ctx.launch_count()
     ctx.verify_filtered(tok, d_q, V, stats if give_stats else None, q_thr, -1, 0, d_t, V, p_thr, dt,
-                        tl.to_device(w.cu_rows.astype(np.int32)), B, K, w.n_target_rows, V, T, tl.to_device(uv), n_acc, nxt)
+                        tl.to_device(w.cu_rows.astype(np.int32)), B, K, w.n_target_rows, V, T, tl.to_device(uv), n_acc, nxt,
+                        p_stats=p_stats)
+    assert ctx.launch_count() - launches == (1 if give_stats else 3)     # no pass over rows whose (m, Z) is given
     torch.cuda.synchronize()
     got = (n_acc.cpu().numpy(), nxt.cpu().numpy())
     c = tl.check_verify_against_oracle(oracle, tokens, qm, tm, w.cu_rows, T, uv, got, "filtered verify %s" % name)
@@ -247,3 +266,5 @@ def test_filtered_entry_points_reject_bad_arguments(ctx):
         ctx.draft_step_filtered(x, 0, 4, 64, 64, 0.0, 0.3, f, None, f, i, f, b)          # greedy has nothing to truncate
     with pytest.raises(SvipError):
         ctx.verify_filtered(i, x, 64, None, None, -1, 0, x, 64, f, 0, None, 1, 1, 2, 64, 1.0, f, i, i)
+    with pytest.raises(SvipError):
+        ctx.row_threshold(x, 0, 4, 64, 64, 1.0, 3, 0.9, f, f.data_ptr() + 4)                 # stats must be 8-byte aligned
