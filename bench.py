@@ -331,7 +331,7 @@ def truncated_round(ctx, torch, rnd, top_k=50, top_p=0.9, reps=10):
     p_stats = torch.zeros(rnd.Rp, 2, device=dev)
     q, ud, tok, ent = rnd.d_q.data_ptr(), rnd.d_ud.data_ptr(), rnd.d_tok.data_ptr(), rnd.d_ent.data_ptr()
     stop, stats = rnd.d_stop.data_ptr(), rnd.d_stats.data_ptr()
-    thr_calls, draft_calls = [], []
+    thr_calls, draft_calls, one_calls = [], [], []
     for j in range(K):
         o = j * B
         a = int(rnd.active[j])
@@ -340,6 +340,9 @@ def truncated_round(ctx, torch, rnd, top_k=50, top_p=0.9, reps=10):
         draft_calls.append(ctx.bind("draft_step_filtered", q + o * V * rnd.esz, rnd.dt, a, V, V, w.T, w.h, ud + 4 * o,
                                     None, q_thr.data_ptr() + 4 * o, tok + 4 * o, ent + 4 * o, stop + o,
                                     stats + 8 * o, sp))
+        one_calls.append(ctx.bind("draft_step_truncated", q + o * V * rnd.esz, rnd.dt, a, V, V, w.T, w.h, top_k, top_p,
+                                  ud + 4 * o, None, q_thr.data_ptr() + 4 * o, tok + 4 * o, ent + 4 * o, stop + o,
+                                  stats + 8 * o, sp))
     t_thr = ctx.bind("row_threshold", rnd.d_t, rnd.dt, rnd.Rp, V, V, w.T, top_k, top_p, p_thr, p_stats, sp)
     pack = ctx.bind("pack_ragged", rnd.d_len, B, w.K_max, rnd.d_cu, None, None, sp)
     ver = ctx.bind("verify_filtered", rnd.d_tok, rnd.d_q, V, rnd.d_stats, q_thr, 1, B, rnd.d_t, V, p_thr, p_stats, rnd.dt,
@@ -360,8 +363,9 @@ def truncated_round(ctx, torch, rnd, top_k=50, top_p=0.9, reps=10):
 
     out = {"top_k": top_k, "top_p": top_p,
            "draft_thresholds_us": timed(thr_calls), "draft_steps_us": timed(draft_calls),
+           "draft_steps_one_call_us": timed(one_calls),
            "target_thresholds_us": timed([t_thr]), "verify_us": timed([pack, ver])}
-    whole = [c for pair in zip(thr_calls, draft_calls) for c in pair] + [t_thr, pack, ver]
+    whole = one_calls + [t_thr, pack, ver]
     out["round_us"] = timed(whole)
     nbytes, _ = rnd.logits_bytes()
     out["logits_GBps"] = nbytes / (out["round_us"] * 1e-6) / 1e9

@@ -206,6 +206,22 @@ int svip_draft_step_filtered(svip_ctx* ctx, const void* logits, svip_dtype dtype
                              long row_stride, float T, float thresh, const float* uniforms,
                              const uint8_t* active, const float* thr, int32_t* token, float* entropy,
                              uint8_t* stop, float* row_stats, void* stream);
+/*
+ * svip_row_threshold and svip_draft_step_filtered in one call: thr[b] receives
+ * the threshold of row b for (top_k, top_p), and token / entropy / stop /
+ * row_stats the truncated draft step at it.  With a small top_k (see
+ * svip_row_threshold) the first kernel finishes the whole step from the few
+ * candidates it holds in shared memory, two passes over the row in all; rows
+ * it cannot finish that way (nucleus alone, large top_k, many ties at the cut)
+ * go through the streaming kernel in a second launch, which skips the others.
+ * Results are those of the two separate calls within the stated tolerances
+ * (sums are formed in another order).  B <= max_rows of svip_create.
+ */
+int svip_draft_step_truncated(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, int V,
+                              long row_stride, float T, float thresh, int top_k, float top_p,
+                              const float* uniforms, const uint8_t* active, float* thr,
+                              int32_t* token, float* entropy, uint8_t* stop, float* row_stats,
+                              void* stream);
 int svip_verify_filtered(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits,
                          long q_row_stride, const float* q_stats, const float* q_thr,
                          long q_seq_stride, long q_pos_stride, const void* target_logits,

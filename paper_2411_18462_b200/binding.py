@@ -83,6 +83,8 @@ def library():
     L.svip_row_threshold.argtypes = [vp, vp, i32, i32, i32, lng, f32, i32, f32, vp, vp, vp]
     L.svip_draft_step_filtered.restype = i32
     L.svip_draft_step_filtered.argtypes = [vp, vp, i32, i32, i32, lng, f32, f32, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.svip_draft_step_truncated.restype = i32
+    L.svip_draft_step_truncated.argtypes = [vp, vp, i32, i32, i32, lng, f32, f32, i32, f32, vp, vp, vp, vp, vp, vp, vp, vp]
     L.svip_verify_filtered.restype = i32
     L.svip_verify_filtered.argtypes = [vp, vp, vp, lng, vp, vp, lng, lng, vp, lng, vp, vp, i32, vp, i32, i32, i32,
                                        i32, f32, vp, vp, vp, vp]
@@ -221,6 +223,13 @@ class Context:
                                                   float(T), float(thresh), _ptr(uniforms), _ptr(active), _ptr(thr),
                                                   _ptr(token), _ptr(entropy), _ptr(stop), _ptr(row_stats),
                                                   _stream(stream)), self._h)
+
+    def draft_step_truncated(self, logits, dtype, B, V, row_stride, T, thresh, top_k, top_p, uniforms, active, thr,
+                             token, entropy, stop, row_stats=None, stream=None):
+        _check(library().svip_draft_step_truncated(self._h, _ptr(logits), int(dtype), int(B), int(V), int(row_stride),
+                                                   float(T), float(thresh), int(top_k), float(top_p), _ptr(uniforms),
+                                                   _ptr(active), _ptr(thr), _ptr(token), _ptr(entropy), _ptr(stop),
+                                                   _ptr(row_stats), _stream(stream)), self._h)
 
     def verify_filtered(self, draft_tokens, q_logits, q_row_stride, q_stats, q_thr, q_seq_stride, q_pos_stride,
                         target_logits, t_row_stride, p_thr, dtype, cu_rows, B, K, n_target_rows, V, T, uniforms,

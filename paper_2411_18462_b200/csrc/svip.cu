@@ -1031,6 +1031,7 @@ struct svip_ctx {
     float2* q_stats;
     int32_t* p_argmax;
     unsigned* status;
+    uint8_t* need;             // device [max_rows]: rows that svip_draft_step_truncated leaves to the streaming kernel
     int* loop_iter;            // device: iteration counter of the drafting loop being replayed
     cudaStream_t loop_stream;  // records the body of a drafting loop
     int loop_open;             // a loop body is being recorded
@@ -1181,6 +1182,7 @@ int svip_create(svip_ctx** out, int device, int max_rows) {
             (const void*)verify_finish_kernel<kBF16>,    (const void*)verify_finish_kernel<kF32>,
             (const void*)row_stats_kernel<kBF16, 2>,     (const void*)row_stats_kernel<kF32, 2>,
             (const void*)row_threshold_kernel<kBF16>,    (const void*)row_threshold_kernel<kF32>,
+            (const void*)row_threshold_kernel<kBF16, true>, (const void*)row_threshold_kernel<kF32, true>,
             (const void*)draft_step_kernel<kBF16, false, 2, false, true>, (const void*)draft_step_kernel<kF32, false, 2, false, true>,
             (const void*)row_stats_kernel<kBF16, 1, true>, (const void*)row_stats_kernel<kF32, 1, true>,
             (const void*)verify_finish_kernel<kBF16, true>, (const void*)verify_finish_kernel<kF32, true>};
@@ -1195,6 +1197,7 @@ int svip_create(svip_ctx** out, int device, int max_rows) {
             cudaMalloc(&c->p_argmax, n * sizeof(int32_t)) != cudaSuccess ||
             cudaMalloc(&c->status, sizeof(unsigned)) != cudaSuccess ||
             cudaMemset(c->status, 0, sizeof(unsigned)) != cudaSuccess ||
+            cudaMalloc(&c->need, n) != cudaSuccess ||
             cudaMalloc(&c->loop_iter, sizeof(int)) != cudaSuccess ||
             cudaMemset(c->loop_iter, 0, sizeof(int)) != cudaSuccess) {
             rc = SVIP_ERR_CUDA;
@@ -1203,7 +1206,7 @@ int svip_create(svip_ctx** out, int device, int max_rows) {
     if (rc != SVIP_OK) {
         cudaGetLastError();
         cudaFree(c->p_stats); cudaFree(c->q_stats); cudaFree(c->p_argmax); cudaFree(c->status);
-        cudaFree(c->loop_iter);
+        cudaFree(c->loop_iter); cudaFree(c->need);
         delete c;
     } else {
         *out = c;
@@ -1218,7 +1221,7 @@ int svip_destroy(svip_ctx* ctx) {
     cudaGetDevice(&prev);
     cudaSetDevice(ctx->device);
     cudaFree(ctx->p_stats); cudaFree(ctx->q_stats); cudaFree(ctx->p_argmax); cudaFree(ctx->status);
-    cudaFree(ctx->loop_iter);
+    cudaFree(ctx->loop_iter); cudaFree(ctx->need);
     if (ctx->loop_stream) cudaStreamDestroy(ctx->loop_stream);
     if (ctx->prof_start) {
         for (int k = 0; k < kProfilePairs; ++k) {
@@ -1342,6 +1345,8 @@ int svip_row_threshold(svip_ctx* ctx, const void* logits, svip_dtype dtype, int 
     a.top_k = (top_k >= 1 && top_k < V) ? top_k : 0; a.top_p = top_p; a.thr = thr;
     a.stats = reinterpret_cast<float2*>(stats);
     if (stats && !aligned_to(stats, 8)) return SVIP_ERR_INVALID_ARG;
+    a.uniforms = nullptr; a.active = nullptr; a.thresh = 0.f; a.token = nullptr; a.entropy = nullptr;
+    a.stop = nullptr; a.need = nullptr;
     const int S = pick_cluster(ctx, n_rows, V, dtype);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = dtype == SVIP_BF16 ? launch_clustered(row_threshold_kernel<kBF16>, n_rows, S, a, st, kRingBytes)
@@ -1349,6 +1354,36 @@ int svip_row_threshold(svip_ctx* ctx, const void* logits, svip_dtype dtype, int 
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
     return SVIP_OK;
+}
+
+int svip_draft_step_truncated(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, int V, long row_stride,
+                              float T, float thresh, int top_k, float top_p, const float* uniforms,
+                              const uint8_t* active, float* thr, int32_t* token, float* entropy, uint8_t* stop,
+                              float* row_stats, void* stream) {
+    if (!ctx || !logits || !thr || !token || !entropy || !stop || !uniforms) return SVIP_ERR_INVALID_ARG;
+    if (dtype != SVIP_F32 && dtype != SVIP_BF16) return SVIP_ERR_UNSUPPORTED;
+    if (B < 0 || V < 1 || V > 0x7fffffe0 || row_stride < 0 || top_k < 0) return SVIP_ERR_INVALID_ARG;
+    if (!(T > 0.f) || std::isinf(T) || !(top_p > 0.f) || std::isnan(thresh)) return SVIP_ERR_INVALID_ARG;
+    if (!aligned_to(logits, dtype == SVIP_BF16 ? 2 : 4)) return SVIP_ERR_INVALID_ARG;
+    if (row_stats && !aligned_to(row_stats, 8)) return SVIP_ERR_INVALID_ARG;
+    if (B == 0) return SVIP_OK;
+    if (B > ctx->max_rows) return SVIP_ERR_WORKSPACE;
+    ThresholdArgs a;
+    a.logits = logits; a.row_stride = row_stride; a.V = V; a.c = scale_for(T);
+    a.top_k = (top_k >= 1 && top_k < V) ? top_k : 0; a.top_p = top_p; a.thr = thr;
+    a.stats = reinterpret_cast<float2*>(row_stats);
+    a.uniforms = uniforms; a.active = active; a.thresh = thresh; a.token = token; a.entropy = entropy;
+    a.stop = stop; a.need = ctx->need;
+    const int S = pick_cluster(ctx, B, V, dtype);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = dtype == SVIP_BF16
+        ? launch_clustered(row_threshold_kernel<kBF16, true>, B, S, a, st, kRingBytes)
+        : launch_clustered(row_threshold_kernel<kF32, true>, B, S, a, st, kRingBytes);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    // the rows the candidates could not finish: the streaming draft step at the thresholds just found
+    return svip_draft_step_filtered(ctx, logits, dtype, B, V, row_stride, T, thresh, uniforms, ctx->need, thr, token,
+                                    entropy, stop, row_stats, stream);
 }
 
 int svip_pack_ragged(svip_ctx* ctx, const int32_t* draft_len, int B, int K_max, int32_t* cu_rows,

@@ -26,6 +26,7 @@ constexpr int kHistCopies = 8;           // interleaved copies of the histogram:
 constexpr float kMassScale = 1099511627776.0f;   // 2^40
 constexpr int kCandPerBlock = 1024;      // candidate keys a block may collect
 constexpr int kPoolCap = 4096;           // candidate keys of the whole cluster (lives in the histogram copies)
+constexpr int kPoolCapDraft = 2048;      // the same when their indices are kept too (draft form)
 
 struct ThresholdArgs {
     const void* logits;
@@ -36,6 +37,14 @@ struct ThresholdArgs {
     float top_p;    // (0, 1), or >= 1 when off
     float* thr;     // [rows] out: tau as a logit value (-inf: nothing is dropped)
     float2* stats;  // [rows] out or NULL: (largest logit, mass of the kept set relative to it)
+    // draft form (kDraft): the whole truncated draft step where the candidates allow it
+    const float* uniforms;   // [rows]
+    const uint8_t* active;   // NULL, or rows with 0 are skipped
+    float thresh;            // h of the stop test
+    int32_t* token;          // [rows] out
+    float* entropy;          // [rows] out
+    uint8_t* stop;           // [rows] out
+    uint8_t* need;           // [rows] out: 1 where the row still needs the streaming draft step
 };
 
 // Monotone image of a float: a < b  <=>  key(a) < key(b).  NaN counts as -inf.
@@ -92,6 +101,7 @@ struct SelectShared {
     // candidate path (top-k with a small k)
     uint32_t lane_key[kThreads];          // key of the largest logit each thread saw
     uint32_t cand[kCandPerBlock];         // keys of this block's elements >= the lower bound
+    uint32_t cand_idx[kCandPerBlock];     // draft form: their positions in the row
     uint32_t cand_n;                      // how many there are (may exceed the capacity: then the path is left)
     // decision of a pass (written by warp 0)
     int bin;
@@ -329,6 +339,75 @@ __device__ __forceinline__ uint32_t pool_select(SelectShared& sh, const uint32_t
     return prefix;
 }
 
+// The truncated draft step from the candidates alone (block-collective, run by one block): the kept
+// tokens are the candidates with key >= key_t.  Their masses are 2^-40 fixed point, so the
+// normaliser, the entropy sums and the running sums of the inverse CDF are integers and do not
+// depend on the order in which the candidates were collected.  The kept candidates are put in
+// index order (`scratch`, 24 KB of shared memory no longer used for streaming) by counting, for
+// each, the kept candidates before it; the token is the first whose running mass exceeds
+// u * total.  Returns false, having written nothing, for a row without finite mass.
+__device__ __forceinline__ bool draft_from_candidates(SelectShared& sh, const uint32_t* pool, const uint32_t* pool_idx,
+                                                      int total, uint32_t key_t, float row_max, float M, bool finite,
+                                                      const ThresholdArgs& a, int row, void* scratch, int tid) {
+    const int lane = tid & 31, warp = tid >> 5;
+    unsigned long long* wq_sorted = static_cast<unsigned long long*>(scratch);
+    uint32_t* idx_sorted = reinterpret_cast<uint32_t*>(wq_sorted + kPoolCapDraft);
+    unsigned long long zq = 0, nk = 0;
+    long long aq = 0;
+    for (int i = tid; i < total; i += kThreads) {
+        const uint32_t key = pool[i];
+        if (key < key_t) continue;
+        const float arg = fmaxf(__fmaf_rn(key_value(key), a.c, -M), kArgFloor);
+        const float w = ex2_approx(arg);
+        const unsigned long long wq = __float2ull_rz(w * kMassScale);
+        zq += wq;
+        aq += __float2ll_rz(w * arg * kMassScale);
+        nk += 1;
+        const uint32_t mine = pool_idx[i];
+        int before = 0;
+        for (int j = 0; j < total; ++j) before += (pool[j] >= key_t && pool_idx[j] < mine) ? 1 : 0;
+        wq_sorted[before] = wq;
+        idx_sorted[before] = mine;
+    }
+    zq = block_sum_u64(sh, zq, tid);
+    aq = static_cast<long long>(block_sum_u64(sh, static_cast<unsigned long long>(aq), tid));
+    nk = block_sum_u64(sh, nk, tid);
+    if (!finite || zq == 0 || nk == 0) return false;
+    if (warp == 0) {
+        const int n = static_cast<int>(nk);
+        const float u = a.uniforms[row];
+        const unsigned long long target = static_cast<unsigned long long>(static_cast<double>(u) * static_cast<double>(zq));
+        const int per = (n + 31) / 32;
+        const int lo = min(lane * per, n), hi = min(lo + per, n);
+        unsigned long long sum = 0;
+        for (int i = lo; i < hi; ++i) sum += wq_sorted[i];
+        unsigned long long incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned long long up = shfl_up_u64(incl, o);
+            if (lane >= o) incl += up;
+        }
+        unsigned long long cum = incl - sum;
+        int pos = kIntMax;
+        for (int i = lo; i < hi; ++i) {
+            cum += wq_sorted[i];
+            if (cum > target && pos == kIntMax) pos = i;
+        }
+        pos = warp_min_int(pos);
+        if (pos == kIntMax) pos = n - 1;
+        if (lane == 0) {
+            const float Z = static_cast<float>(static_cast<double>(zq) / 1099511627776.0);
+            const float A = static_cast<float>(static_cast<double>(aq) / 1099511627776.0);
+            const float H = fmaxf(kLn2 * (log2f(Z) - A / Z), 0.f);
+            a.token[row] = static_cast<int32_t>(idx_sorted[pos]);
+            a.entropy[row] = H;
+            a.stop[row] = __fsqrt_rn(H) > a.thresh ? 1 : 0;
+            if (a.stats) a.stats[row] = make_float2(row_max, Z);
+        }
+    }
+    return true;
+}
+
 // Top-k (and the nucleus inside it) for a small k, in two passes over the row.  Pass 1 leaves the
 // largest logit of every thread; the k-th largest of these S * 512 values is a lower bound t0 of
 // tau_k (they are k distinct elements of the row).  Pass 2 collects every element >= t0 -- a few more
@@ -336,15 +415,20 @@ __device__ __forceinline__ uint32_t pool_select(SelectShared& sh, const uint32_t
 // nucleus cut then come from these candidates alone, which every block of the cluster holds in
 // full.  Returns false (for the whole cluster alike) when the candidates do not fit; nothing has
 // been written then and the caller takes the radix descent over the full row.
-template <int DT>
+// kDraft also keeps the positions of the candidates and lets block 0 finish the whole draft step from
+// them (`drafted`, meaningful in block 0 only); `scratch` is the streaming ring, free by then.
+template <int DT, bool kDraft>
 __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const RowGeom& g, int S, int rank, int tid,
                                                uint32_t slot0, const ThresholdArgs& a, bool use_p, SelectShared& sh,
-                                               uint32_t& key_out) {
+                                               uint32_t& key_out, void* scratch, bool& drafted) {
     constexpr int EPV = ElemTraits<DT>::kEPV;
     constexpr int kLevels = DT == kBF16 ? 2 : 4;
+    constexpr int kCap = kDraft ? kPoolCapDraft : kPoolCap;
     const int lane = tid & 31, warp = tid >> 5;
     uint32_t* pool = &sh.priv[0][0][0];
+    uint32_t* pool_idx = pool + kPoolCapDraft;
     static_assert(sizeof(sh.priv) >= kPoolCap * sizeof(uint32_t), "the pool lives in the histogram copies");
+    drafted = false;
     // pass 1: the largest logit of every thread (fmaxf skips NaN); threads without elements keep key 0
     float best = neg_inf();
     bool any = false;
@@ -364,12 +448,15 @@ __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const
     // except for NaN, which counts as -inf and so belongs to the candidates only when the bound is that low.
     const float t0v = t0 ? key_value(t0) : neg_inf();
     const bool lowest = !(t0v > neg_inf());
-    stream_segment<DT>(g, rank * kWarps + warp, lane, slot0, [&](const float (&x)[EPV], int) {
+    stream_segment<DT>(g, rank * kWarps + warp, lane, slot0, [&](const float (&x)[EPV], int vi) {
 #pragma unroll
         for (int j = 0; j < EPV; ++j) {
             if (x[j] >= t0v || (lowest && !(x[j] == x[j]))) {
                 const uint32_t pos = atomicAdd(&sh.cand_n, 1u);
-                if (pos < kCandPerBlock) sh.cand[pos] = order_key(x[j]);
+                if (pos < kCandPerBlock) {
+                    sh.cand[pos] = order_key(x[j]);
+                    if (kDraft) sh.cand_idx[pos] = static_cast<uint32_t>(vi * EPV + j - g.pre);
+                }
             }
         }
     });
@@ -381,13 +468,16 @@ __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const
         if (nr > kCandPerBlock) fits = false;
         total += static_cast<int>(min(nr, static_cast<uint32_t>(kCandPerBlock)));
     }
-    if (total > kPoolCap) fits = false;
+    if (total > kCap) fits = false;
     if (fits) {
         int at = 0;
         for (int r = 0; r < S; ++r) {
             const SelectShared* peer = cluster.map_shared_rank(&sh, r);
             const int nr = static_cast<int>(peer->cand_n);
-            for (int i = tid; i < nr; i += kThreads) pool[at + i] = peer->cand[i];
+            for (int i = tid; i < nr; i += kThreads) {
+                pool[at + i] = peer->cand[i];
+                if (kDraft) pool_idx[at + i] = peer->cand_idx[i];
+            }
             at += nr;
         }
     }
@@ -398,7 +488,7 @@ __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const
     float row_max = neg_inf();
     bool finite = false;
     float M = 0.f;
-    if (use_p || a.stats) {
+    if (use_p || a.stats || kDraft) {
         // the largest candidate is the largest logit of the row
         uint32_t top = 0;
         for (int i = tid; i < total; i += kThreads) top = max(top, pool[i]);
@@ -434,10 +524,18 @@ __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const
         if (rank == 0 && tid == 0) a.stats[blockIdx.x / S] = kept_stats(row_max, zt, finite);
     }
     key_out = key_t;
+    if (kDraft && rank == 0) {
+        __syncthreads();   // the pool is complete and the ring is idle in every warp
+        drafted = draft_from_candidates(sh, pool, pool_idx, total, key_t, row_max, M, finite, a,
+                                        static_cast<int>(blockIdx.x / S), scratch, tid);
+    }
     return true;
 }
 
-template <int DT>
+// kDraft: the truncated draft step in the same launch wherever the candidate path applies; the rows
+// it could not finish (nucleus alone, large k, heavy ties, no finite mass) are marked in `need` and
+// left to the streaming kernel, with their threshold already in `thr`.
+template <int DT, bool kDraft = false>
 __global__ void __launch_bounds__(kThreads, 2) row_threshold_kernel(ThresholdArgs a) {
     constexpr int kLevels = DT == kBF16 ? 2 : 4;   // the low 16 bits of a bf16 logit carry nothing
     extern __shared__ uint4 ring[];
@@ -453,6 +551,10 @@ __global__ void __launch_bounds__(kThreads, 2) row_threshold_kernel(ThresholdArg
     const RowGeom g = make_geom<DT>(rp, a.V, S * kWarps);
     const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
     pdl_wait();
+    if (kDraft && a.active && !a.active[row]) {   // the whole cluster leaves together
+        if (rank == 0 && tid == 0) a.need[row] = 0;
+        return;
+    }
 
     const bool use_k = a.top_k >= 1 && a.top_k < a.V;
     const bool use_p = a.top_p < 1.0f;
@@ -464,8 +566,12 @@ __global__ void __launch_bounds__(kThreads, 2) row_threshold_kernel(ThresholdArg
     // a small k against the number of threads of the cluster: two passes and a handful of candidates
     if (use_k && a.top_k <= (S * kThreads) / 4) {
         uint32_t key_t = 0;
-        if (candidate_path<DT>(cluster, g, S, rank, tid, slot0, a, use_p, sh, key_t)) {
-            if (rank == 0 && tid == 0) a.thr[row] = key_t ? key_value(key_t) : neg_inf();
+        bool drafted = false;
+        if (candidate_path<DT, kDraft>(cluster, g, S, rank, tid, slot0, a, use_p, sh, key_t, ring, drafted)) {
+            if (rank == 0 && tid == 0) {
+                a.thr[row] = key_t ? key_value(key_t) : neg_inf();
+                if (kDraft) a.need[row] = drafted ? 0 : 1;
+            }
             return;
         }
     }
@@ -494,7 +600,7 @@ __global__ void __launch_bounds__(kThreads, 2) row_threshold_kernel(ThresholdArg
     }
 
     uint32_t key_t = key_k;
-    if (use_p || a.stats) {
+    if (use_p || (a.stats && !kDraft)) {
         if (!have_max) {
             // the masses are taken relative to the largest logit: find it first
             float mx = neg_inf();
@@ -549,8 +655,11 @@ __global__ void __launch_bounds__(kThreads, 2) row_threshold_kernel(ThresholdArg
         if (above == 0 || !finite) key_p = 0;   // a row without mass: the nucleus drops nothing
         key_t = key_p > key_k ? key_p : key_k;
     }
-    if (rank == 0 && tid == 0) a.thr[row] = key_t ? key_value(key_t) : neg_inf();
-    if (a.stats) {
+    if (rank == 0 && tid == 0) {
+        a.thr[row] = key_t ? key_value(key_t) : neg_inf();
+        if (kDraft) a.need[row] = 1;
+    }
+    if (a.stats && !kDraft) {
         // the mass of the kept set: one more pass (the descents above know it only in part)
         const bool finite = fabsf(row_max) <= kMaxLogit;
         const float M = finite ? __fmul_rn(row_max, a.c) : 0.f;

@@ -54,6 +54,7 @@ def test_null_context_is_invalid_argument(lib):
     assert lib.svip_draft_step_filtered(None, 16, 0, 1, 8, 8, 1.0, 0.3, 16, None, 16, 16, 16, 16, None, None) == -1
     assert lib.svip_verify_filtered(None, 16, 16, 8, None, 16, -1, 0, 16, 8, 16, None, 0, None, 1, 1, 2, 8, 1.0, 16, 16,
                                     16, None) == -1
+    assert lib.svip_draft_step_truncated(None, 16, 0, 1, 8, 8, 1.0, 0.3, 2, 0.9, 16, None, 16, 16, 16, 16, None, None) == -1
     assert lib.svip_graph_loop_end(None) == -1
     body = C.c_void_p()
     assert lib.svip_graph_loop_begin(None, None, 16, 4, C.byref(body)) == -1

@@ -268,3 +268,69 @@ def test_filtered_entry_points_reject_bad_arguments(ctx):
         ctx.verify_filtered(i, x, 64, None, None, -1, 0, x, 64, f, 0, None, 1, 1, 2, 64, 1.0, f, i, i)
     with pytest.raises(SvipError):
         ctx.row_threshold(x, 0, 4, 64, 64, 1.0, 3, 0.9, f, f.data_ptr() + 4)                 # stats must be 8-byte aligned
+
+
+@pytest.mark.parametrize("dtype,V", [("bf16", 32000), ("f32", 50021), ("bf16", 152064), ("f32", 777)])
+@pytest.mark.parametrize("k,p", [(50, 1.0), (50, 0.9), (1, 1.0), (0, 0.9), (3000, 0.9)])
+def test_truncated_draft_step_in_one_call(ctx, oracle, dtype, V, k, p):
+    """svip_draft_step_truncated: thresholds and the truncated draft step together.  With a small k the
+    first kernel finishes rows from its candidates; the other cases (nucleus alone, large k, a row of ties)
+    fall through to the streaming kernel.  Either way the outputs must match the oracle on the kept set
+    that the returned thresholds define, and the thresholds must match the oracle's."""
+    import torch
+    rng = np.random.default_rng(V * 7 + k)
+    B, T, h = 20, 0.8, 0.3
+    x = (rng.standard_normal((B, V)) * rng.uniform(0.3, 5.0, size=(B, 1))).astype(np.float32)
+    x[2, rng.integers(0, V)] += 20.0
+    x[4] = 1.5                                   # one group of ties: the candidates cannot hold it
+    rows = W.to_bf16_bits(x) if dtype == "bf16" else x
+    u = rng.random(B).astype(np.float32)
+    active = np.ones(B, dtype=np.uint8); active[[3, 11]] = 0
+    kk = min(k, V - 1) if k else 0
+    d_rows = tl.to_device(rows)
+    for S in (0, 1, 4, 8):
+        ctx.set_cluster_size(S)
+        try:
+            thr = torch.full((B,), 77.0, device="cuda")
+            tok = torch.full((B,), -7, dtype=torch.int32, device="cuda"); ent = torch.full((B,), -1.0, device="cuda")
+            stop = torch.full((B,), 9, dtype=torch.uint8, device="cuda"); stats = torch.full((B, 2), -2.0, device="cuda")
+            ctx.draft_step_truncated(d_rows, tl.dtype_code(rows), B, V, V, T, h, kk, p, tl.to_device(u),
+                                     tl.to_device(active), thr, tok, ent, stop, stats)
+            torch.cuda.synchronize()
+        finally:
+            ctx.set_cluster_size(0)
+        on = np.nonzero(active)[0]; off = np.nonzero(active == 0)[0]
+        thr_h = thr.cpu().numpy()
+        check(oracle, rows[on], T, kk, p, thr_h[on], "truncated step S=%d" % S)
+        masked = oracle.mask_below(rows[on], thr_h[on].astype(np.float64))
+        got = (tok.cpu().numpy()[on], ent.cpu().numpy()[on], stop.cpu().numpy()[on], None)
+        tl.check_draft_against_oracle(oracle, masked, T, h, u[on], got, "truncated step S=%d k=%d p=%g" % (S, kk, p))
+        vals = values_of(rows)
+        assert np.all(vals[on, got[0]] >= thr_h[on])
+        st = stats.cpu().numpy()
+        for b in on[::4]:
+            keep = vals[b] >= float(thr_h[b])
+            Z = np.exp((vals[b][keep] - vals[b].max()) / T).sum()
+            assert st[b, 0] == np.float32(vals[b].max()) and abs(st[b, 1] - Z) <= 1e-5 * Z
+        # sequences that are not drafting are left alone
+        assert np.all(tok.cpu().numpy()[off] == -7) and np.all(ent.cpu().numpy()[off] == -1.0)
+        assert np.all(stop.cpu().numpy()[off] == 9)
+    assert ctx.read_status() == 0
+
+
+def test_truncated_draft_step_bad_arguments(ctx):
+    import torch
+    from paper_2411_18462_b200 import Context, SvipError
+    x = torch.zeros(4, 64, device="cuda"); f = torch.zeros(8, device="cuda")
+    i = torch.zeros(8, dtype=torch.int32, device="cuda"); b = torch.zeros(8, dtype=torch.uint8, device="cuda")
+    with pytest.raises(SvipError):
+        ctx.draft_step_truncated(x, 0, 4, 64, 64, 0.0, 0.3, 5, 0.9, f, None, f, i, f, b)     # greedy
+    with pytest.raises(SvipError):
+        ctx.draft_step_truncated(x, 0, 4, 64, 64, 1.0, 0.3, 5, 0.9, None, None, f, i, f, b)  # no uniforms
+    small = Context(0, 2)
+    try:
+        with pytest.raises(SvipError):
+            small.draft_step_truncated(x, 0, 4, 64, 64, 1.0, 0.3, 5, 0.9, f, None, f, i, f, b)   # more rows than the workspace
+    finally:
+        small.destroy()
+    ctx.draft_step_truncated(x, 0, 0, 64, 64, 1.0, 0.3, 5, 0.9, f, None, f, i, f, b)         # empty batch
