@@ -368,6 +368,9 @@ int svip_vp_locate(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, i
  * Pair r reads target row r (element r*t_row_stride) and draft row r (element
  * r*q_row_stride).  `out` is DEVICE [n_pairs][8] fp32.  Where the target masks
  * a token (-inf) that the draft gives mass, KL, H_qp and gamma are +inf.
+ * Entropies are fp32 sums, good to about 1e-7 nats: for a draft row that is
+ * one-hot to that resolution H_q comes out as 0 and gamma, a ratio that has no
+ * limit there, as +inf or NaN.
  * Needs n_pairs <= max_rows of svip_create.  Three kernels: the two rows'
  * normalisers, then one pass over both rows.
  */
