@@ -1148,7 +1148,7 @@ const char* svip_strerror(int status) {
     }
 }
 
-int svip_version(void) { return 100; }
+int svip_version(void) { return 200; }
 
 int svip_last_cuda_error(const svip_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
 
