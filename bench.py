@@ -279,25 +279,29 @@ def b1_latency(ctx, torch):
         stop1 = torch.zeros(1, dtype=torch.uint8, device="cuda")
         st.synchronize()
         CONSTANT = 1
-        ctx.graph_begin(st)
-        ctx.policy_update(CONSTANT, None, dlen, gamma, act, 1, K, st)
-        body = ctx.graph_loop_begin(st, nact, K)
-        ctx.draft_step_at(dq, 0, 1, V, V, V, dlen, 1, w.T, w.h, ud, act, tok, ent, stop1, stats, body)
-        ctx.policy_advance(CONSTANT, stop1, gamma, dlen, act, 1, K, nact, body)
-        ctx.graph_loop_end()
-        loop = ctx.graph_end(st)
-        for _ in range(20):
-            loop.launch(st)
-        st.synchronize()
-        assert int(dlen.item()) == K
-        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
-        e0.record(st)
-        for _ in range(200):
-            loop.launch(st)
-        e1.record(st)
-        st.synchronize()
-        out["draft_loop_us_per_token"] = 1000.0 * e0.elapsed_time(e1) / 200 / K
-        loop.destroy()
+        # `unroll` tokens per loop iteration: the loop node costs a few microseconds per iteration, which a
+        # body of several (masked) steps spreads over as many tokens
+        for unroll, key in ((1, "draft_loop_us_per_token"), (4, "draft_loop_unrolled4_us_per_token")):
+            ctx.graph_begin(st)
+            ctx.policy_update(CONSTANT, None, dlen, gamma, act, 1, K, st)
+            body = ctx.graph_loop_begin(st, nact, K)
+            for _ in range(unroll):
+                ctx.draft_step_at(dq, 0, 1, V, V, V, dlen, 1, w.T, w.h, ud, act, tok, ent, stop1, stats, body)
+                ctx.policy_advance(CONSTANT, stop1, gamma, dlen, act, 1, K, nact, body)
+            ctx.graph_loop_end()
+            loop = ctx.graph_end(st)
+            for _ in range(20):
+                loop.launch(st)
+            st.synchronize()
+            assert int(dlen.item()) == K
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record(st)
+            for _ in range(200):
+                loop.launch(st)
+            e1.record(st)
+            st.synchronize()
+            out[key] = 1000.0 * e0.elapsed_time(e1) / 200 / K
+            loop.destroy()
 
         def host_loop():
             ctx.policy_update(CONSTANT, None, dlen, gamma, act, 1, K, st)
