@@ -269,6 +269,12 @@ def b1_latency(ctx, torch):
             e1.record(st)
             st.synchronize()
             out[name] = 1000.0 * e0.elapsed_time(e1) / reps
+            # launch to result visible on the host: one replay, then wait for it, timed on the host clock
+            t0 = time.perf_counter()
+            for _ in range(reps):
+                graph.launch(st)
+                st.synchronize()
+            out[name.replace("_us", "_to_host_us")] = 1e6 * (time.perf_counter() - t0) / reps
         g.destroy(); one.destroy()
 
         # the drafting phase as a loop inside the graph (each token: draft step at the sequence's own
