@@ -17,8 +17,8 @@ CSRC = os.path.join(PKG, "csrc")
 INCLUDE = os.path.join(os.path.dirname(PKG), "include")
 LIB = os.path.join(CSRC, "libsvip.so")
 SOURCES = ["svip.cu"]
-HEADERS = [os.path.join(CSRC, "svip_device.cuh"), os.path.join(CSRC, "svip_select.cuh"),
-           os.path.join(INCLUDE, "svip.h")]
+HEADERS = sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".cuh")) + \
+    [os.path.join(INCLUDE, "svip.h")]
 
 
 def _nvcc() -> str:

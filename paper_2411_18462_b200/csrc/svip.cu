@@ -1,17 +1,16 @@
-// SVIP speculative-decoding epilogues for sm_100a: kernels and the C ABI (see include/svip.h).
+// SVIP speculative-decoding epilogues for sm_100a: the host side and the C ABI (see include/svip.h).
 //
-// Kernels
-//   draft_step_kernel    Algorithm 1 inner loop + Eq. 7: one pass over a logits row gives
-//                        max / mass / entropy term / argmax; the sampled token is then found by
-//                        re-reading one warp segment.  A row is shared by a thread-block
-//                        cluster (1..8 blocks) whose partials meet in distributed shared memory.
-//   row_stats_kernel     softmax normalisers (or argmax, greedy) of target rows, and of draft
-//                        rows when the caller has no q_stats.
-//   verify_finish_kernel Algorithms 2 and 4 + the loop of Algorithm 1: ratio tests by one warp
-//                        (ballot + first set bit = first rejection), then the residual
-//                        max(0, p - q) or the bonus row is sampled by inverse CDF.
-//   verify_greedy_kernel Algorithms 3 and 5 on the per-row argmax.
-//   pack_ragged_kernel   exclusive scan of (K_i + 1) and the row -> (sequence, position) maps.
+// The kernels live in the headers included below:
+//   svip_device.cuh    the streaming core: row geometry, cp.async ring, online reduction, warp / block
+//                      scans, picking the segment that holds a sample
+//   svip_draft.cuh     draft_step_kernel (Algorithm 1 inner loop + Eq. 7) and row_stats_kernel (softmax
+//                      normalisers or argmax of target rows; of draft rows when the caller has no q_stats)
+//   svip_verify.cuh    verify_finish_kernel (Algorithms 2 and 4 + the loop of Algorithm 1: ratio tests by
+//                      one warp, first rejection, residual or bonus token) and verify_greedy_kernel
+//                      (Algorithms 3 and 5)
+//   svip_analysis.cuh  pair_stats_kernel (Eq. 1-6)
+//   svip_policy.cuh    vocabulary-parallel combine, draft-length policies, ragged packing
+//   svip_select.cuh    row_threshold_kernel (top-k / nucleus truncation)
 #include "svip_device.cuh"
 
 #include <cmath>
@@ -22,996 +21,10 @@
 
 #include "svip.h"
 
-namespace svip {
-
-constexpr int kPolicyThreads = 256;
-
-struct SegEntry {
-    float m;
-    int idx;
-    float Z;
-    float A;
-};
-
-// Reads every segment entry of the cluster (warp-collective, run by warp 0 of each block), merges
-// them into the row's partial and selects the segment holding the mass u * Z.
-template <int kMode>
-__device__ __forceinline__ void combine_segments(cg::cluster_group& cluster, SegEntry* seg, int S,
-                                                 float c, float u, int lane, Partial& row,
-                                                 SegPick& pick, float abs_target = -1.f) {
-    const int nseg = S * kWarps;
-    const int per = (nseg + 31) / 32;
-    Partial e[kSegPerLane];
-    float m = neg_inf();
-#pragma unroll
-    for (int k = 0; k < kSegPerLane; ++k) {
-        e[k].m = neg_inf(); e[k].idx = kIntMax; e[k].Z = 0.f; e[k].A = 0.f;
-        int s = lane * per + k;
-        if (k < per && s < nseg) {
-            const SegEntry* remote = cluster.map_shared_rank(seg, s / kWarps);
-            SegEntry v = remote[s % kWarps];
-            e[k].m = v.m; e[k].idx = v.idx; e[k].Z = v.Z; e[k].A = v.A;
-        }
-        m = fmaxf(m, e[k].m);
-    }
-    m = warp_max(m);
-    int idx = kIntMax;
-    float mass[kSegPerLane];
-    float asum = 0.f;
-#pragma unroll
-    for (int k = 0; k < kSegPerLane; ++k) {
-        if (e[k].m == m) idx = min(idx, e[k].idx);
-        rescale_to<kMode>(e[k], m, c);
-        mass[k] = e[k].Z;
-        asum += e[k].A;
-    }
-    row.m = m;
-    row.idx = warp_min_int(idx);
-    row.A = warp_sum(asum);
-    pick = pick_segment(mass, per, nseg, u, lane, abs_target);
-    row.Z = pick.total;
-}
-
-// Fine scan of one segment by the whole block.  `wf(vi, w)` yields the weights of the elements
-// of vector vi.  Each thread sums a run of consecutive vectors, one block scan places the runs,
-// and the thread whose run crosses `target` walks its run again element by element.  Returns the
-// virtual element index (vector * EPV + element) of the first element whose cumulative weight
-// exceeds `target`, else the last element with positive weight, else -1.
-template <int EPV, class WF>
-__device__ __forceinline__ int fine_scan(WF& wf, int v_lo, int v_hi, float prefix, float target,
-                                         ScanShared& sh, int tid, int lane, int warp) {
-    constexpr int kRun = 4;
-    const int nv = v_hi - v_lo;
-    const int run = min(kRun, max(1, (nv + kThreads - 1) / kThreads));
-    if (tid == 0) { sh.hit = kIntMax; sh.lastpos = -1; sh.result = -1; }
-    float running = prefix;
-    for (int cb = v_lo; cb < v_hi; cb += kThreads * run) {
-        const int first = cb + tid * run;
-        float ls = 0.f;
-        int lastv = -1;
-        for (int k = 0; k < run; ++k) {
-            int vi = first + k;
-            if (vi < v_hi) {
-                float w[EPV];
-                wf(vi, w);
-                float sv = 0.f;
-#pragma unroll
-                for (int j = 0; j < EPV; ++j) sv += w[j];
-                if (sv > 0.f) lastv = vi;
-                ls += sv;
-            }
-        }
-        float total;
-        const float lo = running + block_scan_excl(ls, sh.wsum, lane, warp, total);
-        if (ls > 0.f && lo + ls > target) atomicMin(&sh.hit, tid);
-        if (lastv >= 0) atomicMax(&sh.lastpos, lastv);
-        __syncthreads();
-        const int win = sh.hit;
-        if (win != kIntMax) {
-            if (tid == win) {
-                float cum = lo;
-                int res = -1, last = -1;
-                for (int k = 0; k < run; ++k) {
-                    int vi = first + k;
-                    if (vi < v_hi) {
-                        float w[EPV];
-                        wf(vi, w);
-#pragma unroll
-                        for (int j = 0; j < EPV; ++j) {
-                            cum += w[j];
-                            if (w[j] > 0.f) {
-                                last = vi * EPV + j;
-                                if (cum > target && res < 0) res = last;
-                            }
-                        }
-                    }
-                }
-                sh.result = res >= 0 ? res : last;
-            }
-            __syncthreads();
-            return sh.result;
-        }
-        running += total;
-    }
-    // rounding left nothing above the target: the last element with weight
-    const int lv = sh.lastpos;
-    if (lv < 0) return -1;
-    if (tid == 0) {
-        float w[EPV];
-        wf(lv, w);
-        int last = -1;
-#pragma unroll
-        for (int j = 0; j < EPV; ++j)
-            if (w[j] > 0.f) last = lv * EPV + j;
-        sh.result = last;
-    }
-    __syncthreads();
-    return sh.result;
-}
-
-// ------------------------------------------------------------------ draft step
-
-struct DraftArgs {
-    const void* logits;
-    long row_stride;
-    int V;
-    float c;          // log2(e) / T   (T = 1 when greedy)
-    float thresh;
-    int greedy;
-    const float* uniforms;
-    int32_t* token;
-    float* entropy;
-    uint8_t* stop;
-    float* row_stats;
-    unsigned* status;
-    const uint8_t* active;   // NULL, or one flag per row: rows with 0 are skipped
-    const float* ext_target; // NULL, or per row the mass to find (units of this row's own Z), see svip_vp_locate
-    int token_offset;        // added to the sampled index (vocabulary shard offset)
-    const int32_t* pos;      // NULL, or per row the draft position p whose logits are read (svip_draft_step_at)
-    long pos_stride;         // elements between the logits of consecutive positions of a row
-    long slot_stride;        // uniforms / token / entropy / row_stats live at index p * slot_stride + row
-    const float* thr;        // NULL, or per row the truncation threshold: only logits >= thr[row] count
-};
-
-template <int DT>
-struct SoftmaxWeights {
-    RowGeom g;
-    float c, M;
-    float thr = -INFINITY;   // logits below it carry no weight (truncated distributions)
-    __device__ __forceinline__ void operator()(int vi, float (&w)[ElemTraits<DT>::kEPV]) const {
-        constexpr int EPV = ElemTraits<DT>::kEPV;
-        float x[EPV];
-        unpack_masked<DT>(g.base[vi], vi, g, x);
-#pragma unroll
-        for (int j = 0; j < EPV; ++j)
-            w[j] = x[j] >= thr ? ex2_approx(fmaxf(__fmaf_rn(x[j], c, -M), kArgFloor)) : 0.f;
-    }
-};
-
-struct RowShared {
-    Partial row;
-    SegPick pick;
-};
-
-// kBlocks is the number of blocks the register budget must leave room for on one SM: 2 for
-// launches that fit the GPU in one wave (latency matters, registers are free), 3 for launches of
-// many waves, where a third resident block streams on while another one is in its epilogue.
-// kPos compiles the position-indexed form (svip_draft_step_at) in, kThr the truncated form
-// (svip_draft_step_filtered).
-template <int DT, bool kGreedy, int kBlocks, bool kPos = false, bool kThr = false>
-__global__ void __launch_bounds__(kThreads, kBlocks) draft_step_kernel(DraftArgs a) {
-    constexpr int EPV = ElemTraits<DT>::kEPV;
-    extern __shared__ uint4 ring[];
-    cg::cluster_group cluster = cg::this_cluster();
-    const int S = cluster.dim_blocks().x;
-    const int rank = cluster.block_rank();
-    const int row = blockIdx.x / S;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    __shared__ SegEntry seg[kWarps];
-    __shared__ ScanShared scan;
-    __shared__ RowShared res;
-
-    pdl_launch_dependents();
-    const char* rp = static_cast<const char*>(a.logits) +
-                     static_cast<size_t>(row) * a.row_stride * ElemTraits<DT>::kBytes;
-    RowGeom g = make_geom<DT>(rp, a.V, S * kWarps);
-    const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
-    pdl_wait();
-    if (a.active && !a.active[row]) return;   // the whole cluster leaves together
-    long p = 0;
-    if (kPos) {
-        p = a.pos[row];
-        rp += p * a.pos_stride * ElemTraits<DT>::kBytes;
-        g = make_geom<DT>(rp, a.V, S * kWarps);
-    }
-    float u = 0.f, ext = -1.f;
-    if (!kGreedy && warp == 0) {   // fetched now, used after the stream
-        if (a.ext_target) ext = fmaxf(__ldg(a.ext_target + row), 0.f);
-        else u = __ldg(a.uniforms + (row + p * a.slot_stride));
-    }
-    const float thr = kThr ? a.thr[row] : neg_inf();
-    Partial t = reduce_segment<DT, 2, kGreedy, kThr>(g, rank * kWarps + warp, a.c, lane, slot0, thr);
-    if (lane == 0) { seg[warp].m = t.m; seg[warp].idx = t.idx; seg[warp].Z = t.Z; seg[warp].A = t.A; }
-    cluster.sync();
-    if (warp == 0) {
-        Partial r; SegPick p;
-        combine_segments<2>(cluster, seg, S, a.c, u, lane, r, p, ext);
-        if (lane == 0) { res.row = r; res.pick = p; }
-    }
-    cluster_arrive();   // done with the peers' shared memory
-    __syncthreads();    // res is visible block-wide
-    const Partial R = res.row;
-    const SegPick P = res.pick;
-    const bool ok = (R.Z > 0.f) && (fabsf(R.m) <= kMaxLogit);
-    // where this row's outputs live (the position is read again rather than kept across the stream)
-    long slot = row;
-    if (kPos && tid == 0) slot += a.pos[row] * a.slot_stride;
-    if (rank == 0 && tid == 0) {
-        float H = 0.f;
-        if (ok) H = fmaxf(kLn2 * (log2f(R.Z) - R.A / R.Z), 0.f);
-        else atomicOr(a.status, SVIP_STATUS_NONFINITE_ROW);
-        if (a.entropy) a.entropy[slot] = H;
-        if (a.stop) a.stop[row] = __fsqrt_rn(H) > a.thresh ? 1 : 0;
-        if (a.row_stats) { a.row_stats[2 * slot] = R.m; a.row_stats[2 * slot + 1] = R.Z; }
-        if (kGreedy || !ok) a.token[slot] = ((R.idx >= 0 && R.idx < a.V) ? R.idx : 0) + a.token_offset;
-    }
-    if (!kGreedy && ok && P.seg / kWarps == rank) {
-        SoftmaxWeights<DT> wf;
-        wf.g = g; wf.c = a.c; wf.M = __fmul_rn(R.m, a.c); wf.thr = thr;
-        int v_lo, v_hi;
-        seg_range(g, P.seg, v_lo, v_hi);
-        int virt = fine_scan<EPV>(wf, v_lo, v_hi, P.prefix, P.target, scan, tid, lane, warp);
-        if (tid == 0) a.token[slot] = (virt >= 0 ? virt - g.pre : 0) + a.token_offset;
-    }
-    cluster_wait();     // no block leaves while a peer may still read its shared memory
-}
-
-// ------------------------------------------------------------------ row statistics (verify, phase 1)
-
-struct StatsArgs {
-    const void* logits;
-    long row_stride;
-    int V;
-    float c;
-    int draft_rows;          // 0: unit = row.  1: unit = (sequence, position) of a draft row
-    int K;
-    const int32_t* cu;
-    long q_seq_stride, q_pos_stride;
-    float2* out_stats;       // (m, Z) per row, indexed by target-row number
-    int32_t* out_argmax;
-    unsigned* status;
-    float4* out_partial;     // kMode 2: (m, Z, A, index of the maximum + idx_offset as int bits)
-    int idx_offset;
-    const float* thr;        // kThr: truncation threshold per row (target rows: by target row; draft rows: by draft row)
-};
-
-template <int DT, int kMode, bool kThr = false>
-__global__ void __launch_bounds__(kThreads) row_stats_kernel(StatsArgs a) {
-    cg::cluster_group cluster = cg::this_cluster();
-    const int S = cluster.dim_blocks().x;
-    const int rank = cluster.block_rank();
-    const int unit = blockIdx.x / S;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    __shared__ SegEntry seg[kWarps];
-    extern __shared__ uint4 ring[];
-
-    pdl_launch_dependents();
-    pdl_wait();
-    long in_row = unit;
-    int out_row = unit;
-    if (a.draft_rows) {
-        int i = unit / a.K, j = unit - i * a.K;
-        int row0 = a.cu ? a.cu[i] : i * (a.K + 1);
-        int Ki = a.cu ? a.cu[i + 1] - row0 - 1 : a.K;
-        if (j >= Ki) return;   // the whole cluster leaves together
-        in_row = a.q_seq_stride < 0 ? static_cast<long>(row0 - i + j)
-                                    : i * a.q_seq_stride + j * a.q_pos_stride;
-        out_row = row0 + j;
-    }
-    const char* rp = static_cast<const char*>(a.logits) +
-                     static_cast<size_t>(in_row) * a.row_stride * ElemTraits<DT>::kBytes;
-    const RowGeom g = make_geom<DT>(rp, a.V, S * kWarps);
-    const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
-    const float thr = kThr ? a.thr[in_row] : neg_inf();
-    Partial t = reduce_segment<DT, kMode, kMode != 1, kThr>(g, rank * kWarps + warp, a.c, lane, slot0, thr);
-    if (lane == 0) { seg[warp].m = t.m; seg[warp].idx = t.idx; seg[warp].Z = t.Z; seg[warp].A = t.A; }
-    cluster.sync();
-    if (rank == 0 && warp == 0) {
-        Partial r; SegPick p;
-        combine_segments<kMode>(cluster, seg, S, a.c, 0.f, lane, r, p);
-        if (lane == 0) {
-            bool ok = fabsf(r.m) <= kMaxLogit && (kMode == 0 || r.Z > 0.f);
-            if (!ok && kMode != 2) atomicOr(a.status, SVIP_STATUS_NONFINITE_ROW);   // a shard may be all masked
-            if (kMode == 1) a.out_stats[out_row] = make_float2(r.m, r.Z);
-            if (kMode == 2) {
-                int gi = ((r.idx >= 0 && r.idx < a.V) ? r.idx : 0) + a.idx_offset;
-                a.out_partial[out_row] = make_float4(r.m, ok ? r.Z : 0.f, ok ? r.A : 0.f, __int_as_float(gi));
-            }
-            if (a.out_argmax) a.out_argmax[out_row] = (r.idx >= 0 && r.idx < a.V) ? r.idx : 0;
-        }
-    }
-    cluster.sync();
-}
-
-// ------------------------------------------------------------------ verify, phase 2 (sampling)
-
-struct FinishArgs {
-    const int32_t* draft_tokens;
-    const void* q_logits;
-    long q_row_stride;
-    const float2* q_stats_user;   // indexed by draft row, or NULL
-    const float2* q_stats_ws;     // indexed by target row (used when q_stats_user is NULL)
-    long q_seq_stride, q_pos_stride;
-    const void* t_logits;
-    long t_row_stride;
-    const float2* p_stats;        // indexed by target row
-    const int32_t* cu;
-    int K, V;
-    float c;
-    const float* uniforms;
-    int32_t* n_accepted;
-    int32_t* next_token;
-    unsigned* status;
-    const float* p_thr;           // kThr: truncation threshold of every target row
-    const float* q_thr;           // kThr: ... of every draft row (indexed like the draft tokens)
-};
-
-// Weights max(0, p - q) of Algorithm 4 (or p alone for the bonus token) for one vector.
-template <int DT>
-struct ResidualWeights {
-    RowGeom gt, gq;
-    const void* qrow;
-    float c, Mp, rZp, Mq, rZq;
-    int bonus;
-    float thr_p = -INFINITY, thr_q = -INFINITY;   // truncated distributions: logits below carry nothing
-    __device__ __forceinline__ void operator()(int vi, float (&w)[ElemTraits<DT>::kEPV]) const {
-        constexpr int EPV = ElemTraits<DT>::kEPV;
-        float x[EPV];
-        unpack_masked<DT>(__ldg(gt.base + vi), vi, gt, x);
-#pragma unroll
-        for (int j = 0; j < EPV; ++j)
-            w[j] = x[j] >= thr_p ? ex2_approx(fmaxf(__fmaf_rn(x[j], c, -Mp), kArgFloor)) * rZp : 0.f;
-        if (bonus) return;
-        float d[EPV];
-        if (gq.pre == gt.pre) {
-            unpack_masked<DT>(__ldg(gq.base + vi), vi, gq, d);
-        } else {
-            // rows with different 16-byte phase: element loads
-#pragma unroll
-            for (int j = 0; j < EPV; ++j) {
-                int i = vi * EPV + j - gt.pre;
-                d[j] = (i >= 0 && i < gt.V) ? ElemTraits<DT>::load_one(qrow, i) : neg_inf();
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < EPV; ++j) {
-            float q = d[j] >= thr_q ? ex2_approx(fmaxf(__fmaf_rn(d[j], c, -Mq), kArgFloor)) * rZq : 0.f;
-            w[j] = fmaxf(w[j] - q, 0.f);
-        }
-    }
-};
-
-// Sum of the residual (or bonus) weights over one warp segment, streamed through the cp.async ring:
-// four stages for the target row and four for the draft row.  Same arithmetic as
-// ResidualWeights::weights (packed), without its masking: vectors that stick out of the row, and
-// rows whose draft row has another 16-byte phase, go through the functor instead.
-template <int DT, bool kThr>
-__device__ __forceinline__ float residual_segment_sum(const ResidualWeights<DT>& wf, int seg, int lane,
-                                                      uint32_t slot0) {
-    constexpr int EPV = ElemTraits<DT>::kEPV;
-    constexpr uint32_t kSlotStride = kThreads * 16;
-    constexpr int kDepth = kStages / 2;
-    const RowGeom& g = wf.gt;
-    int v_lo, v_hi;
-    seg_range(g, seg, v_lo, v_hi);
-    float acc = 0.f;
-    if (!wf.bonus && wf.gq.pre != g.pre) {
-        for (int vi = v_lo + lane; vi < v_hi; vi += 32) {
-            float w[EPV];
-            wf(vi, w);
-#pragma unroll
-            for (int j = 0; j < EPV; ++j) acc += w[j];
-        }
-        return acc;
-    }
-    const bool head_edge = g.pre > 0;
-    const bool tail_edge = ((g.pre + g.V) % EPV) != 0;
-    int i_lo = v_lo, i_hi = v_hi;
-    if (head_edge && v_lo == 0 && v_hi > 0) i_lo = 1;
-    if (tail_edge && v_hi == g.nvec && i_hi > i_lo) i_hi = g.nvec - 1;
-    const int vi0 = i_lo + lane;
-    const int n = i_hi > vi0 ? (i_hi - vi0 + 31) >> 5 : 0;
-    const uint4* st = g.base + vi0;
-    const uint4* sq = wf.gq.base + vi0;
-    const bool two = !wf.bonus;
-#pragma unroll
-    for (int s = 0; s < kDepth; ++s) {
-        if (s < n) {
-            cp_async16(slot0 + s * kSlotStride, st + 32 * s);
-            if (two) cp_async16(slot0 + (kDepth + s) * kSlotStride, sq + 32 * s);
-        }
-        cp_async_commit();
-    }
-    const f32x2 c2 = pack2(wf.c, wf.c);
-    const f32x2 nmp2 = pack2(-wf.Mp, -wf.Mp), nmq2 = pack2(-wf.Mq, -wf.Mq);
-    const f32x2 rzp2 = pack2(wf.rZp, wf.rZp), rzq2 = pack2(wf.rZq, wf.rZq);
-    float acc1 = 0.f;
-    for (int it = 0; it < n; ++it) {
-        cp_async_wait<kDepth - 1>();
-        const uint32_t sa = slot0 + (it & (kDepth - 1)) * kSlotStride;
-        const uint4 rt = lds128(sa);
-        uint4 rq = make_uint4(0, 0, 0, 0);
-        if (two) rq = lds128(sa + kDepth * kSlotStride);
-        const int nx = it + kDepth;
-        if (nx < n) {
-            cp_async16(sa, st + 32 * nx);
-            if (two) cp_async16(sa + kDepth * kSlotStride, sq + 32 * nx);
-        }
-        cp_async_commit();
-        float x[EPV], d[EPV];
-        ElemTraits<DT>::unpack(rt, x);
-        ElemTraits<DT>::unpack(rq, d);
-        if (kThr) {
-            drop_below<EPV>(x, wf.thr_p);
-            drop_below<EPV>(d, wf.thr_q);
-        }
-#pragma unroll
-        for (int j = 0; j < EPV; j += 2) {
-            float a0, a1;
-            unpack2(fma2(pack2(x[j], x[j + 1]), c2, nmp2), a0, a1);
-            f32x2 p2 = mul2(pack2(ex2_approx(a0), ex2_approx(a1)), rzp2);
-            float p0, p1;
-            unpack2(p2, p0, p1);
-            if (two) {
-                unpack2(fma2(pack2(d[j], d[j + 1]), c2, nmq2), a0, a1);
-                f32x2 q2 = mul2(pack2(ex2_approx(a0), ex2_approx(a1)), rzq2);
-                float q0, q1;
-                unpack2(q2, q0, q1);
-                p0 = fmaxf(p0 - q0, 0.f);
-                p1 = fmaxf(p1 - q1, 0.f);
-            }
-            acc += p0;
-            acc1 += p1;
-        }
-    }
-    cp_async_wait<0>();
-    acc += acc1;
-    if (lane == 0) {
-        float w[EPV];
-        if (head_edge && v_lo == 0 && v_hi > 0) {
-            wf(0, w);
-#pragma unroll
-            for (int j = 0; j < EPV; ++j) acc += w[j];
-        }
-        if (tail_edge && v_hi == g.nvec && v_lo < v_hi && !(g.nvec == 1 && head_edge)) {
-            wf(g.nvec - 1, w);
-#pragma unroll
-            for (int j = 0; j < EPV; ++j) acc += w[j];
-        }
-    }
-    // NaN weights (NaN logits) count as zero in the functor; here they would poison the sum
-    if (!(acc == acc)) {
-        acc = 0.f;
-        for (int vi = v_lo + lane; vi < v_hi; vi += 32) {
-            float w[EPV];
-            wf(vi, w);
-#pragma unroll
-            for (int j = 0; j < EPV; ++j) acc += w[j];
-        }
-    }
-    return acc;
-}
-
-struct FinishShared {
-    int n_acc;
-    SegPick pick;
-};
-
-template <int DT, bool kThr = false>
-__global__ void __launch_bounds__(kThreads, 2) verify_finish_kernel(FinishArgs a) {
-    using E = ElemTraits<DT>;
-    constexpr int EPV = E::kEPV;
-    cg::cluster_group cluster = cg::this_cluster();
-    const int S = cluster.dim_blocks().x;
-    const int rank = cluster.block_rank();
-    const int i = blockIdx.x / S;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    __shared__ SegEntry seg[kWarps];
-    __shared__ ScanShared scan;
-    __shared__ FinishShared fs;
-    extern __shared__ uint4 ring[];
-    const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
-
-    pdl_launch_dependents();
-    pdl_wait();
-    const int row0 = a.cu ? a.cu[i] : i * (a.K + 1);
-    const int Ki = a.cu ? a.cu[i + 1] - row0 - 1 : a.K;
-    const long dbase = a.q_seq_stride < 0 ? static_cast<long>(row0 - i) : i * a.q_seq_stride;
-    const long dstep = a.q_seq_stride < 0 ? 1 : a.q_pos_stride;
-    const char* tl = static_cast<const char*>(a.t_logits);
-    const char* ql = static_cast<const char*>(a.q_logits);
-
-    // Algorithm 2 at every position at once; the first rejection is the lowest set bit.
-    if (warp == 0) {
-        int n_acc = Ki;
-        for (int j0 = 0; j0 < Ki; j0 += 32) {
-            int j = j0 + lane;
-            bool rej = false;
-            if (j < Ki) {
-                long dr = dbase + j * dstep;
-                int x = a.draft_tokens[dr];
-                bool acc = false;
-                if (x >= 0 && x < a.V) {
-                    float tv = E::load_one(tl + static_cast<size_t>(row0 + j) * a.t_row_stride * E::kBytes, x);
-                    float dv = E::load_one(ql + static_cast<size_t>(dr) * a.q_row_stride * E::kBytes, x);
-                    float2 ps = a.p_stats[row0 + j];
-                    float2 qs = a.q_stats_user ? a.q_stats_user[dr] : a.q_stats_ws[row0 + j];
-                    // p(x)/q(x) = 2^(ap - aq) * Zq / Zp, from the difference of the two log2 arguments, so
-                    // that a token however unlikely under both models keeps its ratio (no underflow)
-                    const float ap = __fmaf_rn(tv, a.c, -__fmul_rn(ps.x, a.c));
-                    const float aq = __fmaf_rn(dv, a.c, -__fmul_rn(qs.x, a.c));
-                    bool p_zero = !(tv > neg_inf()), q_zero = !(dv > neg_inf());   // NaN counts as -inf
-                    if (kThr) {   // tokens that the truncation dropped have probability zero
-                        p_zero = p_zero || !(tv >= a.p_thr[row0 + j]);
-                        q_zero = q_zero || !(dv >= a.q_thr[dr]);
-                    }
-                    // r < min(1, ratio) without the division: a ratio >= 1 accepts every r in [0,1);
-                    // p(x) == 0 accepts none; q(x) == 0 < p(x) is a ratio of +inf
-                    const float r = a.uniforms[row0 + j];
-                    const float d = fminf(fmaxf(ap - aq, -126.f), 126.f);
-                    const float num = __fmul_rn(exp2f(d), qs.y);
-                    acc = !p_zero && (q_zero || num >= ps.y || __fmul_rn(r, ps.y) < num);
-                }
-                rej = !acc;
-            }
-            unsigned mask = __ballot_sync(0xffffffffu, rej);
-            if (mask) { n_acc = j0 + __ffs(mask) - 1; break; }
-        }
-        if (lane == 0) fs.n_acc = n_acc;
-    }
-    __syncthreads();
-    const int n_acc = fs.n_acc;
-    const float u = a.uniforms[row0 + Ki];
-
-    ResidualWeights<DT> wf;
-    const char* trow = tl + static_cast<size_t>(row0 + n_acc) * a.t_row_stride * E::kBytes;
-    wf.gt = make_geom<DT>(trow, a.V, S * kWarps);
-    wf.c = a.c;
-    {
-        float2 ps = a.p_stats[row0 + n_acc];
-        wf.Mp = __fmul_rn(ps.x, a.c);
-        wf.rZp = 1.0f / ps.y;
-        if (kThr) wf.thr_p = a.p_thr[row0 + n_acc];
-    }
-    wf.bonus = n_acc >= Ki;
-    wf.qrow = nullptr; wf.gq = wf.gt; wf.Mq = 0.f; wf.rZq = 0.f;
-    if (!wf.bonus) {
-        long dr = dbase + n_acc * dstep;
-        wf.qrow = ql + static_cast<size_t>(dr) * a.q_row_stride * E::kBytes;
-        wf.gq = make_geom<DT>(wf.qrow, a.V, S * kWarps);
-        float2 qs = a.q_stats_user ? a.q_stats_user[dr] : a.q_stats_ws[row0 + n_acc];
-        wf.Mq = __fmul_rn(qs.x, a.c);
-        wf.rZq = 1.0f / qs.y;
-        if (kThr) wf.thr_q = a.q_thr[dr];
-    }
-
-    int token = -1;
-    for (int pass = 0; pass < 2; ++pass) {
-        // mass of this warp's segment
-        int v_lo, v_hi;
-        float acc = residual_segment_sum<DT, kThr>(wf, rank * kWarps + warp, lane, slot0);
-        acc = warp_sum(acc);
-        if (lane == 0) { seg[warp].m = 0.f; seg[warp].idx = 0; seg[warp].Z = acc; seg[warp].A = 0.f; }
-        cluster.sync();
-        if (warp == 0) {
-            const int nseg = S * kWarps;
-            const int per = (nseg + 31) / 32;
-            float mass[kSegPerLane];
-#pragma unroll
-            for (int k = 0; k < kSegPerLane; ++k) {
-                int s = lane * per + k;
-                mass[k] = 0.f;
-                if (k < per && s < nseg) mass[k] = cluster.map_shared_rank(seg, s / kWarps)[s % kWarps].Z;
-            }
-            SegPick p = pick_segment(mass, per, nseg, u, lane);
-            if (lane == 0) fs.pick = p;
-        }
-        cluster.sync();
-        const SegPick P = fs.pick;
-        if (P.total > 0.f) {
-            if (P.seg / kWarps == rank) {
-                seg_range(wf.gt, P.seg, v_lo, v_hi);
-                int virt = fine_scan<EPV>(wf, v_lo, v_hi, P.prefix, P.target, scan, tid, lane, warp);
-                token = virt >= 0 ? virt - wf.gt.pre : 0;
-            }
-            break;
-        }
-        // No residual mass (p == q wherever it matters): fall back to sampling from p.
-        if (wf.bonus) {
-            if (rank == 0 && tid == 0) atomicOr(a.status, SVIP_STATUS_NONFINITE_ROW);
-            if (rank == 0) token = 0;
-            break;
-        }
-        wf.bonus = 1;
-    }
-    if (tid == 0) {
-        if (rank == 0) a.n_accepted[i] = n_acc;
-        if (token >= 0) a.next_token[i] = token;
-    }
-}
-
-// ------------------------------------------------------------------ analysis quantities of a row pair
-//
-// Eq. 1-6 and appendix B: for p = softmax(target row / T) and q = softmax(draft row / T), with the
-// normalisers already known, one pass over both rows accumulates
-//   beta = sum min(p, q),   sum q * log2 q,   sum q * (log2 q - log2 p)
-// from which H_q, KL(q||p), the cross entropy H_qp = H_q + KL, gamma = H_qp / H_q and the three lower
-// bounds on beta follow.  KL is accumulated directly (not as a difference of two entropies) so that
-// it keeps its relative precision when p is close to q.
-
-struct PairArgs {
-    const void* t_logits;
-    long t_row_stride;
-    const void* q_logits;
-    long q_row_stride;
-    const float2* p_stats;
-    const float2* q_stats;
-    int V;
-    float c;
-    float c_bound;
-    float* out;   // [pairs][8]
-    unsigned* status;
-};
-
-struct PairSums {
-    float beta, qlq, kl;
-};
-
-template <int DT>
-__global__ void __launch_bounds__(kThreads) pair_stats_kernel(PairArgs a) {
-    using E = ElemTraits<DT>;
-    constexpr int EPV = E::kEPV;
-    cg::cluster_group cluster = cg::this_cluster();
-    const int S = cluster.dim_blocks().x;
-    const int rank = cluster.block_rank();
-    const int r = blockIdx.x / S;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    __shared__ PairSums part[kWarps];
-
-    pdl_launch_dependents();
-    const char* trow = static_cast<const char*>(a.t_logits) + static_cast<size_t>(r) * a.t_row_stride * E::kBytes;
-    const char* qrow = static_cast<const char*>(a.q_logits) + static_cast<size_t>(r) * a.q_row_stride * E::kBytes;
-    const RowGeom gt = make_geom<DT>(trow, a.V, S * kWarps);
-    const RowGeom gq = make_geom<DT>(qrow, a.V, S * kWarps);
-    pdl_wait();
-    const float2 ps = a.p_stats[r], qs = a.q_stats[r];
-    const float Mp = __fmul_rn(ps.x, a.c), Mq = __fmul_rn(qs.x, a.c);
-    const float Lp = log2f(ps.y), Lq = log2f(qs.y);
-    const float rZp = 1.0f / ps.y, rZq = 1.0f / qs.y;
-    int v_lo, v_hi;
-    seg_range(gt, rank * kWarps + warp, v_lo, v_hi);
-    float beta = 0.f, qlq = 0.f, kl = 0.f;
-#pragma unroll 2
-    for (int vi = v_lo + lane; vi < v_hi; vi += 32) {
-        float x[EPV], d[EPV];
-        unpack_masked<DT>(__ldg(gt.base + vi), vi, gt, x);
-        if (gq.pre == gt.pre) {
-            unpack_masked<DT>(__ldg(gq.base + vi), vi, gq, d);
-        } else {
-#pragma unroll
-            for (int j = 0; j < EPV; ++j) {
-                int i = vi * EPV + j - gt.pre;
-                d[j] = (i >= 0 && i < gt.V) ? E::load_one(qrow, i) : neg_inf();
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < EPV; ++j) {
-            float ap = __fmaf_rn(x[j], a.c, -Mp);      // log2 of the unnormalised p
-            float aq = __fmaf_rn(d[j], a.c, -Mq);
-            if (!(ap == ap)) ap = neg_inf();            // NaN logits count as masked
-            float p = ex2_approx(fmaxf(ap, kArgFloor)) * rZp;
-            float q = ex2_approx(fmaxf(aq, kArgFloor)) * rZq;   // NaN -> floor -> 0
-            beta += fminf(p, q);
-            if (q > 0.f) {
-                float lq = aq - Lq;
-                qlq = __fmaf_rn(q, lq, qlq);
-                kl = __fmaf_rn(q, lq - (ap - Lp), kl);   // +inf where p is masked but q is not
-            }
-        }
-    }
-    beta = warp_sum(beta); qlq = warp_sum(qlq); kl = warp_sum(kl);
-    if (lane == 0) { part[warp].beta = beta; part[warp].qlq = qlq; part[warp].kl = kl; }
-    cluster.sync();
-    if (rank == 0 && warp == 0) {
-        const int nseg = S * kWarps;
-        float b = 0.f, s1 = 0.f, s3 = 0.f;
-        for (int s = lane; s < nseg; s += 32) {
-            const PairSums v = cluster.map_shared_rank(part, s / kWarps)[s % kWarps];
-            b += v.beta; s1 += v.qlq; s3 += v.kl;
-        }
-        b = warp_sum(b); s1 = warp_sum(s1); s3 = warp_sum(s3);
-        if (lane == 0) {
-            const bool ok = ps.y > 0.f && qs.y > 0.f && fabsf(ps.x) <= kMaxLogit && fabsf(qs.x) <= kMaxLogit;
-            if (!ok) atomicOr(a.status, SVIP_STATUS_NONFINITE_ROW);
-            const float Hq = fmaxf(-kLn2 * s1, 0.f);
-            const float KL = fmaxf(kLn2 * s3, 0.f);
-            const float Hqp = Hq + KL;
-            float* o = a.out + static_cast<size_t>(r) * 8;
-            o[0] = b;
-            o[1] = Hq;
-            o[2] = Hqp;
-            o[3] = KL;
-            o[4] = Hqp / Hq;
-            o[5] = 1.0f - sqrtf(0.5f * KL);
-            o[6] = 1.0f - sqrtf(-expm1f(-KL));
-            o[7] = 1.0f - sqrtf(a.c_bound * Hq);
-        }
-    }
-    cluster.sync();
-}
-
-// ------------------------------------------------------------------ verify, phase 2 (greedy)
-
-struct GreedyArgs {
-    const int32_t* draft_tokens;
-    const int32_t* p_argmax;
-    const int32_t* cu;
-    long q_seq_stride, q_pos_stride;
-    int B, K;
-    int32_t* n_accepted;
-    int32_t* next_token;
-};
-
-__global__ void __launch_bounds__(kThreads) verify_greedy_kernel(GreedyArgs a) {
-    pdl_launch_dependents();
-    pdl_wait();
-    const int lane = threadIdx.x & 31;
-    const int i = blockIdx.x * kWarps + (threadIdx.x >> 5);
-    if (i >= a.B) return;
-    const int row0 = a.cu ? a.cu[i] : i * (a.K + 1);
-    const int Ki = a.cu ? a.cu[i + 1] - row0 - 1 : a.K;
-    const long dbase = a.q_seq_stride < 0 ? static_cast<long>(row0 - i) : i * a.q_seq_stride;
-    const long dstep = a.q_seq_stride < 0 ? 1 : a.q_pos_stride;
-    int n_acc = Ki;
-    for (int j0 = 0; j0 < Ki; j0 += 32) {
-        int j = j0 + lane;
-        bool rej = false;
-        if (j < Ki) rej = a.draft_tokens[dbase + j * dstep] != a.p_argmax[row0 + j];
-        unsigned mask = __ballot_sync(0xffffffffu, rej);
-        if (mask) { n_acc = j0 + __ffs(mask) - 1; break; }
-    }
-    if (lane == 0) {
-        a.n_accepted[i] = n_acc;
-        a.next_token[i] = a.p_argmax[row0 + n_acc];
-    }
-}
-
-// ------------------------------------------------------------------ vocabulary-parallel draft step
-//
-// The vocabulary is sharded over G ranks (a tensor-parallel LM head).  Each rank reduces its shard of
-// every row to (m, Z, A, argmax); the ranks exchange these 16 bytes per row; then every rank combines
-// them in rank order -- same inputs, same arithmetic, so all ranks agree bit for bit on the entropy,
-// the stop flag, and on which rank's shard holds the sampled token and how far into its mass.
-
-struct VpCombineArgs {
-    const float4* partials;   // [G][B]
-    int G, B, rank;
-    float c, thresh;
-    int greedy;
-    const float* uniforms;
-    float* entropy;
-    uint8_t* stop;
-    int32_t* token;           // greedy: the global argmax; sampling: -1 (the owner fills it in)
-    int32_t* owner;
-    float* ext_target;
-    uint8_t* active;
-    unsigned* status;
-};
-
-__global__ void __launch_bounds__(kPolicyThreads) vp_combine_kernel(VpCombineArgs a) {
-    pdl_launch_dependents();
-    pdl_wait();
-    const int b = blockIdx.x * kPolicyThreads + threadIdx.x;
-    if (b >= a.B) return;
-    float m = neg_inf();
-    for (int g = 0; g < a.G; ++g) m = fmaxf(m, a.partials[static_cast<size_t>(g) * a.B + b].x);
-    const float M = __fmul_rn(m, a.c);
-    float Z = 0.f, A = 0.f;
-    int idx = kIntMax;
-    for (int g = 0; g < a.G; ++g) {
-        const float4 p = a.partials[static_cast<size_t>(g) * a.B + b];
-        if (p.x == m) idx = min(idx, __float_as_int(p.w));
-        if (p.y > 0.f) {
-            float d = __fmul_rn(p.x, a.c) - M;
-            float s = ex2_approx(fmaxf(d, kArgFloor));
-            A += s * __fmaf_rn(d, p.y, p.z);
-            Z += s * p.y;
-        }
-    }
-    const bool ok = Z > 0.f && fabsf(m) <= kMaxLogit;
-    float H = 0.f;
-    if (ok) H = fmaxf(kLn2 * (log2f(Z) - A / Z), 0.f);
-    else atomicOr(a.status, SVIP_STATUS_NONFINITE_ROW);
-    a.entropy[b] = H;
-    a.stop[b] = __fsqrt_rn(H) > a.thresh ? 1 : 0;
-    int owner = -1;
-    float local_target = 0.f;
-    if (!a.greedy && ok) {
-        const float target = a.uniforms[b] * Z;
-        float run = 0.f, before = 0.f;
-        int last = -1;
-        for (int g = 0; g < a.G && owner < 0; ++g) {
-            const float4 p = a.partials[static_cast<size_t>(g) * a.B + b];
-            float mass = 0.f;
-            if (p.y > 0.f) mass = p.y * ex2_approx(fmaxf(__fmul_rn(p.x, a.c) - M, kArgFloor));
-            if (mass > 0.f) {
-                last = g; before = run;
-                if (run + mass > target) owner = g;
-            }
-            run += mass;
-        }
-        if (owner < 0) owner = last;   // rounding: the last shard with mass, searched to its end
-        // the owner looks for (target - before) in units of its own Z, i.e. relative to its own maximum
-        const float4 po = a.partials[static_cast<size_t>(owner) * a.B + b];
-        const float up = ex2_approx(fminf(M - __fmul_rn(po.x, a.c), 126.f));
-        local_target = fminf(fmaxf(target - before, 0.f) * up, po.y);
-    }
-    a.token[b] = a.greedy || !ok ? ((idx != kIntMax) ? idx : 0) : -1;
-    a.owner[b] = owner;
-    a.ext_target[b] = local_target;
-    a.active[b] = owner == a.rank ? 1 : 0;
-}
-
-// ------------------------------------------------------------------ draft-length policies
-//
-// Per-sequence drafting state on the device, so that the loop of Algorithm 1 needs no host round
-// trip per draft token.  ENTROPY is the paper's rule (Eq. 7 flag from the draft step); CONSTANT and
-// HEURISTIC are the two baselines of Section 3.
-
-// Control of a drafting loop recorded as a WHILE node of a CUDA graph.  The kernel that closes an
-// iteration counts it and tells the graph whether the body runs again: only while sequences are
-// still drafting, and never more than `max_iters` times whatever the data say.
-struct LoopCtl {
-    cudaGraphConditionalHandle handle;
-    int* iter;        // iterations done since the loop was entered (NULL: not inside a loop)
-    int max_iters;
-};
-
-__device__ __forceinline__ void loop_decide(const LoopCtl& loop, int n_active) {
-    if (!loop.iter) return;
-    const int it = *loop.iter + 1;
-    *loop.iter = it;
-    cudaGraphSetConditional(loop.handle, (n_active > 0 && it < loop.max_iters) ? 1u : 0u);
-}
-
-struct AdvanceArgs {
-    int policy;
-    const uint8_t* stop;
-    const int32_t* gamma;
-    int32_t* draft_len;
-    uint8_t* active;
-    int B, K_cap;
-    int32_t* n_active;
-    LoopCtl loop;
-};
-
-__global__ void __launch_bounds__(kPolicyThreads) policy_advance_kernel(AdvanceArgs a) {
-    pdl_launch_dependents();
-    pdl_wait();
-    // one block: counts the sequences still drafting while it updates them
-    __shared__ int count;
-    if (threadIdx.x == 0) count = 0;
-    __syncthreads();
-    int mine = 0;
-    for (int i = threadIdx.x; i < a.B; i += kPolicyThreads) {
-        if (!a.active[i]) continue;
-        int len = a.draft_len[i] + 1;
-        a.draft_len[i] = len;
-        bool done;
-        if (a.policy == SVIP_POLICY_ENTROPY) done = a.stop[i] != 0 || len >= a.K_cap;
-        else done = len >= min(a.gamma[i], a.K_cap);
-        if (done) a.active[i] = 0; else ++mine;
-    }
-    if (mine) atomicAdd(&count, mine);
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        if (a.n_active) *a.n_active = count;
-        loop_decide(a.loop, count);
-    }
-}
-
-// Decision of a drafting loop whose body holds no svip_policy_advance on the loop's counter.
-__global__ void loop_decide_kernel(LoopCtl loop, const int32_t* n_active) {
-    pdl_launch_dependents();
-    pdl_wait();
-    if (threadIdx.x == 0) loop_decide(loop, *n_active);
-}
-
-struct UpdateArgs {
-    int policy;
-    const int32_t* n_accepted;
-    int32_t* draft_len;
-    int32_t* gamma;
-    uint8_t* active;
-    int B, K_cap;
-};
-
-__global__ void __launch_bounds__(kPolicyThreads) policy_update_kernel(UpdateArgs a) {
-    pdl_launch_dependents();
-    pdl_wait();
-    int i = blockIdx.x * kPolicyThreads + threadIdx.x;
-    if (i >= a.B) return;
-    if (a.policy == SVIP_POLICY_HEURISTIC) {
-        int g = a.gamma[i];
-        g = a.n_accepted[i] == a.draft_len[i] ? min(g + 2, a.K_cap) : max(g - 1, 1);
-        a.gamma[i] = g;
-    }
-    a.draft_len[i] = 0;
-    a.active[i] = 1;
-}
-
-// ------------------------------------------------------------------ ragged packing
-
-constexpr int kPackThreads = 1024;
-
-__global__ void __launch_bounds__(kPackThreads) pack_ragged_kernel(const int32_t* draft_len, int B, int K_max,
-                                                                   int32_t* cu, int32_t* row_seq,
-                                                                   int32_t* row_pos, unsigned* status) {
-    __shared__ int wsum[32];
-    __shared__ int carry;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    pdl_launch_dependents();
-    pdl_wait();
-    if (tid == 0) carry = 0;
-    __syncthreads();
-    for (int base = 0; base < B; base += kPackThreads) {
-        int i = base + tid;
-        int k = 0;
-        if (i < B) {
-            k = draft_len[i];
-            if (k < 1 || k > K_max) {
-                atomicOr(status, SVIP_STATUS_BAD_DRAFT_LEN);
-                k = k < 1 ? 1 : K_max;
-            }
-            k += 1;
-        }
-        int inc = k;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            int n = __shfl_up_sync(0xffffffffu, inc, o);
-            if (lane >= o) inc += n;
-        }
-        if (lane == 31) wsum[warp] = inc;
-        __syncthreads();
-        int before = 0, tot = 0;
-        for (int w = 0; w < 32; ++w) {
-            int s = wsum[w];
-            if (w < warp) before += s;
-            tot += s;
-        }
-        int c0 = carry;
-        if (i < B) cu[i] = c0 + before + inc - k;
-        __syncthreads();
-        if (tid == 0) carry = c0 + tot;
-        __syncthreads();
-    }
-    const int total = carry;
-    if (tid == 0) cu[B] = total;
-    __syncthreads();
-    if (row_seq || row_pos) {
-        for (int r = tid; r < total; r += kPackThreads) {
-            int lo = 0, hi = B;           // largest i with cu[i] <= r
-            while (hi - lo > 1) {
-                int mid = (lo + hi) >> 1;
-                if (cu[mid] <= r) lo = mid; else hi = mid;
-            }
-            if (row_seq) row_seq[r] = lo;
-            if (row_pos) row_pos[r] = r - cu[lo];
-        }
-    }
-}
-
-}  // namespace svip
+#include "svip_draft.cuh"
+#include "svip_verify.cuh"
+#include "svip_analysis.cuh"
+#include "svip_policy.cuh"
 
 #include "svip_select.cuh"
 
@@ -1931,3 +944,4 @@ int svip_verify_noalloc(int device, const int32_t* draft_tokens, const void* q_l
 }
 
 }  // extern "C"
+
