@@ -27,6 +27,7 @@ constexpr float kMassScale = 1099511627776.0f;   // 2^40
 constexpr int kCandPerBlock = 1024;      // candidate keys a block may collect
 constexpr int kPoolCap = 4096;           // candidate keys of the whole cluster (lives in the histogram copies)
 constexpr int kPoolCapDraft = 2048;      // the same when their indices are kept too (draft form)
+constexpr int kSmallPool = 256;          // up to this many candidates are ranked by plain counting
 
 struct ThresholdArgs {
     const void* logits;
@@ -100,9 +101,10 @@ struct SelectShared {
     unsigned long long warp_above[kWarps];
     // candidate path (top-k with a small k)
     uint32_t lane_key[kThreads];          // key of the largest logit each thread saw
-    uint32_t cand[kCandPerBlock];         // keys of this block's elements >= the lower bound
+    alignas(8) uint32_t cand[kCandPerBlock];   // keys of this block's elements >= the lower bound
     uint32_t cand_idx[kCandPerBlock];     // draft form: their positions in the row
     uint32_t cand_n;                      // how many there are (may exceed the capacity: then the path is left)
+    uint32_t sel;                         // result of a selection by counting
     // decision of a pass (written by warp 0)
     int bin;
     uint32_t cnt_above;
@@ -339,6 +341,47 @@ __device__ __forceinline__ uint32_t pool_select(SelectShared& sh, const uint32_t
     return prefix;
 }
 
+// Selection among a few keys (n <= kSmallPool) by counting, one thread per key: the k-th largest
+// key is the one with fewer than k keys above it and at least k at or above it.  Block-collective.
+__device__ __forceinline__ uint32_t small_select_count(SelectShared& sh, const uint32_t* pool, int n, uint32_t k,
+                                                       int tid) {
+    if (tid == 0) sh.sel = 0;
+    __syncthreads();
+    if (tid < n) {
+        const uint32_t key = pool[tid];
+        uint32_t gt = 0, ge = 0;
+        for (int j = 0; j < n; ++j) {
+            const uint32_t kj = pool[j];
+            gt += kj > key ? 1u : 0u;
+            ge += kj >= key ? 1u : 0u;
+        }
+        if (gt < k && k <= ge) sh.sel = key;   // every thread that qualifies holds the same key
+    }
+    __syncthreads();
+    return sh.sel;
+}
+
+// The same by mass: the largest key (not below key_floor) whose upper set reaches p_rem, i.e. the
+// key with less than p_rem strictly above it and at least p_rem at or above it.  0 if there is none.
+__device__ __forceinline__ uint32_t small_select_mass(SelectShared& sh, const uint32_t* pool,
+                                                      const unsigned long long* wq, int n, uint32_t key_floor,
+                                                      unsigned long long p_rem, int tid) {
+    if (tid == 0) sh.sel = 0;
+    __syncthreads();
+    if (tid < n && pool[tid] >= key_floor) {
+        const uint32_t key = pool[tid];
+        unsigned long long mgt = 0, mge = 0;
+        for (int j = 0; j < n; ++j) {
+            const uint32_t kj = pool[j];
+            if (kj > key) mgt += wq[j];
+            if (kj >= key) mge += wq[j];
+        }
+        if (mgt < p_rem && p_rem <= mge) sh.sel = key;
+    }
+    __syncthreads();
+    return sh.sel;
+}
+
 // The truncated draft step from the candidates alone (block-collective, run by one block): the kept
 // tokens are the candidates with key >= key_t.  Their masses are 2^-40 fixed point, so the
 // normaliser, the entropy sums and the running sums of the inverse CDF are integers and do not
@@ -483,7 +526,10 @@ __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const
     }
     cluster.sync();     // the peers have read this block's candidates
     if (!fits || total < a.top_k) return false;
-    uint32_t key_k = pool_select<kLevels, false>(sh, pool, total, static_cast<uint32_t>(a.top_k), 0ull, 0.f, 0.f, tid);
+    const bool small = total <= kSmallPool;
+    uint32_t key_k = small ? small_select_count(sh, pool, total, static_cast<uint32_t>(a.top_k), tid)
+                           : pool_select<kLevels, false>(sh, pool, total, static_cast<uint32_t>(a.top_k), 0ull, 0.f,
+                                                         0.f, tid);
     uint32_t key_t = key_k;
     float row_max = neg_inf();
     bool finite = false;
@@ -503,16 +549,26 @@ __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const
         M = finite ? __fmul_rn(row_max, a.c) : 0.f;
     }
     if (use_p) {
+        // this block's own candidates have been copied by every peer: their place holds the masses now
+        unsigned long long* wq = reinterpret_cast<unsigned long long*>(sh.cand);
         unsigned long long zk = 0;
-        for (int i = tid; i < total; i += kThreads)
-            if (pool[i] >= key_k) zk += mass_of_key(pool[i], a.c, M);
-        zk = block_sum_u64(sh, zk, tid);
+        if (small) {
+            if (tid < total) wq[tid] = mass_of_key(pool[tid], a.c, M);
+            __syncthreads();
+            for (int j = 0; j < total; ++j)
+                if (pool[j] >= key_k) zk += wq[j];
+        } else {
+            for (int i = tid; i < total; i += kThreads)
+                if (pool[i] >= key_k) zk += mass_of_key(pool[i], a.c, M);
+            zk = block_sum_u64(sh, zk, tid);
+        }
         if (finite && zk > 0) {
             const double want = ceil(static_cast<double>(a.top_p) * static_cast<double>(zk));
             unsigned long long p_rem = static_cast<unsigned long long>(want);
             if (p_rem < 1) p_rem = 1;
             if (p_rem > zk) p_rem = zk;
-            const uint32_t key_p = pool_select<kLevels, true>(sh, pool, total, 0u, p_rem, a.c, M, tid);
+            const uint32_t key_p = small ? small_select_mass(sh, pool, wq, total, key_k, p_rem, tid)
+                                         : pool_select<kLevels, true>(sh, pool, total, 0u, p_rem, a.c, M, tid);
             if (key_p > key_t) key_t = key_p;
         }
     }
