@@ -277,6 +277,24 @@ def b1_latency(ctx, torch):
             out[name.replace("_us", "_to_host_us")] = 1e6 * (time.perf_counter() - t0) / reps
         g.destroy(); one.destroy()
 
+        # one truncated draft step (top-k 50, top-p 0.9) at B = 1, by graph replay
+        thr1 = torch.zeros(1, device="cuda")
+        st.synchronize()
+        ctx.graph_begin(st)
+        ctx.draft_step_truncated(dq, 0, 1, V, V, w.T, w.h, 50, 0.9, ud, None, thr1, tok, ent, stop, stats, st)
+        tg = ctx.graph_end(st)
+        for _ in range(20):
+            tg.launch(st)
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        st.synchronize()
+        e0.record(st)
+        for _ in range(500):
+            tg.launch(st)
+        e1.record(st)
+        st.synchronize()
+        out["truncated_draft_step_us"] = 1000.0 * e0.elapsed_time(e1) / 500
+        tg.destroy()
+
         # the drafting phase as a loop inside the graph (each token: draft step at the sequence's own
         # position + the policy kernel that also decides the loop), against the same two kernels
         # driven from the host, which must read the count of drafting sequences back after every token

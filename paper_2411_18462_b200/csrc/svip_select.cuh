@@ -104,7 +104,8 @@ struct SelectShared {
     alignas(8) uint32_t cand[kCandPerBlock];   // keys of this block's elements >= the lower bound
     uint32_t cand_idx[kCandPerBlock];     // draft form: their positions in the row
     uint32_t cand_n;                      // how many there are (may exceed the capacity: then the path is left)
-    uint32_t sel;                         // result of a selection by counting
+    uint32_t sel, sel2;                   // results of selections by counting
+    uint32_t peer_n[kMaxCluster];         // candidates held by each block of the cluster
     // decision of a pass (written by warp 0)
     int bin;
     uint32_t cnt_above;
@@ -341,45 +342,120 @@ __device__ __forceinline__ uint32_t pool_select(SelectShared& sh, const uint32_t
     return prefix;
 }
 
-// Selection among a few keys (n <= kSmallPool) by counting, one thread per key: the k-th largest
-// key is the one with fewer than k keys above it and at least k at or above it.  Block-collective.
-__device__ __forceinline__ uint32_t small_select_count(SelectShared& sh, const uint32_t* pool, int n, uint32_t k,
-                                                       int tid) {
-    if (tid == 0) sh.sel = 0;
+// Sum over the warp of per-lane masses below 2^48 (a lane adds up at most 8 masses of about 2^40):
+// two 32-bit integer reductions over a 24-bit and a 24-bit limb, neither of which can overflow.
+__device__ __forceinline__ unsigned long long warp_sum_mass(unsigned long long v) {
+    const uint32_t lo = __reduce_add_sync(0xffffffffu, static_cast<uint32_t>(v) & 0xffffffu);
+    const uint32_t hi = __reduce_add_sync(0xffffffffu, static_cast<uint32_t>(v >> 24));
+    return (static_cast<unsigned long long>(hi) << 24) + lo;
+}
+
+// Everything after the candidates are gathered, for a small set (n <= kSmallPool), by plain counting,
+// one warp per candidate (the lanes share the other candidates) and two block barriers: the k-th
+// largest key has fewer than k keys above it and at least k at or above it; the nucleus cut has less
+// than the target mass strictly above it and at least the target at or above it; the sampled token
+// is the kept candidate whose running mass in index order first exceeds u * total.  Masses are the
+// 2^-40 fixed-point integers used everywhere in this file, so nothing depends on the order of the
+// candidates.  Returns the key of tau; `drafted` (block 0, kDraft) tells whether token, entropy
+// and stop flag were written.
+template <bool kDraft>
+__device__ __forceinline__ uint32_t small_finish(SelectShared& sh, const uint32_t* pool, const uint32_t* pool_idx,
+                                                 int n, const ThresholdArgs& a, bool use_p, int row, int rank, int tid,
+                                                 bool& drafted) {
+    const int lane = tid & 31, warp = tid >> 5;
+    // this block's own candidates have been copied by every peer: their place holds the masses now
+    unsigned long long* wq = reinterpret_cast<unsigned long long*>(sh.cand);
+    if (tid == 0) { sh.sel = 0; sh.sel2 = 0; }
+    uint32_t top = 0;
+    for (int j = lane; j < n; j += 32) top = max(top, pool[j]);
+    top = __reduce_max_sync(0xffffffffu, top);
+    const float row_max = key_value(top);          // the largest candidate is the largest logit of the row
+    const bool finite = fabsf(row_max) <= kMaxLogit;
+    const float M = finite ? __fmul_rn(row_max, a.c) : 0.f;
     __syncthreads();
-    if (tid < n) {
-        const uint32_t key = pool[tid];
+    const uint32_t k = static_cast<uint32_t>(a.top_k);
+    for (int i = warp; i < n; i += kWarps) {
+        const uint32_t key = pool[i];
         uint32_t gt = 0, ge = 0;
-        for (int j = 0; j < n; ++j) {
+        for (int j = lane; j < n; j += 32) {
             const uint32_t kj = pool[j];
             gt += kj > key ? 1u : 0u;
             ge += kj >= key ? 1u : 0u;
         }
-        if (gt < k && k <= ge) sh.sel = key;   // every thread that qualifies holds the same key
-    }
-    __syncthreads();
-    return sh.sel;
-}
-
-// The same by mass: the largest key (not below key_floor) whose upper set reaches p_rem, i.e. the
-// key with less than p_rem strictly above it and at least p_rem at or above it.  0 if there is none.
-__device__ __forceinline__ uint32_t small_select_mass(SelectShared& sh, const uint32_t* pool,
-                                                      const unsigned long long* wq, int n, uint32_t key_floor,
-                                                      unsigned long long p_rem, int tid) {
-    if (tid == 0) sh.sel = 0;
-    __syncthreads();
-    if (tid < n && pool[tid] >= key_floor) {
-        const uint32_t key = pool[tid];
-        unsigned long long mgt = 0, mge = 0;
-        for (int j = 0; j < n; ++j) {
-            const uint32_t kj = pool[j];
-            if (kj > key) mgt += wq[j];
-            if (kj >= key) mge += wq[j];
+        gt = __reduce_add_sync(0xffffffffu, gt);
+        ge = __reduce_add_sync(0xffffffffu, ge);
+        if (lane == 0) {
+            if (gt < k && k <= ge) sh.sel = key;   // every candidate that qualifies holds the same key
+            wq[i] = mass_of_key(key, a.c, M);
         }
-        if (mgt < p_rem && p_rem <= mge) sh.sel = key;
     }
     __syncthreads();
-    return sh.sel;
+    const uint32_t key_k = sh.sel;
+    uint32_t key_t = key_k;
+    if (use_p && finite) {
+        unsigned long long zk = 0;
+        for (int j = lane; j < n; j += 32)
+            if (pool[j] >= key_k) zk += wq[j];
+        zk = warp_sum_mass(zk);
+        if (zk > 0) {
+            const double want = ceil(static_cast<double>(a.top_p) * static_cast<double>(zk));
+            unsigned long long p_rem = static_cast<unsigned long long>(want);
+            if (p_rem < 1) p_rem = 1;
+            if (p_rem > zk) p_rem = zk;
+            for (int i = warp; i < n; i += kWarps) {
+                const uint32_t key = pool[i];
+                if (key < key_k) continue;          // warp-uniform
+                unsigned long long mgt = 0, mge = 0;
+                for (int j = lane; j < n; j += 32) {
+                    const uint32_t kj = pool[j];
+                    const unsigned long long w = wq[j];
+                    if (kj > key) mgt += w;
+                    if (kj >= key) mge += w;
+                }
+                mgt = warp_sum_mass(mgt);
+                mge = warp_sum_mass(mge);
+                if (lane == 0 && mgt < p_rem && p_rem <= mge) sh.sel2 = key;
+            }
+        }
+        __syncthreads();
+        if (sh.sel2 > key_t) key_t = sh.sel2;
+    }
+    drafted = false;
+    if (a.stats || kDraft) {
+        unsigned long long zt = 0;
+        for (int j = lane; j < n; j += 32)
+            if (pool[j] >= key_t) zt += wq[j];
+        zt = warp_sum_mass(zt);
+        if (a.stats && rank == 0 && tid == 0) a.stats[row] = kept_stats(row_max, zt, finite);
+        if (kDraft && rank == 0 && finite && zt > 0) {
+            long long term = 0;
+            if (tid < n && pool[tid] >= key_t) {
+                const float arg = fmaxf(__fmaf_rn(key_value(pool[tid]), a.c, -M), kArgFloor);
+                term = __float2ll_rz(ex2_approx(arg) * arg * kMassScale);
+            }
+            const long long aq = static_cast<long long>(block_sum_u64(sh, static_cast<unsigned long long>(term), tid));
+            const float u = a.uniforms[row];
+            const unsigned long long target = static_cast<unsigned long long>(static_cast<double>(u) * static_cast<double>(zt));
+            for (int i = warp; i < n; i += kWarps) {
+                if (pool[i] < key_t) continue;      // warp-uniform
+                const uint32_t at = pool_idx[i];
+                unsigned long long cum = 0;
+                for (int j = lane; j < n; j += 32)
+                    if (pool[j] >= key_t && pool_idx[j] <= at) cum += wq[j];
+                cum = warp_sum_mass(cum);
+                if (lane == 0 && cum > target && cum - wq[i] <= target) {   // exactly one kept candidate
+                    const float Z = static_cast<float>(static_cast<double>(zt) / 1099511627776.0);
+                    const float A = static_cast<float>(static_cast<double>(aq) / 1099511627776.0);
+                    const float H = fmaxf(kLn2 * (log2f(Z) - A / Z), 0.f);
+                    a.token[row] = static_cast<int32_t>(at);
+                    a.entropy[row] = H;
+                    a.stop[row] = __fsqrt_rn(H) > a.thresh ? 1 : 0;
+                }
+            }
+            drafted = true;
+        }
+    }
+    return key_t;
 }
 
 // The truncated draft step from the candidates alone (block-collective, run by one block): the kept
@@ -486,10 +562,12 @@ __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const
     const int n_lane = S * kThreads;
     for (int r = 0; r < S; ++r) pool[r * kThreads + tid] = cluster.map_shared_rank(&sh, r)->lane_key[tid];
     __syncthreads();
-    const uint32_t t0 = pool_select<kLevels, false>(sh, pool, n_lane, static_cast<uint32_t>(a.top_k), 0ull, 0.f, 0.f, tid);
+    // only a lower bound is needed: two digits of the k-th largest maximum, the rest taken as zero
+    const uint32_t t0 = pool_select<2, false>(sh, pool, n_lane, static_cast<uint32_t>(a.top_k), 0ull, 0.f, 0.f, tid) &
+                        0xffff0000u;
     // pass 2: every element at or above the lower bound.  Comparing the logits is comparing the keys,
     // except for NaN, which counts as -inf and so belongs to the candidates only when the bound is that low.
-    const float t0v = t0 ? key_value(t0) : neg_inf();
+    const float t0v = t0 > 0x007fffffu ? key_value(t0) : neg_inf();   // at or below the key of -inf: no bound
     const bool lowest = !(t0v > neg_inf());
     stream_segment<DT>(g, rank * kWarps + warp, lane, slot0, [&](const float (&x)[EPV], int vi) {
 #pragma unroll
@@ -504,32 +582,34 @@ __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const
         }
     });
     cluster.sync();     // every block's candidates are complete (and nobody still reads lane_key)
+    if (tid < S) sh.peer_n[tid] = cluster.map_shared_rank(&sh, tid)->cand_n;   // one remote read each, side by side
+    __syncthreads();
     int total = 0;
     bool fits = true;
     for (int r = 0; r < S; ++r) {
-        const uint32_t nr = cluster.map_shared_rank(&sh, r)->cand_n;
+        const uint32_t nr = sh.peer_n[r];
         if (nr > kCandPerBlock) fits = false;
         total += static_cast<int>(min(nr, static_cast<uint32_t>(kCandPerBlock)));
     }
     if (total > kCap) fits = false;
     if (fits) {
-        int at = 0;
-        for (int r = 0; r < S; ++r) {
+        // candidate t of the cluster is candidate t - (candidates of the blocks before) of its block
+        for (int t = tid; t < total; t += kThreads) {
+            int r = 0, at = t;
+            while (at >= static_cast<int>(sh.peer_n[r])) { at -= static_cast<int>(sh.peer_n[r]); ++r; }
             const SelectShared* peer = cluster.map_shared_rank(&sh, r);
-            const int nr = static_cast<int>(peer->cand_n);
-            for (int i = tid; i < nr; i += kThreads) {
-                pool[at + i] = peer->cand[i];
-                if (kDraft) pool_idx[at + i] = peer->cand_idx[i];
-            }
-            at += nr;
+            pool[t] = peer->cand[at];
+            if (kDraft) pool_idx[t] = peer->cand_idx[at];
         }
     }
     cluster.sync();     // the peers have read this block's candidates
     if (!fits || total < a.top_k) return false;
-    const bool small = total <= kSmallPool;
-    uint32_t key_k = small ? small_select_count(sh, pool, total, static_cast<uint32_t>(a.top_k), tid)
-                           : pool_select<kLevels, false>(sh, pool, total, static_cast<uint32_t>(a.top_k), 0ull, 0.f,
-                                                         0.f, tid);
+    const int row = static_cast<int>(blockIdx.x / S);
+    if (total <= kSmallPool) {
+        key_out = small_finish<kDraft>(sh, pool, pool_idx, total, a, use_p, row, rank, tid, drafted);
+        return true;
+    }
+    uint32_t key_k = pool_select<kLevels, false>(sh, pool, total, static_cast<uint32_t>(a.top_k), 0ull, 0.f, 0.f, tid);
     uint32_t key_t = key_k;
     float row_max = neg_inf();
     bool finite = false;
@@ -549,26 +629,16 @@ __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const
         M = finite ? __fmul_rn(row_max, a.c) : 0.f;
     }
     if (use_p) {
-        // this block's own candidates have been copied by every peer: their place holds the masses now
-        unsigned long long* wq = reinterpret_cast<unsigned long long*>(sh.cand);
         unsigned long long zk = 0;
-        if (small) {
-            if (tid < total) wq[tid] = mass_of_key(pool[tid], a.c, M);
-            __syncthreads();
-            for (int j = 0; j < total; ++j)
-                if (pool[j] >= key_k) zk += wq[j];
-        } else {
-            for (int i = tid; i < total; i += kThreads)
-                if (pool[i] >= key_k) zk += mass_of_key(pool[i], a.c, M);
-            zk = block_sum_u64(sh, zk, tid);
-        }
+        for (int i = tid; i < total; i += kThreads)
+            if (pool[i] >= key_k) zk += mass_of_key(pool[i], a.c, M);
+        zk = block_sum_u64(sh, zk, tid);
         if (finite && zk > 0) {
             const double want = ceil(static_cast<double>(a.top_p) * static_cast<double>(zk));
             unsigned long long p_rem = static_cast<unsigned long long>(want);
             if (p_rem < 1) p_rem = 1;
             if (p_rem > zk) p_rem = zk;
-            const uint32_t key_p = small ? small_select_mass(sh, pool, wq, total, key_k, p_rem, tid)
-                                         : pool_select<kLevels, true>(sh, pool, total, 0u, p_rem, a.c, M, tid);
+            const uint32_t key_p = pool_select<kLevels, true>(sh, pool, total, 0u, p_rem, a.c, M, tid);
             if (key_p > key_t) key_t = key_p;
         }
     }
@@ -577,13 +647,12 @@ __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const
         for (int i = tid; i < total; i += kThreads)
             if (pool[i] >= key_t) zt += mass_of_key(pool[i], a.c, M);
         zt = block_sum_u64(sh, zt, tid);
-        if (rank == 0 && tid == 0) a.stats[blockIdx.x / S] = kept_stats(row_max, zt, finite);
+        if (rank == 0 && tid == 0) a.stats[row] = kept_stats(row_max, zt, finite);
     }
     key_out = key_t;
     if (kDraft && rank == 0) {
         __syncthreads();   // the pool is complete and the ring is idle in every warp
-        drafted = draft_from_candidates(sh, pool, pool_idx, total, key_t, row_max, M, finite, a,
-                                        static_cast<int>(blockIdx.x / S), scratch, tid);
+        drafted = draft_from_candidates(sh, pool, pool_idx, total, key_t, row_max, M, finite, a, row, scratch, tid);
     }
     return true;
 }
