@@ -207,15 +207,15 @@ int svip_draft_step_filtered(svip_ctx* ctx, const void* logits, svip_dtype dtype
                              const uint8_t* active, const float* thr, int32_t* token, float* entropy,
                              uint8_t* stop, float* row_stats, void* stream);
 /*
- * svip_row_threshold and svip_draft_step_filtered in one call: thr[b] receives
- * the threshold of row b for (top_k, top_p), and token / entropy / stop /
- * row_stats the truncated draft step at it.  With a small top_k (see
- * svip_row_threshold) the first kernel finishes the whole step from the few
- * candidates it holds in shared memory, two passes over the row in all; rows
- * it cannot finish that way (nucleus alone, large top_k, many ties at the cut)
- * go through the streaming kernel in a second launch, which skips the others.
+ * svip_row_threshold and svip_draft_step_filtered in one call and one kernel:
+ * thr[b] receives the threshold of row b for (top_k, top_p), and token /
+ * entropy / stop / row_stats the truncated draft step at it.  With a small
+ * top_k (see svip_row_threshold) the kernel finishes the whole step from the
+ * few candidates it holds in shared memory, two passes over the row in all;
+ * rows it cannot finish that way (nucleus alone, large top_k, many ties at
+ * the cut) are streamed once more at the threshold, by the same cluster.
  * Results are those of the two separate calls within the stated tolerances
- * (sums are formed in another order).  B <= max_rows of svip_create.
+ * (sums are formed in another order).
  */
 int svip_draft_step_truncated(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, int V,
                               long row_stride, float T, float thresh, int top_k, float top_p,

@@ -44,7 +44,6 @@ struct svip_ctx {
     float2* q_stats;
     int32_t* p_argmax;
     unsigned* status;
-    uint8_t* need;             // device [max_rows]: rows that svip_draft_step_truncated leaves to the streaming kernel
     int* loop_iter;            // device: iteration counter of the drafting loop being replayed
     cudaStream_t loop_stream;  // records the body of a drafting loop
     int loop_open;             // a loop body is being recorded
@@ -210,7 +209,6 @@ int svip_create(svip_ctx** out, int device, int max_rows) {
             cudaMalloc(&c->p_argmax, n * sizeof(int32_t)) != cudaSuccess ||
             cudaMalloc(&c->status, sizeof(unsigned)) != cudaSuccess ||
             cudaMemset(c->status, 0, sizeof(unsigned)) != cudaSuccess ||
-            cudaMalloc(&c->need, n) != cudaSuccess ||
             cudaMalloc(&c->loop_iter, sizeof(int)) != cudaSuccess ||
             cudaMemset(c->loop_iter, 0, sizeof(int)) != cudaSuccess) {
             rc = SVIP_ERR_CUDA;
@@ -219,7 +217,7 @@ int svip_create(svip_ctx** out, int device, int max_rows) {
     if (rc != SVIP_OK) {
         cudaGetLastError();
         cudaFree(c->p_stats); cudaFree(c->q_stats); cudaFree(c->p_argmax); cudaFree(c->status);
-        cudaFree(c->loop_iter); cudaFree(c->need);
+        cudaFree(c->loop_iter);
         delete c;
     } else {
         *out = c;
@@ -234,7 +232,7 @@ int svip_destroy(svip_ctx* ctx) {
     cudaGetDevice(&prev);
     cudaSetDevice(ctx->device);
     cudaFree(ctx->p_stats); cudaFree(ctx->q_stats); cudaFree(ctx->p_argmax); cudaFree(ctx->status);
-    cudaFree(ctx->loop_iter); cudaFree(ctx->need);
+    cudaFree(ctx->loop_iter);
     if (ctx->loop_stream) cudaStreamDestroy(ctx->loop_stream);
     if (ctx->prof_start) {
         for (int k = 0; k < kProfilePairs; ++k) {
@@ -359,7 +357,7 @@ int svip_row_threshold(svip_ctx* ctx, const void* logits, svip_dtype dtype, int 
     a.stats = reinterpret_cast<float2*>(stats);
     if (stats && !aligned_to(stats, 8)) return SVIP_ERR_INVALID_ARG;
     a.uniforms = nullptr; a.active = nullptr; a.thresh = 0.f; a.token = nullptr; a.entropy = nullptr;
-    a.stop = nullptr; a.need = nullptr;
+    a.stop = nullptr; a.status = ctx->status;
     const int S = pick_cluster(ctx, n_rows, V, dtype);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = dtype == SVIP_BF16 ? launch_clustered(row_threshold_kernel<kBF16>, n_rows, S, a, st, kRingBytes)
@@ -380,13 +378,12 @@ int svip_draft_step_truncated(svip_ctx* ctx, const void* logits, svip_dtype dtyp
     if (!aligned_to(logits, dtype == SVIP_BF16 ? 2 : 4)) return SVIP_ERR_INVALID_ARG;
     if (row_stats && !aligned_to(row_stats, 8)) return SVIP_ERR_INVALID_ARG;
     if (B == 0) return SVIP_OK;
-    if (B > ctx->max_rows) return SVIP_ERR_WORKSPACE;
     ThresholdArgs a;
     a.logits = logits; a.row_stride = row_stride; a.V = V; a.c = scale_for(T);
     a.top_k = (top_k >= 1 && top_k < V) ? top_k : 0; a.top_p = top_p; a.thr = thr;
     a.stats = reinterpret_cast<float2*>(row_stats);
     a.uniforms = uniforms; a.active = active; a.thresh = thresh; a.token = token; a.entropy = entropy;
-    a.stop = stop; a.need = ctx->need;
+    a.stop = stop; a.status = ctx->status;
     const int S = pick_cluster(ctx, B, V, dtype);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = dtype == SVIP_BF16
@@ -394,9 +391,7 @@ int svip_draft_step_truncated(svip_ctx* ctx, const void* logits, svip_dtype dtyp
         : launch_clustered(row_threshold_kernel<kF32, true>, B, S, a, st, kRingBytes);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     ctx->launches += 1;
-    // the rows the candidates could not finish: the streaming draft step at the thresholds just found
-    return svip_draft_step_filtered(ctx, logits, dtype, B, V, row_stride, T, thresh, uniforms, ctx->need, thr, token,
-                                    entropy, stop, row_stats, stream);
+    return SVIP_OK;
 }
 
 int svip_pack_ragged(svip_ctx* ctx, const int32_t* draft_len, int B, int K_max, int32_t* cu_rows,

@@ -176,50 +176,31 @@ struct RowShared {
     SegPick pick;
 };
 
-// kBlocks is the number of blocks the register budget must leave room for on one SM: 2 for
-// launches that fit the GPU in one wave (latency matters, registers are free), 3 for launches of
-// many waves, where a third resident block streams on while another one is in its epilogue.
-// kPos compiles the position-indexed form (svip_draft_step_at) in, kThr the truncated form
-// (svip_draft_step_filtered).
-template <int DT, bool kGreedy, int kBlocks, bool kPos = false, bool kThr = false>
-__global__ void __launch_bounds__(kThreads, kBlocks) draft_step_kernel(DraftArgs a) {
+// The draft step of one row by the cluster that shares it: stream the row (Z, A, maximum), combine the
+// segment partials through distributed shared memory, write entropy / stop flag / normalisers, and
+// let the block that holds the sampled mass find the token.  `rp` / `g` describe the row, `thr` is
+// the truncation threshold when kThr.  Ends with the cluster barrier that keeps a block alive while
+// peers may still read its shared memory.
+template <int DT, bool kGreedy, bool kPos, bool kThr>
+__device__ __forceinline__ void draft_row(const DraftArgs& a, cg::cluster_group& cluster, int S, int rank, int row,
+                                          int tid, const RowGeom g, const uint32_t slot0, const long p, const float thr) {
     constexpr int EPV = ElemTraits<DT>::kEPV;
-    extern __shared__ uint4 ring[];
-    cg::cluster_group cluster = cg::this_cluster();
-    const int S = cluster.dim_blocks().x;
-    const int rank = cluster.block_rank();
-    const int row = blockIdx.x / S;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int lane = tid & 31, warp = tid >> 5;
     __shared__ SegEntry seg[kWarps];
     __shared__ ScanShared scan;
     __shared__ RowShared res;
-
-    pdl_launch_dependents();
-    const char* rp = static_cast<const char*>(a.logits) +
-                     static_cast<size_t>(row) * a.row_stride * ElemTraits<DT>::kBytes;
-    RowGeom g = make_geom<DT>(rp, a.V, S * kWarps);
-    const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
-    pdl_wait();
-    if (a.active && !a.active[row]) return;   // the whole cluster leaves together
-    long p = 0;
-    if (kPos) {
-        p = a.pos[row];
-        rp += p * a.pos_stride * ElemTraits<DT>::kBytes;
-        g = make_geom<DT>(rp, a.V, S * kWarps);
-    }
     float u = 0.f, ext = -1.f;
     if (!kGreedy && warp == 0) {   // fetched now, used after the stream
         if (a.ext_target) ext = fmaxf(__ldg(a.ext_target + row), 0.f);
         else u = __ldg(a.uniforms + (row + p * a.slot_stride));
     }
-    const float thr = kThr ? a.thr[row] : neg_inf();
     Partial t = reduce_segment<DT, 2, kGreedy, kThr>(g, rank * kWarps + warp, a.c, lane, slot0, thr);
     if (lane == 0) { seg[warp].m = t.m; seg[warp].idx = t.idx; seg[warp].Z = t.Z; seg[warp].A = t.A; }
     cluster.sync();
     if (warp == 0) {
-        Partial r; SegPick p;
-        combine_segments<2>(cluster, seg, S, a.c, u, lane, r, p, ext);
-        if (lane == 0) { res.row = r; res.pick = p; }
+        Partial r; SegPick pk;
+        combine_segments<2>(cluster, seg, S, a.c, u, lane, r, pk, ext);
+        if (lane == 0) { res.row = r; res.pick = pk; }
     }
     cluster_arrive();   // done with the peers' shared memory
     __syncthreads();    // res is visible block-wide
@@ -247,6 +228,37 @@ __global__ void __launch_bounds__(kThreads, kBlocks) draft_step_kernel(DraftArgs
         if (tid == 0) a.token[slot] = (virt >= 0 ? virt - g.pre : 0) + a.token_offset;
     }
     cluster_wait();     // no block leaves while a peer may still read its shared memory
+}
+
+// kBlocks is the number of blocks the register budget must leave room for on one SM: 2 for
+// launches that fit the GPU in one wave (latency matters, registers are free), 3 for launches of
+// many waves, where a third resident block streams on while another one is in its epilogue.
+// kPos compiles the position-indexed form (svip_draft_step_at) in, kThr the truncated form
+// (svip_draft_step_filtered).
+template <int DT, bool kGreedy, int kBlocks, bool kPos = false, bool kThr = false>
+__global__ void __launch_bounds__(kThreads, kBlocks) draft_step_kernel(DraftArgs a) {
+    extern __shared__ uint4 ring[];
+    cg::cluster_group cluster = cg::this_cluster();
+    const int S = cluster.dim_blocks().x;
+    const int rank = cluster.block_rank();
+    const int row = blockIdx.x / S;
+    const int tid = threadIdx.x;
+
+    pdl_launch_dependents();
+    const char* rp = static_cast<const char*>(a.logits) +
+                     static_cast<size_t>(row) * a.row_stride * ElemTraits<DT>::kBytes;
+    RowGeom g = make_geom<DT>(rp, a.V, S * kWarps);
+    const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
+    pdl_wait();
+    if (a.active && !a.active[row]) return;   // the whole cluster leaves together
+    long p = 0;
+    if (kPos) {
+        p = a.pos[row];
+        rp += p * a.pos_stride * ElemTraits<DT>::kBytes;
+        g = make_geom<DT>(rp, a.V, S * kWarps);
+    }
+    const float thr = kThr ? a.thr[row] : neg_inf();
+    draft_row<DT, kGreedy, kPos, kThr>(a, cluster, S, rank, row, tid, g, slot0, p, thr);
 }
 
 // ------------------------------------------------------------------ row statistics (verify, phase 1)

@@ -18,6 +18,7 @@
 #pragma once
 
 #include "svip_device.cuh"
+#include "svip_draft.cuh"
 
 namespace svip {
 
@@ -45,7 +46,7 @@ struct ThresholdArgs {
     int32_t* token;          // [rows] out
     float* entropy;          // [rows] out
     uint8_t* stop;           // [rows] out
-    uint8_t* need;           // [rows] out: 1 where the row still needs the streaming draft step
+    unsigned* status;        // device status word
 };
 
 // Monotone image of a float: a < b  <=>  key(a) < key(b).  NaN counts as -inf.
@@ -356,8 +357,8 @@ __device__ __forceinline__ unsigned long long warp_sum_mass(unsigned long long v
 // than the target mass strictly above it and at least the target at or above it; the sampled token
 // is the kept candidate whose running mass in index order first exceeds u * total.  Masses are the
 // 2^-40 fixed-point integers used everywhere in this file, so nothing depends on the order of the
-// candidates.  Returns the key of tau; `drafted` (block 0, kDraft) tells whether token, entropy
-// and stop flag were written.
+// candidates.  Returns the key of tau; `drafted` (kDraft; the same in every block) tells whether
+// block 0 has written token, entropy and stop flag.
 template <bool kDraft>
 __device__ __forceinline__ uint32_t small_finish(SelectShared& sh, const uint32_t* pool, const uint32_t* pool_idx,
                                                  int n, const ThresholdArgs& a, bool use_p, int row, int rank, int tid,
@@ -427,7 +428,8 @@ __device__ __forceinline__ uint32_t small_finish(SelectShared& sh, const uint32_
             if (pool[j] >= key_t) zt += wq[j];
         zt = warp_sum_mass(zt);
         if (a.stats && rank == 0 && tid == 0) a.stats[row] = kept_stats(row_max, zt, finite);
-        if (kDraft && rank == 0 && finite && zt > 0) {
+        drafted = kDraft && finite && zt > 0;   // the same in every block of the cluster
+        if (drafted && rank == 0) {
             long long term = 0;
             if (tid < n && pool[tid] >= key_t) {
                 const float arg = fmaxf(__fmaf_rn(key_value(pool[tid]), a.c, -M), kArgFloor);
@@ -452,7 +454,6 @@ __device__ __forceinline__ uint32_t small_finish(SelectShared& sh, const uint32_
                     a.stop[row] = __fsqrt_rn(H) > a.thresh ? 1 : 0;
                 }
             }
-            drafted = true;
         }
     }
     return key_t;
@@ -535,7 +536,7 @@ __device__ __forceinline__ bool draft_from_candidates(SelectShared& sh, const ui
 // full.  Returns false (for the whole cluster alike) when the candidates do not fit; nothing has
 // been written then and the caller takes the radix descent over the full row.
 // kDraft also keeps the positions of the candidates and lets block 0 finish the whole draft step from
-// them (`drafted`, meaningful in block 0 only); `scratch` is the streaming ring, free by then.
+// them (`drafted`, the same in every block); `scratch` is the streaming ring, free by then.
 template <int DT, bool kDraft>
 __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const RowGeom& g, int S, int rank, int tid,
                                                uint32_t slot0, const ThresholdArgs& a, bool use_p, SelectShared& sh,
@@ -650,16 +651,36 @@ __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const
         if (rank == 0 && tid == 0) a.stats[row] = kept_stats(row_max, zt, finite);
     }
     key_out = key_t;
-    if (kDraft && rank == 0) {
-        __syncthreads();   // the pool is complete and the ring is idle in every warp
-        drafted = draft_from_candidates(sh, pool, pool_idx, total, key_t, row_max, M, finite, a, row, scratch, tid);
+    if (kDraft) {
+        // whether the row has finite mass decides, for all blocks alike, who finishes the step
+        unsigned long long zt = 0;
+        for (int i = tid; i < total; i += kThreads)
+            if (pool[i] >= key_t) zt += mass_of_key(pool[i], a.c, M);
+        zt = block_sum_u64(sh, zt, tid);
+        drafted = finite && zt > 0;
+        if (drafted && rank == 0) {
+            __syncthreads();   // the pool is complete and the ring is idle in every warp
+            draft_from_candidates(sh, pool, pool_idx, total, key_t, row_max, M, finite, a, row, scratch, tid);
+        }
     }
     return true;
 }
 
-// kDraft: the truncated draft step in the same launch wherever the candidate path applies; the rows
-// it could not finish (nucleus alone, large k, heavy ties, no finite mass) are marked in `need` and
-// left to the streaming kernel, with their threshold already in `thr`.
+// The streaming draft step of the row at the threshold just found, for the rows the candidates
+// could not finish (nucleus alone, large k, heavy ties, no finite mass).  Cluster-collective.
+template <int DT>
+__device__ __forceinline__ void draft_at_threshold(const ThresholdArgs& a, cg::cluster_group& cluster, int S, int rank,
+                                                   int row, int tid, const RowGeom& g, uint32_t slot0, float thr) {
+    DraftArgs d;
+    d.logits = a.logits; d.row_stride = a.row_stride; d.V = a.V; d.c = a.c; d.thresh = a.thresh; d.greedy = 0;
+    d.uniforms = a.uniforms; d.token = a.token; d.entropy = a.entropy; d.stop = a.stop;
+    d.row_stats = reinterpret_cast<float*>(a.stats); d.status = a.status; d.active = nullptr;
+    d.ext_target = nullptr; d.token_offset = 0; d.pos = nullptr; d.pos_stride = 0; d.slot_stride = 0; d.thr = nullptr;
+    draft_row<DT, false, false, true>(d, cluster, S, rank, row, tid, g, slot0, 0, thr);
+}
+
+// kDraft: the truncated draft step in the same launch: from the candidates where that path applies,
+// else by streaming the row once more at the threshold just found.
 template <int DT, bool kDraft = false>
 __global__ void __launch_bounds__(kThreads, 2) row_threshold_kernel(ThresholdArgs a) {
     constexpr int kLevels = DT == kBF16 ? 2 : 4;   // the low 16 bits of a bf16 logit carry nothing
@@ -676,10 +697,7 @@ __global__ void __launch_bounds__(kThreads, 2) row_threshold_kernel(ThresholdArg
     const RowGeom g = make_geom<DT>(rp, a.V, S * kWarps);
     const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
     pdl_wait();
-    if (kDraft && a.active && !a.active[row]) {   // the whole cluster leaves together
-        if (rank == 0 && tid == 0) a.need[row] = 0;
-        return;
-    }
+    if (kDraft && a.active && !a.active[row]) return;   // the whole cluster leaves together
 
     const bool use_k = a.top_k >= 1 && a.top_k < a.V;
     const bool use_p = a.top_p < 1.0f;
@@ -693,10 +711,9 @@ __global__ void __launch_bounds__(kThreads, 2) row_threshold_kernel(ThresholdArg
         uint32_t key_t = 0;
         bool drafted = false;
         if (candidate_path<DT, kDraft>(cluster, g, S, rank, tid, slot0, a, use_p, sh, key_t, ring, drafted)) {
-            if (rank == 0 && tid == 0) {
-                a.thr[row] = key_t ? key_value(key_t) : neg_inf();
-                if (kDraft) a.need[row] = drafted ? 0 : 1;
-            }
+            const float thr = key_t ? key_value(key_t) : neg_inf();
+            if (rank == 0 && tid == 0) a.thr[row] = thr;
+            if (kDraft && !drafted) draft_at_threshold<DT>(a, cluster, S, rank, row, tid, g, slot0, thr);
             return;
         }
     }
@@ -780,9 +797,10 @@ __global__ void __launch_bounds__(kThreads, 2) row_threshold_kernel(ThresholdArg
         if (above == 0 || !finite) key_p = 0;   // a row without mass: the nucleus drops nothing
         key_t = key_p > key_k ? key_p : key_k;
     }
-    if (rank == 0 && tid == 0) {
-        a.thr[row] = key_t ? key_value(key_t) : neg_inf();
-        if (kDraft) a.need[row] = 1;
+    if (rank == 0 && tid == 0) a.thr[row] = key_t ? key_value(key_t) : neg_inf();
+    if (kDraft) {
+        draft_at_threshold<DT>(a, cluster, S, rank, row, tid, g, slot0, key_t ? key_value(key_t) : neg_inf());
+        return;
     }
     if (a.stats && !kDraft) {
         // the mass of the kept set: one more pass (the descents above know it only in part)

@@ -320,17 +320,11 @@ def test_truncated_draft_step_in_one_call(ctx, oracle, dtype, V, k, p):
 
 def test_truncated_draft_step_bad_arguments(ctx):
     import torch
-    from paper_2411_18462_b200 import Context, SvipError
+    from paper_2411_18462_b200 import SvipError
     x = torch.zeros(4, 64, device="cuda"); f = torch.zeros(8, device="cuda")
     i = torch.zeros(8, dtype=torch.int32, device="cuda"); b = torch.zeros(8, dtype=torch.uint8, device="cuda")
     with pytest.raises(SvipError):
         ctx.draft_step_truncated(x, 0, 4, 64, 64, 0.0, 0.3, 5, 0.9, f, None, f, i, f, b)     # greedy
     with pytest.raises(SvipError):
         ctx.draft_step_truncated(x, 0, 4, 64, 64, 1.0, 0.3, 5, 0.9, None, None, f, i, f, b)  # no uniforms
-    small = Context(0, 2)
-    try:
-        with pytest.raises(SvipError):
-            small.draft_step_truncated(x, 0, 4, 64, 64, 1.0, 0.3, 5, 0.9, f, None, f, i, f, b)   # more rows than the workspace
-    finally:
-        small.destroy()
     ctx.draft_step_truncated(x, 0, 0, 64, 64, 1.0, 0.3, 5, 0.9, f, None, f, i, f, b)         # empty batch
