@@ -422,9 +422,19 @@ def cpu_baseline(w, seconds_budget=20.0):
     dt = time.perf_counter() - t0
     rejected = int((nacc < lens).sum())
     nbytes = (len(rows_q) + len(rows_t) + rejected) * w.V * w.elem_bytes
+    # the same on one thread, over a sixteenth of the sample (whole sequences)
+    n1 = max(1, n_seq // 16)
+    q1 = int(lens[:n1].sum()); t1 = int(cu[n1])
+    t0 = time.perf_counter()
+    tok1, _, _ = O.draft_step(q[:q1], w.T, w.h, ud[:q1], threads=1)
+    nacc1, _, _ = O.verify(tok1.astype(np.int32), q[:q1], t[:t1], cu[:n1 + 1], w.T, uv[:t1], threads=1)
+    dt1 = time.perf_counter() - t0
+    bytes1 = (q1 + t1 + int((nacc1 < lens[:n1]).sum())) * w.V * w.elem_bytes
     return {"value": nbytes / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
             "sample": "%d of %d sequences (%d draft + %d target rows), one pass, %.1f s" % (
-                n_seq, w.B, len(rows_q), len(rows_t), dt)}
+                n_seq, w.B, len(rows_q), len(rows_t), dt),
+            "single_thread_value": bytes1 / dt1 / 1e9,
+            "single_thread_sample": "%d sequences (%d rows), %.1f s" % (n1, q1 + t1, dt1)}
 
 
 def run_ours(args):
