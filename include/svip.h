@@ -63,6 +63,8 @@ typedef enum {
 /* bits of the device status word */
 #define SVIP_STATUS_NONFINITE_ROW 1u /* some row's maximum was +inf, or every logit was -inf / NaN */
 #define SVIP_STATUS_BAD_DRAFT_LEN 2u /* svip_pack_ragged saw K_i outside [1, K_max] (it was clamped) */
+#define SVIP_STATUS_WAIT_TIMEOUT 4u  /* a block waited a second for its cluster's partial results and gave up; the
+                                        outputs of that call are not valid */
 
 /* draft-side layout selector for svip_verify: rows packed sequence after sequence */
 #define SVIP_Q_PACKED (-1L)

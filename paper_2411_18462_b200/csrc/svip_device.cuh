@@ -253,6 +253,63 @@ __device__ __forceinline__ void cluster_wait() {
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
+// ---------------------------------------------------------------------------
+// Exchange of segment partials inside a cluster without a closing barrier: every warp pushes its
+// 16-byte entry into the shared memory of every block of the cluster (st.async through distributed
+// shared memory), and each push counts its bytes on the receiving block's mbarrier.  A block then
+// only waits on its own mbarrier until all entries of the cluster have landed: one one-way trip
+// instead of a barrier round trip followed by remote reads.  Nothing is read remotely, so a block may
+// leave as soon as its own mbarrier has completed (all writes aimed at it have arrived by then).
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n"
+        " mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+        " selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // one second: far beyond any exchange, short for a hang
+
+// Waits for the phase `parity` of the mbarrier, at most limit_ns nanoseconds.  Returns false if the
+// time ran out (the caller records it in the status word and carries on with what it has).
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
+                                                  unsigned long long limit_ns = kWaitLimitNs) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (global_timer_ns() - t0 > limit_ns) return false;
+    }
+}
+// Address of the same shared-memory location in block `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t saddr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+// 16 bytes into a peer's shared memory; the peer's mbarrier is credited with 16 bytes when they land.
+__device__ __forceinline__ void push16(uint32_t remote_addr, uint32_t remote_bar, uint32_t a, uint32_t b,
+                                       uint32_t c, uint32_t d) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
+                 ::"r"(remote_addr), "r"(a), "r"(b), "r"(c), "r"(d), "r"(remote_bar) : "memory");
+}
+
 typedef unsigned long long f32x2;   // two packed fp32 values
 __device__ __forceinline__ f32x2 pack2(float a, float b) {
     f32x2 r;
@@ -663,9 +720,9 @@ __device__ __forceinline__ SegPick pick_segment(const float (&mass)[kSegPerLane]
 // Shared scratch of the fine scan.
 struct ScanShared {
     float wsum[kWarps];
-    int hit;       // lowest thread whose run of vectors crosses the target
-    int lastpos;   // highest vector with positive weight
-    int result;    // the element found
+    unsigned long long key;   // (lowest thread whose run crosses the target) << 32 | the element it found
+    int lastpos;              // highest vector with positive weight
+    int result;               // the element found on the fallback path
 };
 
 }  // namespace svip

@@ -16,13 +16,26 @@ struct SegEntry {
     float A;
 };
 
-// Reads every segment entry of the cluster (warp-collective, run by warp 0 of each block), merges
-// them into the row's partial and selects the segment holding the mass u * Z.
-template <int kMode>
-__device__ __forceinline__ void combine_segments(cg::cluster_group& cluster, SegEntry* seg, int S,
-                                                 float c, float u, int lane, Partial& row,
-                                                 SegPick& pick, float abs_target = -1.f) {
-    const int nseg = S * kWarps;
+// Where the entries read by combine_segments live: `Remote` reads entry s from the block that
+// produced it, through distributed shared memory (the caller brackets this with cluster barriers);
+// `Local` reads a block-local table that the peers have filled (SegExchange below).
+struct RemoteSegments {
+    cg::cluster_group& cluster;
+    SegEntry* seg;
+    __device__ __forceinline__ SegEntry operator()(int s) const {
+        return cluster.map_shared_rank(seg, s / kWarps)[s % kWarps];
+    }
+};
+struct LocalSegments {
+    const SegEntry* all;
+    __device__ __forceinline__ SegEntry operator()(int s) const { return all[s]; }
+};
+
+// Merges the nseg segment entries of a row into the row's partial and selects the segment holding
+// the mass u * Z.  Warp-collective; every warp that runs it on the same entries gets the same bits.
+template <int kMode, class Source>
+__device__ __forceinline__ void combine_entries(const Source& src, int nseg, float c, float u, int lane,
+                                                Partial& row, SegPick& pick, float abs_target = -1.f) {
     const int per = (nseg + 31) / 32;
     Partial e[kSegPerLane];
     float m = neg_inf();
@@ -31,8 +44,7 @@ __device__ __forceinline__ void combine_segments(cg::cluster_group& cluster, Seg
         e[k].m = neg_inf(); e[k].idx = kIntMax; e[k].Z = 0.f; e[k].A = 0.f;
         int s = lane * per + k;
         if (k < per && s < nseg) {
-            const SegEntry* remote = cluster.map_shared_rank(seg, s / kWarps);
-            SegEntry v = remote[s % kWarps];
+            SegEntry v = src(s);
             e[k].m = v.m; e[k].idx = v.idx; e[k].Z = v.Z; e[k].A = v.A;
         }
         m = fmaxf(m, e[k].m);
@@ -55,65 +67,132 @@ __device__ __forceinline__ void combine_segments(cg::cluster_group& cluster, Seg
     row.Z = pick.total;
 }
 
-// Fine scan of one segment by the whole block.  `wf(vi, w)` yields the weights of the elements
-// of vector vi.  Each thread sums a run of consecutive vectors, one block scan places the runs,
-// and the thread whose run crosses `target` walks its run again element by element.  Returns the
-// virtual element index (vector * EPV + element) of the first element whose cumulative weight
-// exceeds `target`, else the last element with positive weight, else -1.
+// Reads every segment entry of the cluster through distributed shared memory (run by warp 0 of a
+// block, between two cluster barriers).
+template <int kMode>
+__device__ __forceinline__ void combine_segments(cg::cluster_group& cluster, SegEntry* seg, int S,
+                                                 float c, float u, int lane, Partial& row,
+                                                 SegPick& pick, float abs_target = -1.f) {
+    RemoteSegments src{cluster, seg};
+    combine_entries<kMode>(src, S * kWarps, c, u, lane, row, pick, abs_target);
+}
+
+// The segment entries of a row, pushed by the warps that produced them into every block of the
+// cluster (see the exchange primitives in svip_device.cuh).
+struct SegExchange {
+    SegEntry all[kMaxSeg];     // entry of segment s at index s
+    unsigned long long bar;    // mbarrier: completes when S * kWarps entries have landed here
+};
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+// To be run by every thread of every block of the cluster before the row is streamed.
+__device__ __forceinline__ void exchange_open(SegExchange& ex, int S, int tid) {
+    if (S == 1) return;
+    if (tid == 0) {
+        const uint32_t bar = smem_addr(&ex.bar);
+        mbar_init(bar, 1);
+        mbar_arrive_expect_tx(bar, static_cast<uint32_t>(S * kWarps * sizeof(SegEntry)));
+    }
+    cluster_arrive();   // a peer pushes only after its cluster_wait(), hence after this initialisation
+}
+
+// The calling warp publishes the entry of its segment (rank * kWarps + warp) to every block.
+__device__ __forceinline__ void exchange_push(SegExchange& ex, int S, int rank, int warp, int lane, const Partial& t) {
+    if (S == 1) {
+        if (lane == 0) { SegEntry& e = ex.all[warp]; e.m = t.m; e.idx = t.idx; e.Z = t.Z; e.A = t.A; }
+        return;
+    }
+    cluster_wait();
+    if (lane < S) {
+        const uint32_t dst = map_to_rank(smem_addr(&ex.all[rank * kWarps + warp]), lane);
+        const uint32_t bar = map_to_rank(smem_addr(&ex.bar), lane);
+        push16(dst, bar, __float_as_uint(t.m), static_cast<uint32_t>(t.idx), __float_as_uint(t.Z), __float_as_uint(t.A));
+    }
+}
+
+// Until all entries are here (S > 1; bounded): false if the wait ran out.
+__device__ __forceinline__ bool exchange_wait(SegExchange& ex) {
+    return mbar_wait_bounded(smem_addr(&ex.bar), 0);
+}
+
+// Fine scan of one segment by the whole block.  The functor splits into `load(vi)` (the raw 16-byte
+// vectors of element-vector vi) and `weights(vi, raw, w)` (their weights), so that a thread issues all
+// its loads at once and keeps them in registers.  Each thread sums a run of consecutive vectors, one
+// block scan places the runs, and in every warp the lowest lane whose run crosses `target` walks its
+// run again element by element; the lowest such thread of the block wins.  Returns the virtual
+// element index (vector * EPV + element) of the first element whose cumulative weight exceeds
+// `target`, else the last element with positive weight, else -1.  All threads return the same value.
 template <int EPV, class WF>
-__device__ __forceinline__ int fine_scan(WF& wf, int v_lo, int v_hi, float prefix, float target,
+__device__ __forceinline__ int fine_scan(const WF& wf, int v_lo, int v_hi, float prefix, float target,
                                          ScanShared& sh, int tid, int lane, int warp) {
     constexpr int kRun = 4;
+    constexpr unsigned long long kNone = ~0ull;
     const int nv = v_hi - v_lo;
     const int run = min(kRun, max(1, (nv + kThreads - 1) / kThreads));
-    if (tid == 0) { sh.hit = kIntMax; sh.lastpos = -1; sh.result = -1; }
+    if (tid == 0) { sh.key = kNone; sh.lastpos = -1; sh.result = -1; }
     float running = prefix;
     for (int cb = v_lo; cb < v_hi; cb += kThreads * run) {
         const int first = cb + tid * run;
+        typename WF::Raw raw[kRun];
+#pragma unroll
+        for (int k = 0; k < kRun; ++k)
+            if (k < run && first + k < v_hi) raw[k] = wf.load(first + k);
         float ls = 0.f;
         int lastv = -1;
-        for (int k = 0; k < run; ++k) {
-            int vi = first + k;
-            if (vi < v_hi) {
+#pragma unroll
+        for (int k = 0; k < kRun; ++k) {
+            if (k < run && first + k < v_hi) {
                 float w[EPV];
-                wf(vi, w);
+                wf.weights(first + k, raw[k], w);
                 float sv = 0.f;
 #pragma unroll
                 for (int j = 0; j < EPV; ++j) sv += w[j];
-                if (sv > 0.f) lastv = vi;
+                if (sv > 0.f) lastv = first + k;
                 ls += sv;
             }
         }
-        float total;
-        const float lo = running + block_scan_excl(ls, sh.wsum, lane, warp, total);
-        if (ls > 0.f && lo + ls > target) atomicMin(&sh.hit, tid);
-        if (lastv >= 0) atomicMax(&sh.lastpos, lastv);
+        const float inc = warp_scan_incl(ls, lane);
+        __syncthreads();   // wsum is free again; the initial key is visible
+        if (lane == 31) sh.wsum[warp] = inc;
         __syncthreads();
-        const int win = sh.hit;
-        if (win != kIntMax) {
-            if (tid == win) {
-                float cum = lo;
-                int res = -1, last = -1;
-                for (int k = 0; k < run; ++k) {
-                    int vi = first + k;
-                    if (vi < v_hi) {
-                        float w[EPV];
-                        wf(vi, w);
+        float before = 0.f, total = 0.f;
 #pragma unroll
-                        for (int j = 0; j < EPV; ++j) {
-                            cum += w[j];
-                            if (w[j] > 0.f) {
-                                last = vi * EPV + j;
-                                if (cum > target && res < 0) res = last;
-                            }
+        for (int w = 0; w < kWarps; ++w) {
+            const float sw = sh.wsum[w];
+            if (w < warp) before += sw;
+            total += sw;
+        }
+        const float lo = running + (before + (inc - ls));
+        const unsigned crossing = __ballot_sync(0xffffffffu, ls > 0.f && lo + ls > target);
+        if (crossing && lane == __ffs(crossing) - 1) {
+            float cum = lo;
+            int res = -1, last = -1;
+#pragma unroll
+            for (int k = 0; k < kRun; ++k) {
+                if (k < run && first + k < v_hi) {
+                    float w[EPV];
+                    wf.weights(first + k, raw[k], w);
+#pragma unroll
+                    for (int j = 0; j < EPV; ++j) {
+                        cum += w[j];
+                        if (w[j] > 0.f) {
+                            last = (first + k) * EPV + j;
+                            if (cum > target && res < 0) res = last;
                         }
                     }
                 }
-                sh.result = res >= 0 ? res : last;
             }
-            __syncthreads();
-            return sh.result;
+            atomicMin(&sh.key, (static_cast<unsigned long long>(tid) << 32) |
+                                   static_cast<unsigned>(res >= 0 ? res : last));
         }
+        const int lv = __reduce_max_sync(0xffffffffu, lastv);
+        if (lane == 0 && lv >= 0) atomicMax(&sh.lastpos, lv);
+        __syncthreads();
+        const unsigned long long key = sh.key;
+        if (key != kNone) return static_cast<int>(static_cast<unsigned>(key & 0xffffffffull));
         running += total;
     }
     // rounding left nothing above the target: the last element with weight
@@ -121,7 +200,7 @@ __device__ __forceinline__ int fine_scan(WF& wf, int v_lo, int v_hi, float prefi
     if (lv < 0) return -1;
     if (tid == 0) {
         float w[EPV];
-        wf(lv, w);
+        wf.weights(lv, wf.load(lv), w);
         int last = -1;
 #pragma unroll
         for (int j = 0; j < EPV; ++j)
@@ -161,10 +240,12 @@ struct SoftmaxWeights {
     RowGeom g;
     float c, M;
     float thr = -INFINITY;   // logits below it carry no weight (truncated distributions)
-    __device__ __forceinline__ void operator()(int vi, float (&w)[ElemTraits<DT>::kEPV]) const {
+    typedef uint4 Raw;
+    __device__ __forceinline__ Raw load(int vi) const { return g.base[vi]; }
+    __device__ __forceinline__ void weights(int vi, const Raw& raw, float (&w)[ElemTraits<DT>::kEPV]) const {
         constexpr int EPV = ElemTraits<DT>::kEPV;
         float x[EPV];
-        unpack_masked<DT>(g.base[vi], vi, g, x);
+        unpack_masked<DT>(raw, vi, g, x);
 #pragma unroll
         for (int j = 0; j < EPV; ++j)
             w[j] = x[j] >= thr ? ex2_approx(fmaxf(__fmaf_rn(x[j], c, -M), kArgFloor)) : 0.f;
@@ -176,33 +257,35 @@ struct RowShared {
     SegPick pick;
 };
 
-// The draft step of one row by the cluster that shares it: stream the row (Z, A, maximum), combine the
-// segment partials through distributed shared memory, write entropy / stop flag / normalisers, and
-// let the block that holds the sampled mass find the token.  `rp` / `g` describe the row, `thr` is
-// the truncation threshold when kThr.  Ends with the cluster barrier that keeps a block alive while
-// peers may still read its shared memory.
+// The draft step of one row by the cluster that shares it: stream the row (Z, A, maximum), push the
+// segment partials to every block of the cluster, combine them (every block the same bits), write
+// entropy / stop flag / normalisers, and let the block that holds the sampled mass find the token.
+// `g` describes the row, `thr` is the truncation threshold when kThr.  No block reads a peer's shared
+// memory, and a block leaves only after every entry aimed at it has landed.
 template <int DT, bool kGreedy, bool kPos, bool kThr>
 __device__ __forceinline__ void draft_row(const DraftArgs& a, cg::cluster_group& cluster, int S, int rank, int row,
                                           int tid, const RowGeom g, const uint32_t slot0, const long p, const float thr) {
     constexpr int EPV = ElemTraits<DT>::kEPV;
     const int lane = tid & 31, warp = tid >> 5;
-    __shared__ SegEntry seg[kWarps];
+    __shared__ SegExchange ex;
     __shared__ ScanShared scan;
     __shared__ RowShared res;
+    exchange_open(ex, S, tid);
     float u = 0.f, ext = -1.f;
     if (!kGreedy && warp == 0) {   // fetched now, used after the stream
         if (a.ext_target) ext = fmaxf(__ldg(a.ext_target + row), 0.f);
         else u = __ldg(a.uniforms + (row + p * a.slot_stride));
     }
     Partial t = reduce_segment<DT, 2, kGreedy, kThr>(g, rank * kWarps + warp, a.c, lane, slot0, thr);
-    if (lane == 0) { seg[warp].m = t.m; seg[warp].idx = t.idx; seg[warp].Z = t.Z; seg[warp].A = t.A; }
-    cluster.sync();
+    exchange_push(ex, S, rank, warp, lane, t);
+    if (S == 1) __syncthreads();
     if (warp == 0) {
+        if (S > 1 && !exchange_wait(ex) && lane == 0) atomicOr(a.status, SVIP_STATUS_WAIT_TIMEOUT);
         Partial r; SegPick pk;
-        combine_segments<2>(cluster, seg, S, a.c, u, lane, r, pk, ext);
+        LocalSegments src{ex.all};
+        combine_entries<2>(src, S * kWarps, a.c, u, lane, r, pk, ext);
         if (lane == 0) { res.row = r; res.pick = pk; }
     }
-    cluster_arrive();   // done with the peers' shared memory
     __syncthreads();    // res is visible block-wide
     const Partial R = res.row;
     const SegPick P = res.pick;
@@ -227,7 +310,6 @@ __device__ __forceinline__ void draft_row(const DraftArgs& a, cg::cluster_group&
         int virt = fine_scan<EPV>(wf, v_lo, v_hi, P.prefix, P.target, scan, tid, lane, warp);
         if (tid == 0) a.token[slot] = (virt >= 0 ? virt - g.pre : 0) + a.token_offset;
     }
-    cluster_wait();     // no block leaves while a peer may still read its shared memory
 }
 
 // kBlocks is the number of blocks the register budget must leave room for on one SM: 2 for

@@ -35,17 +35,27 @@ struct ResidualWeights {
     float c, Mp, rZp, Mq, rZq;
     int bonus;
     float thr_p = -INFINITY, thr_q = -INFINITY;   // truncated distributions: logits below carry nothing
+    struct Raw { uint4 t, q; };
+    __device__ __forceinline__ Raw load(int vi) const {
+        Raw r;
+        r.t = __ldg(gt.base + vi);
+        r.q = (!bonus && gq.pre == gt.pre) ? __ldg(gq.base + vi) : make_uint4(0, 0, 0, 0);
+        return r;
+    }
     __device__ __forceinline__ void operator()(int vi, float (&w)[ElemTraits<DT>::kEPV]) const {
+        weights(vi, load(vi), w);
+    }
+    __device__ __forceinline__ void weights(int vi, const Raw& raw, float (&w)[ElemTraits<DT>::kEPV]) const {
         constexpr int EPV = ElemTraits<DT>::kEPV;
         float x[EPV];
-        unpack_masked<DT>(__ldg(gt.base + vi), vi, gt, x);
+        unpack_masked<DT>(raw.t, vi, gt, x);
 #pragma unroll
         for (int j = 0; j < EPV; ++j)
             w[j] = x[j] >= thr_p ? ex2_approx(fmaxf(__fmaf_rn(x[j], c, -Mp), kArgFloor)) * rZp : 0.f;
         if (bonus) return;
         float d[EPV];
         if (gq.pre == gt.pre) {
-            unpack_masked<DT>(__ldg(gq.base + vi), vi, gq, d);
+            unpack_masked<DT>(raw.q, vi, gq, d);
         } else {
             // rows with different 16-byte phase: element loads
 #pragma unroll
