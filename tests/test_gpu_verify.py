@@ -236,3 +236,97 @@ def test_accept_ratio_of_very_unlikely_tokens(ctx, oracle, bf16):
     probs = np.array([a[0] for a in ap])
     assert (probs < 0.9).sum() > 5 and (probs >= 1.0).sum() > 5            # both outcomes are exercised
     assert 0 < n_o.sum() < B
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_draft_token_outside_the_draft_support(ctx, oracle, bf16):
+    """A draft token whose own draft logit is -inf while the target's is finite: q(x) = 0 < p(x), the
+    ratio of Algorithm 2 is +inf and every draw accepts, also the largest one.  With the target logit
+    at -inf too there is nothing to accept: rejected whatever the draw."""
+    rng = np.random.default_rng(515 + int(bf16))
+    B, V, K, T = 6, 3001, 3, 0.9
+    lens, cu, q, tgt, ud, uv = small_case(rng, B, V, K, False, ragged=False)
+    tok, _, _ = oracle.draft_step(q, T, 0.3, ud)
+    tok = tok.astype(np.int32)
+    # position 1 of every sequence: the draft model excludes its own token
+    for i in range(B):
+        r = int(cu[i]) - i + 1
+        x = int(rng.integers(0, V))
+        tok[r] = x
+        q[r, x] = -np.inf
+        tgt[cu[i] + 1, x] = rng.standard_normal() if i % 2 == 0 else -np.inf
+    if bf16:
+        q = W.to_bf16_bits(q); tgt = W.to_bf16_bits(tgt)
+    uv = uv.copy()
+    uv, _ = tl.guard_accept_uniforms(oracle, tok, q, tgt, cu, T, uv)
+    uv[cu[:-1]] = 0.0                            # position 0 accepted (p(x) > 0 for a token drawn from q)
+    uv[cu[:-1] + 1] = 1.0 - 2.0 ** -24           # the hardest draw at the position under test
+    for S in (0, 1, 4):
+        ctx.set_cluster_size(S)
+        try:
+            for with_stats in (False, True):
+                stats = tl.gpu_draft_step(ctx, q, T, 0.3, ud)[3] if with_stats else None
+                got = tl.gpu_verify(ctx, tok, q, tgt, cu, K, T, uv, q_stats=stats, fixed_K=True)
+                tl.check_verify_against_oracle(oracle, tok, q, tgt, cu, T, uv, got, "q(x)=0 S=%d" % S)
+                assert np.all(got[0][0::2] >= 2), got[0]      # q(x) = 0 < p(x): accepted
+                assert np.all(got[0][1::2] == 1), got[0]      # q(x) = 0 = p(x): rejected
+        finally:
+            ctx.set_cluster_size(0)
+    assert ctx.read_status() == 0
+
+
+def _nearly_equal_pair(rng, V, q_of_x):
+    """A draft row and a target row that differ in ONE logit, the target's one unit in the last place
+    lower, at a token of draft probability about q_of_x: p(x)/q(x) = 1 - 2e-6, so the largest draw
+    rejects, and max(0, p - q) is carried by the normalisers' difference alone (about 2e-6 * q(x))."""
+    d = (rng.standard_normal(V) * 1.5).astype(np.float32)
+    x = int(rng.integers(0, V))
+    Z = np.exp(d.astype(np.float64) - d.max()).sum()
+    d[x] = np.float32(d.max() + np.log(q_of_x * Z))
+    if not 16.0 <= abs(d[x]) < 32.0:                        # one unit in the last place = 1.9e-6 there
+        shift = np.float32((-24.0 if d[x] < 0 else 24.0) - d[x])
+        d = (d + shift).astype(np.float32)
+    t = d.copy()
+    t[x] = np.nextafter(d[x], np.float32(-np.inf))
+    return d, t, x
+
+
+def test_rejection_with_a_residual_below_fp32_resolution(ctx, oracle):
+    """Algorithm 4 when p and q agree to the last place.  After a rejection max(0, p - q) has mass in exact
+    arithmetic, but it can vanish in the arithmetic that computes it; the correction token is then drawn
+    from p (p and q are indistinguishable there).  Two families:
+      (a) the differing token is so unlikely (1e-11) that even the fp64 normalisers coincide: oracle and
+          GPU both see a zero residual and both sample from p: full parity;
+      (b) the differing token has probability 1e-3 .. 1e-5: the fp64 residual has mass ~1e-9..1e-11, the
+          fp32 one is zero or rounding noise: only what is unique is compared (the rejection itself, a
+          token the target gives weight, a clear status word)."""
+    rng = np.random.default_rng(99)
+    V, T = 8192, 1.0
+    top = np.float32(1.0 - 2.0 ** -24)
+    n_a = n_b_zero64 = 0
+    for case, q_of_x in enumerate((1e-11, 1e-11, 1e-11, 1e-3, 1e-4, 1e-5, 1e-3, 1e-4)):
+        d, t, x = _nearly_equal_pair(rng, V, q_of_x)
+        q_rows = d[None, :]
+        t_rows = np.stack([t, (rng.standard_normal(V)).astype(np.float32)])
+        cu = np.array([0, 2], dtype=np.int64)
+        tok = np.array([x], dtype=np.int32)
+        p64 = oracle.softmax(t_rows[0], T); q64 = oracle.softmax(q_rows[0], T)
+        _, S64 = oracle.residual(p64, q64)
+        for u in (0.0, 0.37, 0.93):
+            uv = np.array([top, u], dtype=np.float32)
+            n_o, nx_o, ap = oracle.verify(tok, q_rows, t_rows, cu, T, uv.astype(np.float64), want_accept_prob=True)
+            assert n_o[0] == 0 and ap[0][0] < float(top)             # the oracle rejects
+            for S in (0, 1, 2):
+                ctx.set_cluster_size(S)
+                try:
+                    got = tl.gpu_verify(ctx, tok, q_rows, t_rows, cu, 1, T, uv, fixed_K=True)
+                finally:
+                    ctx.set_cluster_size(0)
+                assert got[0][0] == 0, "the GPU must reject as well (case %d)" % case
+                assert 0 <= got[1][0] < V and p64[got[1][0]] > 0.0
+                if S64 == 0.0:        # family (a): both sides fall back to p
+                    tl.check_verify_against_oracle(oracle, tok, q_rows, t_rows, cu, T, uv, got, "zero residual")
+                    n_a += 1
+        n_b_zero64 += int(S64 == 0.0)
+    assert n_a >= 9 and n_b_zero64 <= 5      # both families occurred
+    assert ctx.read_status() == 0

@@ -200,6 +200,37 @@ def test_zero_target_probability_always_rejects(oracle):
         assert n == 0 and a[0] == 0.0 and nx != 2
 
 
+def test_token_outside_draft_support_is_accepted_iff_target_has_it(oracle):
+    """q(x) = 0 < p(x): the ratio of Algorithm 2 is +inf, so min(1, p/q) = 1 and every r in [0,1)
+    accepts (the limit of p/q as q -> 0+ shows it: the acceptance probability rises to 1 and stays).
+    q(x) = 0 = p(x): nothing to accept, rejected for every r."""
+    V = 6
+    top = 1.0 - 2.0 ** -24
+    t_rows = np.zeros((2, V), dtype=np.float32)
+    t_rows[0] = [0.3, -1.0, 0.5, 0.0, 2.0, -0.7]
+    for x in range(V):
+        q_rows = np.array([[0.1, 0.2, -0.4, 1.0, 0.0, 0.6]], dtype=np.float32)
+        q_rows[0, x] = -np.inf
+        for r_val in (0.0, 0.5, top):
+            n, nx, a = _verify_one(oracle, [x], q_rows, t_rows, 1.0, [r_val, 0.5])
+            assert a[0] == 1.0 and n == 1
+            assert nx == oracle.invcdf(oracle.softmax(t_rows[1], 1.0), 0.5)
+        # the limit: the draft logit of x sinks, the acceptance probability rises to 1 and stays there
+        last = 0.0
+        for lx in (0.0, -5.0, -20.0, -80.0, -700.0, -1e30):
+            q_rows[0, x] = lx
+            _, _, a = _verify_one(oracle, [x], q_rows, t_rows, 1.0, [0.0, 0.5])
+            assert a[0] >= last
+            last = a[0]
+        assert last == 1.0
+        # both models exclude x: rejected whatever the draw, and the correction avoids x
+        q_rows[0, x] = -np.inf
+        t2 = t_rows.copy(); t2[0, x] = -np.inf
+        for r_val in (0.0, top):
+            n, nx, a = _verify_one(oracle, [x], q_rows, t2, 1.0, [r_val, 0.5])
+            assert a[0] == 0.0 and n == 0 and nx != x
+
+
 def test_accept_probability_is_min_one_ratio(oracle):
     rng = np.random.default_rng(8)
     V = 12

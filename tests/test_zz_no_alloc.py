@@ -6,11 +6,13 @@ such callers can neither cudaMalloc nor create an svip context (creating one all
 workspace).  The entry point under test takes no context and keeps its workspace in a fixed array
 inside the library.  Here it must agree with svip_verify -- same accept counts and same next
 tokens, bit for bit, since both run the same kernels on the same inputs -- on two calls in a row
-(the second call reuses the array that the first one filled), and refuse more rows than the array
-holds.  This file sorts last so that a run stopping at the first failure has run everything else.
+(the second call reuses the array that the first one filled), agree with the fp64 oracle within the
+tolerances of the other parity tests, and refuse more rows than the array holds.  This file sorts last so that a run stopping at the first failure has run everything else.
 """
 import numpy as np
 import pytest
+
+import svip_testlib as tl
 
 pytestmark = pytest.mark.gpu
 
@@ -34,7 +36,7 @@ def _case(rng, B, V, K_max, bf16):
     return lens, cu, q, tgt, tokens, rng.random(Rp).astype(np.float32)
 
 
-def test_noalloc_matches_verify_on_two_calls_in_a_row():
+def test_noalloc_matches_verify_on_two_calls_in_a_row(oracle):
     import torch
     from paper_2411_18462_b200 import Context, build, verify_noalloc, SvipError
     build.build()
@@ -46,6 +48,8 @@ def test_noalloc_matches_verify_on_two_calls_in_a_row():
     for B, V, K_max, bf16, T in ((24, 9000, 7, True, 1.0), (5, 4099, 3, False, 0.7), (9, 1000, 4, True, 0.0)):
         lens, cu, q, tgt, tokens, u = _case(rng, B, V, K_max, bf16)
         Rp = int(cu[-1])
+        # accept draws off the decision boundary (oracle values), as in the other parity tests
+        u, _ = tl.guard_accept_uniforms(oracle, tokens, q, tgt, cu, T, u)
         d_tok, d_q, d_t, d_cu, d_u = dev(tokens), dev(q), dev(tgt), dev(cu), dev(u)
         out = [torch.full((B,), -5, dtype=torch.int32, device="cuda") for _ in range(4)]
         status = torch.full((1,), 77, dtype=torch.int32, device="cuda")
@@ -62,6 +66,9 @@ def test_noalloc_matches_verify_on_two_calls_in_a_row():
         verify_noalloc(0, d_tok, d_q, V, None, -1, 0, d_t, V, dt, d_cu, B, K_max, Rp, V, T, d_u, out[2], out[3])
         torch.cuda.synchronize()
         assert torch.equal(out[0], out[2]) and torch.equal(out[1], out[3])
+        # and against the oracle, like svip_verify itself
+        tl.check_verify_against_oracle(oracle, tokens, q, tgt, cu, T, u, (out[2].cpu().numpy(), out[3].cpu().numpy()),
+                                       "noalloc B=%d V=%d T=%g" % (B, V, T))
     # more rows than the fixed array holds: a clear error, nothing launched
     with pytest.raises(SvipError) as e:
         verify_noalloc(0, d_tok, d_q, V, None, -1, 0, d_t, V, dt, None, 8193, 1, 2 * 8193, V, 1.0, d_u, out[2], out[3])
