@@ -117,7 +117,7 @@ class Round:
         self.ctx, self.w, self.torch, self.stream = ctx, w, torch, stream
         order, q_pm, active = workloads.position_major(w)
         B, V, K = w.B, w.V, q_pm.shape[0]
-        self.B, self.V, self.K, self.active = B, V, K, active
+        self.B, self.V, self.K, self.active, self.order = B, V, K, active, order
         lens = w.draft_len[order].astype(np.int32)
         cu_sorted = np.concatenate([[0], np.cumsum(lens.astype(np.int64) + 1)])
         t_sorted = np.empty_like(w.target_logits)
@@ -219,6 +219,24 @@ class Round:
         rejected = int((nacc < self.lens).sum())
         rows = int(self.lens.sum()) + self.Rp + rejected
         return rows * self.V * self.esz, rejected
+
+    def results_by_sequence(self):
+        """The last step's outputs in the workload's own indexing: per packed draft row (token, entropy,
+        stop flag) and per sequence (n_accepted, next_token)."""
+        self.torch.cuda.synchronize()
+        w, B = self.w, self.B
+        tok = self.d_tok.cpu().numpy().reshape(self.K, B); ent = self.d_ent.cpu().numpy().reshape(self.K, B)
+        stop = self.d_stop.cpu().numpy().reshape(self.K, B)
+        nacc = self.d_nacc.cpu().numpy(); nxt = self.d_next.cpu().numpy()
+        out = {"token": np.zeros(w.n_draft_rows, np.int64), "entropy": np.zeros(w.n_draft_rows),
+               "stop": np.zeros(w.n_draft_rows, np.uint8), "n_accepted": np.zeros(B, np.int64),
+               "next_token": np.zeros(B, np.int64)}
+        for k, i in enumerate(self.order):
+            n = int(self.lens[k]); r0 = int(w.cu_rows[i]) - int(i)
+            out["token"][r0:r0 + n] = tok[:n, k]; out["entropy"][r0:r0 + n] = ent[:n, k]
+            out["stop"][r0:r0 + n] = stop[:n, k]
+            out["n_accepted"][i] = nacc[k]; out["next_token"][i] = nxt[k]
+        return out
 
     def check_stop_flags(self):
         """The stop rule must reproduce the workload's draft lengths (generator contract)."""
@@ -401,40 +419,257 @@ def truncated_round(ctx, torch, rnd, top_k=50, top_p=0.9, reps=10):
     return out
 
 
-def cpu_baseline(w, seconds_budget=20.0):
-    """The fp64 oracle, as it stands, on a bounded sample of the same workload, on all host cores."""
-    from oracle import svip_oracle as O
-    cores = len(os.sched_getaffinity(0))
-    # about 4500 rows: 10-20 s of CPU work
-    rows_per_seq = 2.0 * float(w.draft_len.mean()) + 1.0
-    n_seq = min(w.B, max(64, int(round(4500.0 / rows_per_seq))))
+def pair_stats_leg(ctx, torch, rnd, peak, reps=10):
+    """svip_pair_stats over every (draft row, target row under it) pair of the round, on contiguous copies of
+    the resident rows (gathered outside the timed region).  Algorithmic bytes: both rows of a pair once."""
+    w, B, V = rnd.w, rnd.B, rnd.V
+    if not w.T > 0:
+        return None
+    dev = rnd.d_q.device
+    cu = np.concatenate([[0], np.cumsum(rnd.lens.astype(np.int64) + 1)])
+    q_idx = np.concatenate([np.arange(rnd.lens[k]) * B + k for k in range(B)])
+    t_idx = np.concatenate([cu[k] + np.arange(rnd.lens[k]) for k in range(B)])
+    n = int(q_idx.size)
+    q = rnd.d_q.index_select(0, torch.from_numpy(q_idx).to(dev))
+    t = rnd.d_t.index_select(0, torch.from_numpy(t_idx).to(dev))
+    out = torch.zeros(n, 8, device=dev)
+    call = ctx.bind("pair_stats", q, V, t, V, rnd.dt, n, V, w.T, 0.18, out, rnd.stream)
+    call()
+    torch.cuda.synchronize()
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    us = 1000.0 * e0.elapsed_time(e1) / reps
+    nbytes = 2 * n * V * rnd.esz
+    res = out.cpu().numpy()
+    return {"pairs": n, "us_per_call": us, "algorithmic_bytes": nbytes, "GBps": nbytes / (us * 1e-6) / 1e9,
+            "frac_of_measured_peak": nbytes / (us * 1e-6) / 1e9 / peak,
+            "mean_beta": float(res[:, 0].mean()), "mean_H_q": float(res[:, 1].mean()),
+            "non_finite_outputs": int((~np.isfinite(res)).sum())}
+
+
+CDF_TOL = 1e-5        # a sampled token may differ from the oracle's only across a CDF boundary closer than this
+ACCEPT_GUARD = 1e-4   # an accept decision may differ only if the draw is this close to the acceptance probability
+STOP_GUARD = 1e-3     # a stop flag may differ only if sqrt(H) is this close to h
+ENTROPY_ATOL = 1e-4
+
+
+def _within_cdf_tolerance(weights, u, token):
+    c = np.cumsum(np.asarray(weights, dtype=np.float64))
+    total = c[-1]
+    if not total > 0 or not (0 <= token < len(c)) or not weights[token] > 0:
+        return False
+    lo = (c[token - 1] if token > 0 else 0.0) / total
+    return bool(lo - CDF_TOL <= float(u) <= c[token] / total + CDF_TOL)
+
+
+def _oracle_sample(w, n_seq):
+    """The first n_seq sequences of the workload as packed arrays of their own."""
     sel = list(range(n_seq))
     rows_q = np.concatenate([np.arange(w.cu_rows[i] - i, w.cu_rows[i] - i + w.draft_len[i]) for i in sel])
     rows_t = np.concatenate([np.arange(w.cu_rows[i], w.cu_rows[i + 1]) for i in sel])
-    q = np.ascontiguousarray(w.q_logits[rows_q]); t = np.ascontiguousarray(w.target_logits[rows_t])
     lens = w.draft_len[sel]
     cu = np.concatenate([[0], np.cumsum(lens.astype(np.int64) + 1)])
-    ud = w.draft_uniforms[rows_q]; uv = w.verify_uniforms[rows_t]
-    O.lib()
+    return {"rows_q": rows_q, "rows_t": rows_t, "lens": lens, "cu": cu,
+            "q": np.ascontiguousarray(w.q_logits[rows_q]), "t": np.ascontiguousarray(w.target_logits[rows_t]),
+            "ud": w.draft_uniforms[rows_q], "uv": w.verify_uniforms[rows_t]}
+
+
+def _oracle_pass(O, w, s, threads):
+    """One pass of the oracle over a sample: every draft row, then the verification round.  Returns
+    (seconds, algorithmic bytes, results)."""
     t0 = time.perf_counter()
-    tok, H, stop = O.draft_step(q, w.T, w.h, ud, threads=cores)
-    nacc, nxt, _ = O.verify(tok.astype(np.int32), q, t, cu, w.T, uv, threads=cores)
+    tok, H, stop = O.draft_step(s["q"], w.T, w.h, s["ud"], threads=threads)
+    nacc, nxt, _ = O.verify(tok.astype(np.int32), s["q"], s["t"], s["cu"], w.T, s["uv"], threads=threads)
     dt = time.perf_counter() - t0
-    rejected = int((nacc < lens).sum())
-    nbytes = (len(rows_q) + len(rows_t) + rejected) * w.V * w.elem_bytes
+    rejected = int((nacc < s["lens"]).sum())
+    nbytes = (len(s["rows_q"]) + len(s["rows_t"]) + rejected) * w.V * w.elem_bytes
+    return dt, nbytes, (tok, H, stop, nacc, nxt)
+
+
+def _boundary_checks(O, w, s, oracle_out, gpu, threads):
+    """Untimed comparison of the GPU's last step with the oracle on the sample: how many results are identical
+    and how many of the others fall inside the stated tolerances (and are therefore allowed to differ)."""
+    tok, H, stop, nacc, nxt = oracle_out
+    rq = s["rows_q"]
+    g_tok, g_H, g_stop = gpu["token"][rq], gpu["entropy"][rq], gpu["stop"][rq]
+    out = {"draft_rows": int(len(rq)), "sequences": int(len(s["lens"]))}
+    out["entropy_max_abs_err"] = float(np.max(np.abs(g_H - H)))
+    near = np.abs(np.sqrt(H) - w.h) <= STOP_GUARD
+    out["stop_near_threshold"] = int(near.sum())
+    out["stop_flags_wrong"] = int((g_stop[~near] != stop[~near]).sum())
+    bad = np.nonzero(g_tok != tok)[0]
+    out["draft_tokens_identical"] = int(len(rq) - bad.size)
+    tb = beyond = 0
+    for r in bad:
+        if w.T > 0 and _within_cdf_tolerance(O.softmax(s["q"][r], w.T), s["ud"][r], int(g_tok[r])):
+            tb += 1
+        else:
+            beyond += 1
+    out["token_boundary"] = tb
+    out["draft_tokens_beyond_tolerance"] = beyond
+    # verification: only sequences whose draft tokens are the oracle's can be compared
+    cu, lens = s["cu"], s["lens"]
+    same_draft = np.array([np.array_equal(g_tok[cu[i] - i: cu[i] - i + lens[i]], tok[cu[i] - i: cu[i] - i + lens[i]])
+                           for i in range(len(lens))])
+    out["sequences_not_compared"] = int((~same_draft).sum())
+    inside = wrong = n_same = nx_same = nx_boundary = nx_beyond = 0
+    guard_draws = 0
+    aprob = None
+    if w.T > 0:
+        _, _, aprob = O.verify(tok.astype(np.int32), s["q"], s["t"], cu, w.T, s["uv"], want_accept_prob=True,
+                               threads=threads)
+        for i, a in enumerate(aprob):
+            r = s["uv"][cu[i]: cu[i] + lens[i]].astype(np.float64)
+            guard_draws += int(((np.abs(r - a) < ACCEPT_GUARD) & (a < 1.0)).sum())
+    for i in np.nonzero(same_draft)[0]:
+        gn, gx = int(gpu["n_accepted"][i]), int(gpu["next_token"][i])
+        if gn != nacc[i]:
+            j = min(gn, int(nacc[i]))
+            ok = aprob is not None and abs(float(s["uv"][cu[i] + j]) - aprob[i][j]) < ACCEPT_GUARD
+            inside += int(ok); wrong += int(not ok)
+            continue
+        n_same += 1
+        if gx == nxt[i]:
+            nx_same += 1
+            continue
+        ok = False
+        if w.T > 0:
+            p = O.softmax(s["t"][cu[i] + nacc[i]], w.T)
+            wts = p
+            if nacc[i] < lens[i]:
+                wts, S = O.residual(p, O.softmax(s["q"][cu[i] - i + nacc[i]], w.T))
+                if not S > 0:
+                    wts = p
+            ok = _within_cdf_tolerance(wts, s["uv"][cu[i] + lens[i]], gx)
+        nx_boundary += int(ok); nx_beyond += int(not ok)
+    out.update({"accept_draws_inside_guard": guard_draws, "n_accepted_identical": n_same,
+                "n_accepted_decided_inside_guard": inside, "n_accepted_wrong": wrong,
+                "next_identical": nx_same, "next_boundary": nx_boundary, "next_beyond_tolerance": nx_beyond})
+    out["tolerances"] = {"entropy_abs": ENTROPY_ATOL, "cdf": CDF_TOL, "accept_guard": ACCEPT_GUARD, "stop_guard": STOP_GUARD}
+    out["ok"] = bool(out["entropy_max_abs_err"] <= ENTROPY_ATOL and out["stop_flags_wrong"] == 0 and beyond == 0
+                     and wrong == 0 and nx_beyond == 0)
+    return out
+
+
+def cpu_baseline(w, gpu_results=None, passes=3):
+    """The fp64 oracle, as it stands, on a bounded sample of the same workload, on all host cores: median of
+    `passes` passes.  With the GPU's results of the same sequences, an untimed comparison follows (`checks`:
+    identical results and boundary cases, counted)."""
+    from oracle import svip_oracle as O
+    cores = len(os.sched_getaffinity(0))
+    # about 4500 rows: a few seconds of CPU work per pass
+    rows_per_seq = 2.0 * float(w.draft_len.mean()) + 1.0
+    n_seq = min(w.B, max(64, int(round(4500.0 / rows_per_seq))))
+    s = _oracle_sample(w, n_seq)
+    O.lib()
+    runs = [_oracle_pass(O, w, s, cores) for _ in range(passes)]
+    runs.sort(key=lambda r: r[0])
+    dt, nbytes, res = runs[len(runs) // 2]
+    n_rows = len(s["rows_q"]) + len(s["rows_t"])
     # the same on one thread, over a sixteenth of the sample (whole sequences)
     n1 = max(1, n_seq // 16)
-    q1 = int(lens[:n1].sum()); t1 = int(cu[n1])
-    t0 = time.perf_counter()
-    tok1, _, _ = O.draft_step(q[:q1], w.T, w.h, ud[:q1], threads=1)
-    nacc1, _, _ = O.verify(tok1.astype(np.int32), q[:q1], t[:t1], cu[:n1 + 1], w.T, uv[:t1], threads=1)
-    dt1 = time.perf_counter() - t0
-    bytes1 = (q1 + t1 + int((nacc1 < lens[:n1]).sum())) * w.V * w.elem_bytes
-    return {"value": nbytes / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
-            "sample": "%d of %d sequences (%d draft + %d target rows), one pass, %.1f s" % (
-                n_seq, w.B, len(rows_q), len(rows_t), dt),
-            "single_thread_value": bytes1 / dt1 / 1e9,
-            "single_thread_sample": "%d sequences (%d rows), %.1f s" % (n1, q1 + t1, dt1)}
+    s1 = _oracle_sample(w, n1)
+    dt1, bytes1, _ = _oracle_pass(O, w, s1, 1)
+    out = {"value": nbytes / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
+           "sample": "%d of %d sequences (%d draft + %d target rows), median of %d passes, %.2f s per pass" % (
+               n_seq, w.B, len(s["rows_q"]), len(s["rows_t"]), passes, dt),
+           "rows_per_s": n_rows / dt, "us_per_step": 1e6 * dt * (w.B / n_seq),
+           "us_per_step_note": "one pass scaled to the whole batch (%d sequences)" % w.B,
+           "single_thread_value": bytes1 / dt1 / 1e9,
+           "single_thread_sample": "%d sequences (%d rows), one pass, %.1f s" % (
+               n1, len(s1["rows_q"]) + len(s1["rows_t"]), dt1)}
+    checks = _boundary_checks(O, w, s, res, gpu_results, cores) if gpu_results is not None else None
+    return out, checks
+
+
+# --------------------------------------------------------------------------- timing one workload
+
+def measure(ctx, torch, dist, world, rnd, steps, warmup):
+    """`warmup` untimed rounds, then `steps` timed ones (CUDA events on the launching stream, barrier and
+    synchronize on both sides).  The row-statistics kernel is timed by the library's event pair around its
+    launch, the draft-step kernel as the mean over the draft launches of a round."""
+    stream = torch.cuda.current_stream()
+    for _ in range(warmup):
+        rnd.step()
+    step_bytes, rejected = rnd.logits_bytes()
+    stops_ok = rnd.check_stop_flags()
+    status = ctx.read_status(stream.cuda_stream)
+    ctx.profile_enable(True)
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    n_timed = min(steps, 1024)
+    draft_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_timed)]
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    launches0 = ctx.launch_count()
+    e0.record(stream)
+    for k in range(steps):
+        rnd.step(draft_ev[k] if k < n_timed else None)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    m = {"steps": steps, "step_bytes": step_bytes, "rejected": rejected, "stops_ok": stops_ok, "status": status,
+         "launches": ctx.launch_count() - launches0, "local_ms": e0.elapsed_time(e1), "n_timed": n_timed,
+         "draft_ms": sum(a.elapsed_time(b) for a, b in draft_ev)}
+    m["stats_ms"], m["stats_n"] = ctx.profile_read()
+    ctx.profile_enable(False)
+    return m
+
+
+def rooflines(w, rnd, m, total_ms, peak, peak_kind):
+    """The two streaming kernels against the HBM roofline; the one with the larger share of the step first."""
+    steps = m["steps"]
+    stats_bytes = w.n_target_rows * w.V * w.elem_bytes
+    stats_n, stats_ms = m["stats_n"], m["stats_ms"]
+    stats_gbs = stats_bytes / (stats_ms / max(stats_n, 1) * 1e-3) / 1e9 if stats_n else None
+    n_draft = rnd.K
+    draft_bytes = w.n_draft_rows * w.V * w.elem_bytes / n_draft
+    draft_us = m["draft_ms"] * 1e3 / max(m["n_timed"] * n_draft, 1)
+    draft_gbs = draft_bytes / (draft_us * 1e-6) / 1e9
+    dt_name = "bf16" if w.dtype == "bf16" else "f32"
+    mode = "sampling" if w.T > 0 else "greedy"
+    roof_stats = {"bound": "hbm", "kernel": "row_stats_kernel<%s> (target rows of svip_verify)" % dt_name,
+                  "achieved": stats_gbs, "peak": peak, "peak_kind": "%s copy bandwidth" % peak_kind, "unit": "GB/s",
+                  "frac": (stats_gbs / peak) if stats_gbs else None, "launches_timed": stats_n,
+                  "bytes_per_launch": stats_bytes, "us_per_launch": stats_ms * 1e3 / max(stats_n, 1),
+                  "share_of_step": stats_ms / max(stats_n, 1) / (total_ms / steps),
+                  "traffic": ROW_STATS_TRAFFIC_PER_ALGORITHMIC_BYTE * stats_bytes
+                  if (w.dtype == "bf16" and ROW_STATS_TRAFFIC_PER_ALGORITHMIC_BYTE) else None}
+    roof_draft = {"bound": "hbm", "kernel": "draft_step_kernel<%s, %s> (mean over the %d launches of a round)"
+                  % (dt_name, mode, n_draft), "achieved": draft_gbs, "peak": peak,
+                  "peak_kind": "%s copy bandwidth" % peak_kind, "unit": "GB/s", "frac": draft_gbs / peak,
+                  "launches_timed": m["n_timed"] * n_draft, "bytes_per_launch": draft_bytes, "us_per_launch": draft_us,
+                  "share_of_step": m["draft_ms"] / m["n_timed"] / (total_ms / steps),
+                  "traffic": DRAFT_F32_TRAFFIC_PER_ALGORITHMIC_BYTE * draft_bytes
+                  if (w.dtype == "f32" and DRAFT_F32_TRAFFIC_PER_ALGORITHMIC_BYTE) else None}
+    return (roof_draft, roof_stats) if roof_draft["share_of_step"] >= roof_stats["share_of_step"] \
+        else (roof_stats, roof_draft)
+
+
+def other_workload(ctx, torch, name, rank, peak, peak_kind, steps):
+    """A short timed run of another published configuration on the same GPU (kept small: a few hundred ms)."""
+    spec = workloads.SPECS[name]
+    w = workloads.make_workload(name, seed=sharding.rank_seed(workloads.BASE_SEED + spec["index"], rank))
+    rnd = Round(ctx, w, torch, torch.cuda.current_stream().cuda_stream)
+    m = measure(ctx, torch, None, 1, rnd, steps, 3)
+    ms = m["local_ms"]
+    first, second = rooflines(w, rnd, m, ms, peak, peak_kind)
+    keep = ("kernel", "achieved", "frac", "us_per_launch", "bytes_per_launch", "share_of_step", "launches_timed")
+    out = {"workload": describe(w), "dtype": w.dtype, "steps": steps, "us_per_step": 1e3 * ms / steps,
+           "logits_GBps": m["step_bytes"] * steps / (ms * 1e-3) / 1e9,
+           "frac_of_measured_peak": m["step_bytes"] * steps / (ms * 1e-3) / 1e9 / peak,
+           "kernels_per_step": m["launches"] // steps, "rejected_sequences": m["rejected"],
+           "stop_flags_match_draft_lengths": bool(m["stops_ok"]) if name == "ragged" else None,
+           "status_word": m["status"],
+           "roofline": {k: first[k] for k in keep}, "roofline_other": {k: second[k] for k in keep}}
+    del rnd
+    torch.cuda.empty_cache()
+    return out
 
 
 def run_ours(args):
@@ -457,38 +692,16 @@ def run_ours(args):
     ctx = Context(dev, max(1 << 14, w.n_target_rows))
     stream = torch.cuda.current_stream()
     rnd = Round(ctx, w, torch, stream.cuda_stream)
-    for _ in range(max(args.warmup, 3)):
-        rnd.step()
-    step_bytes, rejected = rnd.logits_bytes()
-    stops_ok = rnd.check_stop_flags()
-    status = ctx.read_status(stream.cuda_stream)
+    warmup = max(args.warmup, 3)
 
+    # the clocks are sampled from before the warm-up until the end-to-end leg is over
     uuid = str(torch.cuda.get_device_properties(dev).uuid)
     uuid = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
     sampler = ClockSampler(uuid)
-    ctx.profile_enable(True)
-    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize()
     sampler.start()
-    launches0 = ctx.launch_count()
-    n_timed = min(args.steps, 1024)
-    draft_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_timed)]
-    e0.record(stream)
-    for k in range(args.steps):
-        rnd.step(draft_ev[k] if k < n_timed else None)
-    e1.record(stream)
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    draft_ms = sum(a.elapsed_time(b) for a, b in draft_ev)
-    launches = ctx.launch_count() - launches0
-    clocks = sampler.stop()
-    local_ms = e0.elapsed_time(e1)
-    stats_ms, stats_n = ctx.profile_read()
-    ctx.profile_enable(False)
-    total_ms, total_bytes = sharding.aggregate(local_ms, step_bytes * args.steps, device=torch.device("cuda", dev))
+    m = measure(ctx, torch, dist, world, rnd, args.steps, warmup)
+    step_bytes = m["step_bytes"]
+    total_ms, total_bytes = sharding.aggregate(m["local_ms"], step_bytes * args.steps, device=torch.device("cuda", dev))
 
     # end to end: host buffers in, results out, every step
     e2e_steps = 0 if args.skip_extras else max(1, min(args.steps, 5))
@@ -506,6 +719,7 @@ def run_ours(args):
     t1.record(stream)
     torch.cuda.synchronize()
     e2e_ms, e2e_bytes = sharding.aggregate(t0.elapsed_time(t1), step_bytes * e2e_steps, device=torch.device("cuda", dev))
+    clocks = sampler.stop()
 
     if rank != 0:
         if world > 1:
@@ -513,49 +727,26 @@ def run_ours(args):
         return
     peak, peak_kind = measured_peak()
     value = total_bytes / (total_ms * 1e-3) / 1e9
-    # the two streaming kernels, each timed live inside the timed region: the row-statistics kernel by
-    # the library's own event pair around its launch, the draft-step kernel as the mean over the
-    # launches of a round (events around the draft launches: launch gaps are inside)
-    stats_bytes = w.n_target_rows * w.V * w.elem_bytes
-    stats_gbs = stats_bytes / (stats_ms / max(stats_n, 1) * 1e-3) / 1e9 if stats_n else None
-    n_draft = rnd.K
-    draft_bytes = w.n_draft_rows * w.V * w.elem_bytes / n_draft
-    draft_us = draft_ms * 1e3 / max(n_timed * n_draft, 1)
-    draft_gbs = draft_bytes / (draft_us * 1e-6) / 1e9
-    dt_name = "bf16" if w.dtype == "bf16" else "f32"
-    roof_stats = {"bound": "hbm", "kernel": "row_stats_kernel<%s> (target rows of svip_verify)" % dt_name,
-                  "achieved": stats_gbs, "peak": peak, "peak_kind": "%s copy bandwidth" % peak_kind, "unit": "GB/s",
-                  "frac": (stats_gbs / peak) if stats_gbs else None, "launches_timed": stats_n,
-                  "bytes_per_launch": stats_bytes, "us_per_launch": stats_ms * 1e3 / max(stats_n, 1),
-                  "share_of_step": stats_ms / max(stats_n, 1) / (total_ms / args.steps),
-                  "traffic": ROW_STATS_TRAFFIC_PER_ALGORITHMIC_BYTE * stats_bytes if w.dtype == "bf16" else None}
-    roof_draft = {"bound": "hbm", "kernel": "draft_step_kernel<%s, sampling> (mean over the %d launches of a round)"
-                  % (dt_name, n_draft), "achieved": draft_gbs, "peak": peak,
-                  "peak_kind": "%s copy bandwidth" % peak_kind, "unit": "GB/s", "frac": draft_gbs / peak,
-                  "launches_timed": n_timed * n_draft, "bytes_per_launch": draft_bytes, "us_per_launch": draft_us,
-                  "share_of_step": draft_ms / n_timed / (total_ms / args.steps),
-                  "traffic": DRAFT_F32_TRAFFIC_PER_ALGORITHMIC_BYTE * draft_bytes
-                  if (w.dtype == "f32" and DRAFT_F32_TRAFFIC_PER_ALGORITHMIC_BYTE) else None}
-    # `roofline` is the kernel with the larger share of the step; the other one rides along
-    dominant, other = (roof_draft, roof_stats) if roof_draft["share_of_step"] >= roof_stats["share_of_step"] \
-        else (roof_stats, roof_draft)
+    dominant, other = rooflines(w, rnd, m, total_ms, peak, peak_kind)
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "warmup": warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": describe(w), "sequences_per_gpu": w.B, "draft_rows": w.n_draft_rows,
-                   "target_rows": w.n_target_rows, "rejected_sequences": rejected,
+                   "target_rows": w.n_target_rows, "rejected_sequences": m["rejected"],
                    "logits_bytes_per_step": step_bytes, "l2": "inputs (%.2f GB per step) larger than L2, no flush" % (step_bytes / 1e9),
-                   "launch": "one stream, %d kernels per step" % (launches // max(args.steps, 1)),
-                   "stop_flags_match_draft_lengths": bool(stops_ok) if w.name == "ragged" else None,
-                   "status_word": status},
+                   "launch": "one stream, %d kernels per step" % (m["launches"] // max(args.steps, 1)),
+                   "stop_flags_match_draft_lengths": bool(m["stops_ok"]) if w.name == "ragged" else None,
+                   "status_word": m["status"]},
         "pct_of_hbm_peak_nominal": 100.0 * value / world / NOMINAL_HBM_GBS,
         "pct_of_hbm_peak_measured": 100.0 * value / world / peak,
+        "us_per_step": 1e3 * total_ms / args.steps,
         "roofline": dominant, "roofline_other": other,
         "e2e": {"value": (e2e_bytes / (e2e_ms * 1e-3) / 1e9) if e2e_steps else None, "unit": "GB/s",
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
-        "gpu_launches": launches, "clocks": clocks,
+        "gpu_launches": m["launches"], "clocks": clocks,
     }
+    gpu_results = rnd.results_by_sequence()
     if not args.skip_extras:
         try:
             line["b1"] = b1_latency(ctx, torch)
@@ -565,8 +756,24 @@ def run_ours(args):
             line["truncated"] = truncated_round(ctx, torch, rnd)
         except Exception as exc:
             line["truncated"] = {"error": repr(exc)}
+        try:
+            line["pair_stats"] = pair_stats_leg(ctx, torch, rnd, peak)
+        except Exception as exc:
+            line["pair_stats"] = {"error": repr(exc)}
     if not args.no_cpu_baseline and not args.skip_extras:
-        line["cpu_baseline"] = cpu_baseline(w)
+        line["cpu_baseline"], line["checks"] = cpu_baseline(w, gpu_results)
+    if not args.skip_extras and world == 1 and args.batch is None:
+        del rnd
+        torch.cuda.empty_cache()
+        line["other_workloads"] = {}
+        for name in ("ragged", "reasoning"):
+            if name == args.workload:
+                continue
+            try:
+                line["other_workloads"][name] = other_workload(ctx, torch, name, rank, peak, peak_kind,
+                                                               max(3, min(args.steps, 50)))
+            except Exception as exc:
+                line["other_workloads"][name] = {"error": repr(exc)}
     line["paper_context"] = ("end-to-end speedups over fixed draft length reported by the paper: up to 17% "
                              "(MT-Bench, 8K context) and 22% (QwQ long-form reasoning); hardware not stated")
     print(json.dumps(line))
@@ -575,39 +782,46 @@ def run_ours(args):
 
 
 def run_reference(args):
-    """The oracle as the reference arm: each step is a bounded sample of the same workload."""
+    """The oracle as the reference arm, on the same workload.  A step is one pass of the oracle over a bounded
+    sample of whole sequences: the whole batch when a pass takes about a second or less, else as many sequences
+    (a multiple of the core count, never fewer than that) as keep the run within a few minutes."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     from oracle import svip_oracle as O
     spec = workloads.SPECS[args.workload]
     cores = len(os.sched_getaffinity(0))
-    n_seq = 2
-    w = workloads.make_workload(args.workload, B=n_seq, seed=workloads.BASE_SEED + spec["index"])
+    w = workloads.make_workload(args.workload, seed=workloads.BASE_SEED + spec["index"], B=args.batch)
     O.lib()
-
-    def step():
-        tok, H, stop = O.draft_step(w.q_logits, w.T, w.h, w.draft_uniforms, threads=cores)
-        nacc, nxt, _ = O.verify(tok.astype(np.int32), w.q_logits, w.target_logits, w.cu_rows, w.T,
-                                w.verify_uniforms, threads=cores)
-        return int((nacc < w.draft_len).sum())
-
-    rej = 0
-    for _ in range(max(args.warmup, 1)):
-        rej = step()
-    t0 = time.perf_counter()
+    warmup = max(args.warmup, 1)
+    # size the sample from one pass over `cores` sequences
+    n0 = min(w.B, cores)
+    dt0, _, _ = _oracle_pass(O, w, _oracle_sample(w, n0), cores)
+    budget_s = 150.0
+    per_seq = dt0 / n0
+    n_seq = int(budget_s / max(args.steps + warmup, 1) / per_seq)
+    n_seq = min(w.B, max(n0, (n_seq // cores) * cores))
+    s = _oracle_sample(w, n_seq)
+    for _ in range(warmup):
+        _oracle_pass(O, w, s, cores)
+    times, nbytes = [], 0
+    t_all = time.perf_counter()
     for _ in range(args.steps):
-        step()
-    dt = time.perf_counter() - t0
-    nbytes = (w.n_draft_rows + w.n_target_rows + rej) * w.V * w.elem_bytes
-    value = nbytes * args.steps / dt / 1e9
-    sample = "%d sequences of the workload per step (%d draft + %d target rows)" % (n_seq, w.n_draft_rows,
-                                                                                  w.n_target_rows)
+        dt, nbytes, _ = _oracle_pass(O, w, s, cores)
+        times.append(dt)
+    total = time.perf_counter() - t_all
+    value = nbytes * args.steps / total / 1e9
+    med = float(np.median(times))
+    n_rows = len(s["rows_q"]) + len(s["rows_t"])
+    sample = "%d of %d sequences of the workload per step (%d draft + %d target rows)" % (
+        n_seq, w.B, len(s["rows_q"]), len(s["rows_t"]))
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": max(args.warmup, 1), "ms_per_step": 1000.0 * dt / args.steps,
+        "steps": args.steps, "warmup": warmup, "ms_per_step": 1000.0 * total / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": describe(w, B=spec["B"]), "sample": sample},
+        "config": {"workload": describe(w), "sample": sample, "whole_batch": bool(n_seq == w.B)},
+        "median_step": {"GBps": nbytes / med / 1e9, "rows_per_s": n_rows / med, "us_per_step": 1e6 * med,
+                        "us_per_whole_batch": 1e6 * med * w.B / n_seq},
         "cpu_baseline": {"value": value, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}))
