@@ -12,6 +12,9 @@
  *   - acceptance test:   Algorithm 2 (sampling), Algorithm 3 (greedy)
  *   - correction token:  Algorithm 4 (sampling), Algorithm 5 (greedy)
  *   - verify loop, bonus token: Algorithm 1 (outer loop body) / Algorithm 6
+ *   - several candidates per position (tree verification, the EAGLE-2 setting
+ *     of Section 3.3): not defined by the paper; the published recursive
+ *     rejection rule, see svip_oracle_verify_tree
  *   - expected acceptance beta, TVD, KL: Eq. 1 - Eq. 4
  *   - top-k / nucleus truncation (end of this file): not defined by the paper;
  *     the published definitions, ties kept by threshold, pinned by hand-made
@@ -221,6 +224,114 @@ int svip_oracle_verify(long K, const int32_t *draft_tokens,
     *n_accepted = n_acc;
     *next_token = next;
     free(p);
+    free(q);
+    return 0;
+}
+
+/*
+ * Verification of a TREE of draft candidates for one sequence (several
+ * candidates per position, as in the EAGLE-2 setting of Section 3.3).  The
+ * paper names that setting but states no accept rule for it; the rule here is
+ * the published multi-candidate generalisation of Algorithms 2 and 4
+ * (recursive rejection sampling), which keeps the paper's premise that every
+ * emitted token follows the target distribution when the candidates of a node
+ * are drawn independently from the draft distribution q of that node:
+ *
+ *   at a node with target distribution p and draft distribution q, and
+ *   candidates x_1..x_m (its children, in index order):
+ *     p_1 = p
+ *     for i = 1..m:  accept x_i if r_i < min(1, p_i(x_i) / q(x_i));
+ *                    else p_{i+1} = max(0, p_i - q) / sum max(0, p_i - q)
+ *     a child accepted: descend into it; none accepted (or no child):
+ *     the next token is drawn from p_{m+1} (from p itself at a leaf) and the
+ *     walk ends.
+ *   With one child per node this is exactly svip_oracle_verify.
+ *
+ * Layout: nodes 0..N-1, parent[i] = -1 for a child of the root, else an index
+ * below i; token[i] the candidate token.  Row k of q_rows / t_rows belongs to
+ * the root for k = 0 and to node k-1 otherwise (N+1 rows each, strides in
+ * elements); q rows of leaves are not read.  r[i] is the accept draw of node
+ * i, r[N] the draw for the final token.
+ * Outputs: *n_accepted, path[0..n_accepted) (the accepted nodes, root to
+ * leaf), *next_token, and, if accept_prob is given (N entries), min(1, p_i/q)
+ * of every candidate that was tried (-1 for the others).
+ * T == 0: a child is accepted iff its token is the argmax of the node's
+ * target row (first such child); the next token is that argmax otherwise.
+ * A residual without mass (cannot happen after a rejection in exact
+ * arithmetic) leaves the distribution as it was, as in svip_oracle_verify.
+ */
+int svip_oracle_verify_tree(long N, const int32_t *parent, const int32_t *token,
+                            const void *q_rows, long q_stride,
+                            const void *t_rows, long t_stride,
+                            int dtype, long V, double T, const double *r,
+                            long *n_accepted, int32_t *path, long *next_token,
+                            double *accept_prob)
+{
+    size_t esz = dtype == SVIP_ORACLE_F32 ? 4 : 2;
+    const char *qb = (const char *)q_rows;
+    const char *tb = (const char *)t_rows;
+    long n = 0, cur = -1;
+    if (accept_prob)
+        for (long i = 0; i < N; ++i) accept_prob[i] = -1.0;
+
+    if (!(T > 0.0)) {
+        for (;;) {
+            long am = svip_oracle_argmax(tb + (size_t)(cur + 1) * t_stride * esz, dtype, V);
+            long taken = -1;
+            for (long i = 0; i < N && taken < 0; ++i) {
+                if (parent[i] != cur) continue;
+                int ok = am == (long)token[i];
+                if (accept_prob) accept_prob[i] = ok ? 1.0 : 0.0;
+                if (ok) taken = i;
+            }
+            if (taken < 0) { *next_token = am; break; }
+            path[n++] = (int32_t)taken;
+            cur = taken;
+        }
+        *n_accepted = n;
+        return 0;
+    }
+
+    double *w = (double *)malloc((size_t)V * sizeof(double));   /* weights of the current p_i */
+    double *q = (double *)malloc((size_t)V * sizeof(double));
+    if (!w || !q) { free(w); free(q); return -1; }
+    for (;;) {
+        svip_oracle_softmax(tb + (size_t)(cur + 1) * t_stride * esz, dtype, V, T, w);
+        double tot = 1.0;                                       /* p_i = w / tot; p_1 = p */
+        int have_q = 0;
+        long taken = -1;
+        for (long i = 0; i < N && taken < 0; ++i) {
+            if (parent[i] != cur) continue;
+            if (!have_q) {
+                svip_oracle_softmax(qb + (size_t)(cur + 1) * q_stride * esz, dtype, V, T, q);
+                have_q = 1;
+            }
+            long x = (long)token[i];
+            double px = w[x] / tot, a;
+            if (q[x] > 0.0) { a = px / q[x]; if (a > 1.0) a = 1.0; }
+            else a = px > 0.0 ? 1.0 : 0.0;
+            if (accept_prob) accept_prob[i] = a;
+            if (r[i] < a) { taken = i; break; }
+            /* rejected: p_{i+1} = max(0, p_i - q), renormalised */
+            double S = 0.0;
+            for (long v = 0; v < V; ++v) {
+                double d = w[v] / tot - q[v];
+                S += d > 0.0 ? d : 0.0;
+            }
+            if (S > 0.0) {
+                for (long v = 0; v < V; ++v) {
+                    double d = w[v] / tot - q[v];
+                    w[v] = d > 0.0 ? d : 0.0;
+                }
+                tot = S;
+            }
+        }
+        if (taken < 0) { *next_token = svip_oracle_invcdf(w, V, r[N]); break; }
+        path[n++] = (int32_t)taken;
+        cur = taken;
+    }
+    *n_accepted = n;
+    free(w);
     free(q);
     return 0;
 }

@@ -66,6 +66,10 @@ def lib():
         L.svip_oracle_threshold.restype = C.c_int
         L.svip_oracle_threshold.argtypes = [C.c_void_p, C.c_int, C.c_long, C.c_double, C.c_long, C.c_double,
                                             dp, dp, dp, C.POINTER(C.c_long)]
+        L.svip_oracle_verify_tree.restype = C.c_int
+        L.svip_oracle_verify_tree.argtypes = [
+            C.c_long, C.c_void_p, C.c_void_p, C.c_void_p, C.c_long, C.c_void_p, C.c_long,
+            C.c_int, C.c_long, C.c_double, dp, C.POINTER(C.c_long), C.c_void_p, C.POINTER(C.c_long), dp]
         L.svip_oracle_residual.restype = C.c_double
         L.svip_oracle_residual.argtypes = [dp, dp, C.c_long, dp]
         _lib = L
@@ -222,6 +226,43 @@ def verify(draft_tokens: np.ndarray, q_logits: np.ndarray, target_logits: np.nda
 
     _pmap(one, B, threads)
     return n_acc, nxt, (aprob if want_accept_prob else None)
+
+
+def verify_tree(parent: np.ndarray, tokens: np.ndarray, q_logits: np.ndarray, target_logits: np.ndarray,
+                T: float, uniforms: np.ndarray, want_accept_prob: bool = False, threads: int = 1):
+    """Tree (multi-candidate) verification of B sequences with N candidate nodes each.
+
+    ``parent`` and ``tokens`` are int [B,N] (parent -1 = child of the root, else a lower node index);
+    ``q_logits`` and ``target_logits`` are [B*(N+1),V]: row b*(N+1) belongs to the root of sequence b, row
+    b*(N+1)+1+i to its node i.  ``uniforms`` is [B,N+1]: an accept draw per node, then the final draw.
+    Returns (n_accepted int64[B], path int32[B,N] padded with -1, next_token int64[B], accept_prob | None).
+    """
+    parent = np.ascontiguousarray(parent, dtype=np.int32); tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+    B, N = parent.shape
+    q_logits = _rows2d(q_logits); target_logits = _rows2d(target_logits)
+    V = target_logits.shape[1]
+    code = _dtype_code(target_logits)
+    assert _dtype_code(q_logits) == code and q_logits.shape == target_logits.shape == (B * (N + 1), V)
+    u = np.ascontiguousarray(uniforms, dtype=np.float64).reshape(B, N + 1)
+    n_acc = np.zeros(B, dtype=np.int64); nxt = np.zeros(B, dtype=np.int64)
+    path = np.full((B, max(N, 1)), -1, dtype=np.int32)
+    aprob = np.full((B, max(N, 1)), -1.0) if want_accept_prob else None
+    L = lib()
+
+    def one(b):
+        na = C.c_long(); nx = C.c_long()
+        rc = L.svip_oracle_verify_tree(
+            N, parent[b].ctypes.data, tokens[b].ctypes.data,
+            q_logits.ctypes.data + b * (N + 1) * q_logits.strides[0], V,
+            target_logits.ctypes.data + b * (N + 1) * target_logits.strides[0], V,
+            code, V, float(T), _dptr(u[b]), C.byref(na), path[b].ctypes.data, C.byref(nx),
+            C.cast(aprob[b].ctypes.data, C.POINTER(C.c_double)) if aprob is not None else None)
+        if rc != 0:
+            raise MemoryError("oracle verify_tree")
+        n_acc[b] = na.value; nxt[b] = nx.value
+
+    _pmap(one, B, threads)
+    return n_acc, path[:, :N], nxt, aprob[:, :N] if aprob is not None else None
 
 
 def pair_stats(target_logits: np.ndarray, q_logits: np.ndarray, T: float, c_bound: float, threads: int = 1):
