@@ -140,8 +140,8 @@ def test_a_rule_without_renormalisation_would_fail(oracle):
     (Guards the pin above: it is sharp enough to see that mistake.)"""
     rng = np.random.default_rng(7)
     V, Bn = 4, 40000
-    q = oracle.softmax((rng.standard_normal(V) * 1.2).astype(np.float32), 1.0)
-    p = oracle.softmax((rng.standard_normal(V) * 1.2).astype(np.float32), 1.0)
+    # p_2 = (1/3, 2/3, 0, 0): token 0 has p_2 / q = 1.11 (always accepted), unnormalised 0.33
+    p = np.array([0.4, 0.3, 0.2, 0.1]); q = np.array([0.3, 0.1, 0.3, 0.3])
     x = rng.choice(V, size=(Bn, 2), p=q)
     u = rng.random((Bn, 3))
     out = np.zeros(Bn, np.int64)
