@@ -66,6 +66,9 @@ typedef enum {
 #define SVIP_STATUS_WAIT_TIMEOUT 4u  /* a block waited a second for its cluster's partial results and gave up; the
                                         outputs of that call are not valid */
 
+#define SVIP_STATUS_BAD_TREE 8u      /* svip_verify_tree saw a parent index that is not below its node, or more
+                                        rejected candidates at one node than it supports (the rest was ignored) */
+
 /* draft-side layout selector for svip_verify: rows packed sequence after sequence */
 #define SVIP_Q_PACKED (-1L)
 
@@ -381,10 +384,61 @@ int svip_pair_stats(svip_ctx* ctx, const void* q_logits, long q_row_stride, cons
                     float* out, void* stream);
 
 /*
+ * Verification of a TREE of draft candidates: several candidates per position,
+ * as when the length policy runs on top of a tree drafter (the EAGLE-2 setting
+ * of Section 3.3).  The paper states no accept rule for that setting; this is
+ * the published multi-candidate generalisation of Algorithms 2 and 4
+ * (recursive rejection sampling), under which every emitted token follows the
+ * target distribution if the candidates of a node were drawn independently
+ * from the node's draft distribution.  At a node with target distribution p,
+ * draft distribution q and candidates x_1..x_m (its children, in index order):
+ *     p_1 = p;  x_i is accepted if r_i < min(1, p_i(x_i) / q(x_i)),
+ *     else p_{i+1} = max(0, p_i - q) / sum max(0, p_i - q);
+ * an accepted candidate becomes the current node; when none is accepted, or
+ * the node has no child, the next token is drawn from p_{m+1} (from p at a
+ * leaf) with the sequence's last draw, and the walk ends.  With one candidate
+ * per node the call computes what svip_verify computes.  T == 0: a child is
+ * accepted iff its token is the lowest-index argmax of the node's target row,
+ * else that argmax is the next token (Algorithms 3 and 5 at every node).
+ *
+ *   B sequences with N candidate nodes each (N >= 1).
+ *   tokens, parent   DEVICE int32 [B, N]: candidate token of node i and its
+ *                    parent, -1 for a child of the root, else an index < i.
+ *   q_logits, target_logits   DEVICE [B * (N + 1), V] rows (strides in
+ *                    elements): row b*(N+1) belongs to the root of sequence b
+ *                    (the distributions after the accepted prefix), row
+ *                    b*(N+1)+1+i to its node i.  Draft rows of leaves are not
+ *                    read by the walk.
+ *   q_stats          DEVICE [B * (N + 1), 2] (max logit, Z) of the draft rows
+ *                    as svip_draft_step writes them, or NULL (one more pass
+ *                    over the draft rows then computes them).  Unused if T == 0.
+ *   uniforms         DEVICE [B, N + 1], in [0,1): the accept draw of node i,
+ *                    then the draw for the final token.  Unused if T == 0.
+ *   n_accepted       DEVICE int32 [B]: length of the accepted path.
+ *   path             DEVICE int32 [B, N]: the accepted nodes from the root
+ *                    down, then -1.
+ *   next_token       DEVICE int32 [B].
+ * Needs B * (N + 1) <= max_rows of svip_create.  At most 15 candidates of one
+ * node can be rejected; further ones are ignored and SVIP_STATUS_BAD_TREE is
+ * set, as for a parent index that is not below its node.  Each rejection costs
+ * one pass over the node's two rows (they are read from L2 after the first
+ * pass), so the call is bound by the length of that chain, not by bandwidth.
+ */
+int svip_verify_tree(svip_ctx* ctx, const int32_t* tokens, const int32_t* parent, const void* q_logits,
+                     long q_row_stride, const float* q_stats, const void* target_logits, long t_row_stride,
+                     svip_dtype dtype, int B, int N, int V, float T, const float* uniforms,
+                     int32_t* n_accepted, int32_t* path, int32_t* next_token, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * Instrumentation and self-test.  Not part of the method (the paper has no
+ * counterpart); benchmarks and tests use these, a serving loop does not.
+ * ------------------------------------------------------------------------- */
+
+/*
  * Timing of the row-statistics kernel (the one pass over all target rows inside
  * svip_verify, its dominant kernel) with CUDA events recorded on the caller's
- * stream around that launch.  The paper has no counterpart; benchmarks use it
- * to report the kernel's bandwidth without a profiler.
+ * stream around that launch.  Benchmarks use it to report the kernel's
+ * bandwidth without a profiler.
  *   svip_profile_enable(ctx, 1) creates the events (not inside a graph
  *   capture) and turns recording on; (ctx, 0) turns it off.  While on, every
  *   svip_verify call records one event pair (at most 4096 pairs are kept
@@ -395,6 +449,18 @@ int svip_pair_stats(svip_ctx* ctx, const void* q_logits, long q_row_stride, cons
  */
 int svip_profile_enable(svip_ctx* ctx, int on);
 int svip_profile_read(svip_ctx* ctx, double* total_ms, long* launches);
+
+/*
+ * Exercises the time-out of the one wait the kernels contain: the blocks of a
+ * cluster wait for one another's partial results on an mbarrier, for at most a
+ * second; if the time runs out they set SVIP_STATUS_WAIT_TIMEOUT and carry on,
+ * so that a lost peer ends in an error status and not in a hang.  This call
+ * launches one block that waits, with the same routine, for `wait_ns`
+ * nanoseconds (1 .. 10^8) on an mbarrier that nothing completes.  Afterwards
+ * svip_read_status reports SVIP_STATUS_WAIT_TIMEOUT and the context works as
+ * before.
+ */
+int svip_selftest_wait_timeout(svip_ctx* ctx, long wait_ns, void* stream);
 
 /*
  * CUDA-graph replay for latency-bound use (small B).  Between begin and end

@@ -254,7 +254,9 @@ int svip_oracle_verify(long K, const int32_t *draft_tokens,
  * i, r[N] the draw for the final token.
  * Outputs: *n_accepted, path[0..n_accepted) (the accepted nodes, root to
  * leaf), *next_token, and, if accept_prob is given (N entries), min(1, p_i/q)
- * of every candidate that was tried (-1 for the others).
+ * of every candidate that was tried (-1 for the others), and, if final_w is
+ * given (V entries, sampling only), the unnormalised weights the next token was
+ * drawn from.
  * T == 0: a child is accepted iff its token is the argmax of the node's
  * target row (first such child); the next token is that argmax otherwise.
  * A residual without mass (cannot happen after a rejection in exact
@@ -265,7 +267,7 @@ int svip_oracle_verify_tree(long N, const int32_t *parent, const int32_t *token,
                             const void *t_rows, long t_stride,
                             int dtype, long V, double T, const double *r,
                             long *n_accepted, int32_t *path, long *next_token,
-                            double *accept_prob)
+                            double *accept_prob, double *final_w)
 {
     size_t esz = dtype == SVIP_ORACLE_F32 ? 4 : 2;
     const char *qb = (const char *)q_rows;
@@ -326,7 +328,11 @@ int svip_oracle_verify_tree(long N, const int32_t *parent, const int32_t *token,
                 tot = S;
             }
         }
-        if (taken < 0) { *next_token = svip_oracle_invcdf(w, V, r[N]); break; }
+        if (taken < 0) {
+            *next_token = svip_oracle_invcdf(w, V, r[N]);
+            if (final_w) memcpy(final_w, w, (size_t)V * sizeof(double));
+            break;
+        }
         path[n++] = (int32_t)taken;
         cur = taken;
     }

@@ -69,7 +69,7 @@ def lib():
         L.svip_oracle_verify_tree.restype = C.c_int
         L.svip_oracle_verify_tree.argtypes = [
             C.c_long, C.c_void_p, C.c_void_p, C.c_void_p, C.c_long, C.c_void_p, C.c_long,
-            C.c_int, C.c_long, C.c_double, dp, C.POINTER(C.c_long), C.c_void_p, C.POINTER(C.c_long), dp]
+            C.c_int, C.c_long, C.c_double, dp, C.POINTER(C.c_long), C.c_void_p, C.POINTER(C.c_long), dp, dp]
         L.svip_oracle_residual.restype = C.c_double
         L.svip_oracle_residual.argtypes = [dp, dp, C.c_long, dp]
         _lib = L
@@ -229,13 +229,15 @@ def verify(draft_tokens: np.ndarray, q_logits: np.ndarray, target_logits: np.nda
 
 
 def verify_tree(parent: np.ndarray, tokens: np.ndarray, q_logits: np.ndarray, target_logits: np.ndarray,
-                T: float, uniforms: np.ndarray, want_accept_prob: bool = False, threads: int = 1):
+                T: float, uniforms: np.ndarray, want_accept_prob: bool = False, threads: int = 1,
+                final_weights: np.ndarray | None = None):
     """Tree (multi-candidate) verification of B sequences with N candidate nodes each.
 
     ``parent`` and ``tokens`` are int [B,N] (parent -1 = child of the root, else a lower node index);
     ``q_logits`` and ``target_logits`` are [B*(N+1),V]: row b*(N+1) belongs to the root of sequence b, row
     b*(N+1)+1+i to its node i.  ``uniforms`` is [B,N+1]: an accept draw per node, then the final draw.
     Returns (n_accepted int64[B], path int32[B,N] padded with -1, next_token int64[B], accept_prob | None).
+    ``final_weights``, a float64 [B,V] array, receives the unnormalised weights each next token was drawn from.
     """
     parent = np.ascontiguousarray(parent, dtype=np.int32); tokens = np.ascontiguousarray(tokens, dtype=np.int32)
     B, N = parent.shape
@@ -256,7 +258,8 @@ def verify_tree(parent: np.ndarray, tokens: np.ndarray, q_logits: np.ndarray, ta
             q_logits.ctypes.data + b * (N + 1) * q_logits.strides[0], V,
             target_logits.ctypes.data + b * (N + 1) * target_logits.strides[0], V,
             code, V, float(T), _dptr(u[b]), C.byref(na), path[b].ctypes.data, C.byref(nx),
-            C.cast(aprob[b].ctypes.data, C.POINTER(C.c_double)) if aprob is not None else None)
+            C.cast(aprob[b].ctypes.data, C.POINTER(C.c_double)) if aprob is not None else None,
+            C.cast(final_weights[b].ctypes.data, C.POINTER(C.c_double)) if final_weights is not None else None)
         if rc != 0:
             raise MemoryError("oracle verify_tree")
         n_acc[b] = na.value; nxt[b] = nx.value

@@ -17,6 +17,8 @@ SVIP_BF16 = 1
 SVIP_Q_PACKED = -1
 SVIP_STATUS_NONFINITE_ROW = 1
 SVIP_STATUS_BAD_DRAFT_LEN = 2
+SVIP_STATUS_WAIT_TIMEOUT = 4
+SVIP_STATUS_BAD_TREE = 8
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 # SVIP_LIBRARY in the environment points at another build of the same ABI (a debug build, say)
@@ -71,6 +73,10 @@ def library():
     L.svip_profile_enable.argtypes = [vp, i32]
     L.svip_profile_read.restype = i32
     L.svip_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_long)]
+    L.svip_verify_tree.restype = i32
+    L.svip_verify_tree.argtypes = [vp, vp, vp, vp, lng, vp, vp, lng, i32, i32, i32, i32, f32, vp, vp, vp, vp, vp]
+    L.svip_selftest_wait_timeout.restype = i32
+    L.svip_selftest_wait_timeout.argtypes = [vp, lng, vp]
     L.svip_draft_step_masked.restype = i32
     L.svip_draft_step_masked.argtypes = [vp, vp, i32, i32, i32, lng, f32, f32, vp, vp, vp, vp, vp, vp, vp]
     L.svip_draft_step_at.restype = i32
@@ -284,6 +290,16 @@ class Context:
         _check(library().svip_pair_stats(self._h, _ptr(q_logits), int(q_row_stride), _ptr(target_logits),
                                          int(t_row_stride), int(dtype), int(n_pairs), int(V), float(T),
                                          float(c_bound), _ptr(out), _stream(stream)), self._h)
+
+    def verify_tree(self, tokens, parent, q_logits, q_row_stride, q_stats, target_logits, t_row_stride, dtype, B, N, V,
+                    T, uniforms, n_accepted, path, next_token, stream=None):
+        _check(library().svip_verify_tree(self._h, _ptr(tokens), _ptr(parent), _ptr(q_logits), int(q_row_stride),
+                                          _ptr(q_stats), _ptr(target_logits), int(t_row_stride), int(dtype), int(B),
+                                          int(N), int(V), float(T), _ptr(uniforms), _ptr(n_accepted), _ptr(path),
+                                          _ptr(next_token), _stream(stream)), self._h)
+
+    def selftest_wait_timeout(self, wait_ns: int, stream=None):
+        _check(library().svip_selftest_wait_timeout(self._h, int(wait_ns), _stream(stream)), self._h)
 
     def profile_enable(self, on: bool):
         _check(library().svip_profile_enable(self._h, 1 if on else 0), self._h)

@@ -11,6 +11,7 @@
 //   svip_analysis.cuh  pair_stats_kernel (Eq. 1-6)
 //   svip_policy.cuh    vocabulary-parallel combine, draft-length policies, ragged packing
 //   svip_select.cuh    row_threshold_kernel (top-k / nucleus truncation)
+//   svip_tree.cuh      verify_tree_kernel (several candidates per position: recursive rejection sampling)
 #include "svip_device.cuh"
 
 #include <cmath>
@@ -27,6 +28,7 @@
 #include "svip_policy.cuh"
 
 #include "svip_select.cuh"
+#include "svip_tree.cuh"
 
 // ==================================================================== host side / C ABI
 
@@ -576,6 +578,91 @@ int svip_profile_read(svip_ctx* ctx, double* total_ms, long* launches) {
     *total_ms = sum;
     *launches = ctx->prof_used;
     ctx->prof_used = 0;
+    return SVIP_OK;
+}
+
+int svip_verify_tree(svip_ctx* ctx, const int32_t* tokens, const int32_t* parent, const void* q_logits,
+                     long q_row_stride, const float* q_stats, const void* target_logits, long t_row_stride,
+                     svip_dtype dtype, int B, int N, int V, float T, const float* uniforms,
+                     int32_t* n_accepted, int32_t* path, int32_t* next_token, void* stream) {
+    if (!ctx || !tokens || !parent || !target_logits || !n_accepted || !path || !next_token) return SVIP_ERR_INVALID_ARG;
+    if (dtype != SVIP_F32 && dtype != SVIP_BF16) return SVIP_ERR_UNSUPPORTED;
+    if (B < 0 || N < 1 || V < 1 || V > 0x7fffffe0 || t_row_stride < 0 || q_row_stride < 0) return SVIP_ERR_INVALID_ARG;
+    if (!(T >= 0.f) || std::isinf(T)) return SVIP_ERR_INVALID_ARG;
+    const bool sampling = T > 0.f;
+    if (sampling && (!q_logits || !uniforms)) return SVIP_ERR_INVALID_ARG;
+    const size_t esz = dtype == SVIP_BF16 ? 2 : 4;
+    if (!aligned_to(target_logits, esz) || (q_logits && !aligned_to(q_logits, esz))) return SVIP_ERR_INVALID_ARG;
+    if (q_stats && !aligned_to(q_stats, 8)) return SVIP_ERR_INVALID_ARG;
+    if (static_cast<long>(B) * (static_cast<long>(N) + 1) >= 0x7fffffffL) return SVIP_ERR_INVALID_ARG;
+    if (B == 0) return SVIP_OK;
+    const long n_rows = static_cast<long>(B) * (N + 1);
+    if (n_rows > ctx->max_rows) return SVIP_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const float c = scale_for(T);
+    cudaError_t e;
+
+    StatsArgs s;
+    s.logits = target_logits; s.row_stride = t_row_stride; s.V = V; s.c = c; s.draft_rows = 0; s.K = 1;
+    s.cu = nullptr; s.q_seq_stride = 0; s.q_pos_stride = 0;
+    s.out_stats = ctx->p_stats; s.out_argmax = sampling ? nullptr : ctx->p_argmax; s.status = ctx->status;
+    s.out_partial = nullptr; s.idx_offset = 0; s.thr = nullptr;
+    const int S = pick_cluster(ctx, n_rows, V, dtype);
+    if (sampling)
+        e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 1>, n_rows, S, s, st, kRingBytes)
+                               : launch_clustered(row_stats_kernel<kF32, 1>, n_rows, S, s, st, kRingBytes);
+    else
+        e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 0>, n_rows, S, s, st, kRingBytes)
+                               : launch_clustered(row_stats_kernel<kF32, 0>, n_rows, S, s, st, kRingBytes);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+
+    if (!sampling) {
+        TreeGreedyArgs g;
+        g.tokens = tokens; g.parent = parent; g.p_argmax = ctx->p_argmax; g.B = B; g.N = N;
+        g.n_accepted = n_accepted; g.path = path; g.next_token = next_token;
+        e = launch_ex(verify_tree_greedy_kernel, static_cast<unsigned>((B + kPolicyThreads - 1) / kPolicyThreads),
+                      kPolicyThreads, 0, 0, st, g);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        ctx->launches += 1;
+        return SVIP_OK;
+    }
+
+    if (!q_stats) {
+        StatsArgs d = s;
+        d.logits = q_logits; d.row_stride = q_row_stride; d.out_stats = ctx->q_stats; d.out_argmax = nullptr;
+        e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 1>, n_rows, S, d, st, kRingBytes)
+                               : launch_clustered(row_stats_kernel<kF32, 1>, n_rows, S, d, st, kRingBytes);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        ctx->launches += 1;
+    }
+
+    TreeArgs t;
+    t.tokens = tokens; t.parent = parent; t.q_logits = q_logits; t.q_row_stride = q_row_stride;
+    t.q_stats = q_stats ? reinterpret_cast<const float2*>(q_stats) : ctx->q_stats;
+    t.t_logits = target_logits; t.t_row_stride = t_row_stride; t.p_stats = ctx->p_stats;
+    t.N = N; t.V = V; t.c = c; t.uniforms = uniforms; t.n_accepted = n_accepted; t.path = path;
+    t.next_token = next_token; t.status = ctx->status;
+    // the walk is a chain of passes over two rows: spread a sequence over as many blocks as the batch leaves room for
+    int Sf = pick_cluster(ctx, B, V, dtype);
+    if (ctx->cluster_override == 0) {
+        const long row_bytes = static_cast<long>(V) * static_cast<long>(esz);
+        while (Sf < kMaxCluster && 2 * row_bytes / Sf > (512L << 10)) Sf *= 2;
+        if (Sf > kMaxCluster) Sf = kMaxCluster;
+    }
+    e = dtype == SVIP_BF16 ? launch_clustered(verify_tree_kernel<kBF16>, B, Sf, t, st, 0)
+                           : launch_clustered(verify_tree_kernel<kF32>, B, Sf, t, st, 0);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    return SVIP_OK;
+}
+
+int svip_selftest_wait_timeout(svip_ctx* ctx, long wait_ns, void* stream) {
+    if (!ctx || wait_ns < 1 || wait_ns > 100000000L) return SVIP_ERR_INVALID_ARG;
+    cudaError_t e = launch_ex(wait_timeout_kernel, 1, 32, 0, 0, static_cast<cudaStream_t>(stream),
+                              static_cast<unsigned long long>(wait_ns), ctx->status);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    ctx->launches += 1;
     return SVIP_OK;
 }
 

@@ -229,4 +229,19 @@ __global__ void __launch_bounds__(kPackThreads) pack_ragged_kernel(const int32_t
     }
 }
 
+// One block waits on an mbarrier that expects bytes nobody sends, with the bounded wait of the
+// cluster exchange, and reports the time-out in the status word (svip_selftest_wait_timeout).
+__global__ void __launch_bounds__(32) wait_timeout_kernel(unsigned long long wait_ns, unsigned* status) {
+    __shared__ unsigned long long bar;
+    pdl_launch_dependents();
+    pdl_wait();
+    const uint32_t b = static_cast<uint32_t>(__cvta_generic_to_shared(&bar));
+    if (threadIdx.x == 0) {
+        mbar_init(b, 1);
+        mbar_arrive_expect_tx(b, 16);
+    }
+    __syncwarp();
+    if (!mbar_wait_bounded(b, 0, wait_ns) && threadIdx.x == 0) atomicOr(status, SVIP_STATUS_WAIT_TIMEOUT);
+}
+
 }  // namespace svip

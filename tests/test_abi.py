@@ -59,6 +59,7 @@ def test_null_context_is_invalid_argument(lib):
     body = C.c_void_p()
     assert lib.svip_graph_loop_begin(None, None, 16, 4, C.byref(body)) == -1
     assert lib.svip_launch_count(None) == 0
+    assert lib.svip_selftest_wait_timeout(None, 1000, None) == -1
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):

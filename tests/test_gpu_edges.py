@@ -110,3 +110,29 @@ def test_masked_draft_step_leaves_skipped_rows_alone(ctx, oracle):
     assert np.all(tok.cpu().numpy()[~on] == -3) and np.all(ent.cpu().numpy()[~on] == -3.0)
     assert np.all(stop.cpu().numpy()[~on] == 7) and np.all(stats.cpu().numpy()[~on] == -3.0)
     assert ctx.read_status() == 0
+
+
+def test_a_wait_that_nothing_ends_times_out_with_a_status_bit(ctx, oracle):
+    """The blocks of a cluster wait for one another's partial results on an mbarrier, for a bounded time.
+    The self-test waits with the same routine on an mbarrier that nothing completes: the wait must run out,
+    report SVIP_STATUS_WAIT_TIMEOUT, and leave the context usable (the next draft step is correct)."""
+    import time
+    import torch
+    from paper_2411_18462_b200 import SvipError, binding
+    assert ctx.read_status() == 0
+    t0 = time.perf_counter()
+    ctx.selftest_wait_timeout(2_000_000)          # two milliseconds
+    torch.cuda.synchronize()
+    waited = time.perf_counter() - t0
+    assert ctx.read_status() == binding.SVIP_STATUS_WAIT_TIMEOUT
+    assert 0.0015 < waited < 1.0, waited
+    assert ctx.read_status() == 0                 # reading clears the word
+    for bad in (0, -5, 10**9):
+        with pytest.raises(SvipError):
+            ctx.selftest_wait_timeout(bad)
+    rng = np.random.default_rng(3)
+    x = (rng.standard_normal((6, 40000)) * 2).astype(np.float32)
+    u = rng.random(6).astype(np.float32)
+    got = tl.gpu_draft_step(ctx, x, 1.0, 0.3, u)   # clusters of several blocks: the real exchange
+    tl.check_draft_against_oracle(oracle, x, 1.0, 0.3, u, got, "after the time-out")
+    assert ctx.read_status() == 0
