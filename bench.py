@@ -420,8 +420,11 @@ def truncated_round(ctx, torch, rnd, top_k=50, top_p=0.9, reps=10):
 
 
 def pair_stats_leg(ctx, torch, rnd, peak, reps=10):
-    """svip_pair_stats over every (draft row, target row under it) pair of the round, on contiguous copies of
-    the resident rows (gathered outside the timed region).  Algorithmic bytes: both rows of a pair once."""
+    """The analysis quantities (Eq. 1-6) of every (draft row, target row under it) pair of the round, on
+    contiguous copies of the resident rows (gathered outside the timed region).  Algorithmic bytes: both rows of
+    a pair once.  Two forms: svip_pair_stats (normalisers computed inside: the rows are streamed twice) and
+    svip_pair_stats_given with the normalisers a round has anyway (the draft step's row_stats; for the target
+    rows one svip_row_threshold pass with nothing cut, timed beside it)."""
     w, B, V = rnd.w, rnd.B, rnd.V
     if not w.T > 0:
         return None
@@ -430,25 +433,37 @@ def pair_stats_leg(ctx, torch, rnd, peak, reps=10):
     q_idx = np.concatenate([np.arange(rnd.lens[k]) * B + k for k in range(B)])
     t_idx = np.concatenate([cu[k] + np.arange(rnd.lens[k]) for k in range(B)])
     n = int(q_idx.size)
-    q = rnd.d_q.index_select(0, torch.from_numpy(q_idx).to(dev))
+    qi = torch.from_numpy(q_idx).to(dev)
+    q = rnd.d_q.index_select(0, qi)
     t = rnd.d_t.index_select(0, torch.from_numpy(t_idx).to(dev))
+    q_stats = rnd.d_stats.index_select(0, qi).contiguous()
+    p_stats = torch.zeros(n, 2, device=dev); thr = torch.zeros(n, device=dev)
     out = torch.zeros(n, 8, device=dev)
-    call = ctx.bind("pair_stats", q, V, t, V, rnd.dt, n, V, w.T, 0.18, out, rnd.stream)
-    call()
-    torch.cuda.synchronize()
-    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(reps):
-        call()
-    e1.record()
-    torch.cuda.synchronize()
-    us = 1000.0 * e0.elapsed_time(e1) / reps
+    calls = {"pair_stats": ctx.bind("pair_stats", q, V, t, V, rnd.dt, n, V, w.T, 0.18, out, rnd.stream),
+             "target_normalisers": ctx.bind("row_threshold", t, rnd.dt, n, V, V, w.T, 0, 1.0, thr, p_stats, rnd.stream),
+             "pair_stats_given": ctx.bind("pair_stats_given", q, V, q_stats, t, V, p_stats, rnd.dt, n, V, w.T, 0.18,
+                                          out, rnd.stream)}
     nbytes = 2 * n * V * rnd.esz
-    res = out.cpu().numpy()
-    return {"pairs": n, "us_per_call": us, "algorithmic_bytes": nbytes, "GBps": nbytes / (us * 1e-6) / 1e9,
-            "frac_of_measured_peak": nbytes / (us * 1e-6) / 1e9 / peak,
-            "mean_beta": float(res[:, 0].mean()), "mean_H_q": float(res[:, 1].mean()),
-            "non_finite_outputs": int((~np.isfinite(res)).sum())}
+    res = {"pairs": n, "algorithmic_bytes": nbytes}
+    for name, call in calls.items():
+        call()
+        torch.cuda.synchronize()
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            call()
+        e1.record()
+        torch.cuda.synchronize()
+        us = 1000.0 * e0.elapsed_time(e1) / reps
+        if name == "target_normalisers":
+            res[name + "_us"] = us
+            continue
+        o = out.cpu().numpy()
+        res[name] = {"us_per_call": us, "GBps": nbytes / (us * 1e-6) / 1e9,
+                     "frac_of_measured_peak": nbytes / (us * 1e-6) / 1e9 / peak,
+                     "mean_beta": float(o[:, 0].mean()), "mean_H_q": float(o[:, 1].mean()),
+                     "nan_outputs": int(np.isnan(o).sum())}
+    return res
 
 
 CDF_TOL = 1e-5        # a sampled token may differ from the oracle's only across a CDF boundary closer than this

@@ -373,15 +373,25 @@ int svip_vp_locate(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, i
  * Pair r reads target row r (element r*t_row_stride) and draft row r (element
  * r*q_row_stride).  `out` is DEVICE [n_pairs][8] fp32.  Where the target masks
  * a token (-inf) that the draft gives mass, KL, H_qp and gamma are +inf.
- * Entropies are fp32 sums, good to about 1e-7 nats: for a draft row that is
- * one-hot to that resolution H_q comes out as 0 and gamma, a ratio that has no
- * limit there, as +inf or NaN.
- * Needs n_pairs <= max_rows of svip_create.  Three kernels: the two rows'
- * normalisers, then one pass over both rows.
+ * Entropies are fp32 sums, good to about 1e-7 nats.  gamma = H_qp / H_q =
+ * 1 + KL / H_q: where H_q comes out as 0 (a draft row that is one-hot to that
+ * resolution) gamma is +inf if KL > 0 and 1 if KL is 0 too; no NaN is written.
+ * One kernel: both rows are streamed once for the normalisers, the entropy and
+ * KL, then once more for beta, which needs the normalisers.
+ *
+ * svip_pair_stats_given is the same for callers that already hold the rows'
+ * normalisers: q_stats / p_stats are DEVICE [n_pairs, 2] (max logit, Z) of the
+ * draft / target row of every pair, as svip_draft_step writes its row_stats and
+ * svip_row_threshold its stats (with top_k = 0, top_p = 1 for the whole row),
+ * at the same T.  Everything then comes out of one pass over the two rows.
+ * Both NULL: the call is svip_pair_stats.
  */
 int svip_pair_stats(svip_ctx* ctx, const void* q_logits, long q_row_stride, const void* target_logits,
                     long t_row_stride, svip_dtype dtype, int n_pairs, int V, float T, float c_bound,
                     float* out, void* stream);
+int svip_pair_stats_given(svip_ctx* ctx, const void* q_logits, long q_row_stride, const float* q_stats,
+                          const void* target_logits, long t_row_stride, const float* p_stats, svip_dtype dtype,
+                          int n_pairs, int V, float T, float c_bound, float* out, void* stream);
 
 /*
  * Verification of a TREE of draft candidates: several candidates per position,

@@ -388,7 +388,9 @@ double svip_oracle_residual(const double *p, const double *q, long V, double *w)
  *   out[1] H_q    = entropy of the draft distribution                 (Eq. 4)
  *   out[2] H_qp   = cross entropy -sum q ln p                         (Eq. 4)
  *   out[3] KL     = KL(q || p) = H_qp - H_q                           (Eq. 3 / Eq. 4)
- *   out[4] gamma  = H_qp / H_q                                        (Section 2.2)
+ *   out[4] gamma  = H_qp / H_q = 1 + KL / H_q                         (Section 2.2);
+ *                   for a one-hot draft row (H_q = 0): +inf if KL > 0, 1 if KL = 0
+ *                   (gamma - 1 = KL / H_q is 0 for KL = 0 whatever H_q)
  *   out[5] 1 - sqrt(KL / 2)                 Pinsker "oracle bound"    (Eq. 3)
  *   out[6] 1 - sqrt(1 - exp(-KL))           Bretagnolle-Huber bound   (Appendix B)
  *   out[7] 1 - sqrt(c * H_q)                approximation bound       (Eq. 6)
@@ -410,7 +412,7 @@ int svip_oracle_pair_stats(const void *t_row, const void *q_row, int dtype, long
     out[1] = Hq;
     out[2] = Hqp;
     out[3] = KL;
-    out[4] = Hqp / Hq;
+    out[4] = Hq > 0.0 ? Hqp / Hq : (KL > 0.0 ? INFINITY : 1.0);
     out[5] = 1.0 - sqrt(0.5 * (KL > 0.0 ? KL : 0.0));
     out[6] = 1.0 - sqrt(1.0 - exp(-(KL > 0.0 ? KL : 0.0)));
     out[7] = 1.0 - sqrt(c_bound * Hq);

@@ -73,6 +73,8 @@ def library():
     L.svip_profile_enable.argtypes = [vp, i32]
     L.svip_profile_read.restype = i32
     L.svip_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_long)]
+    L.svip_pair_stats_given.restype = i32
+    L.svip_pair_stats_given.argtypes = [vp, vp, lng, vp, vp, lng, vp, i32, i32, i32, f32, f32, vp, vp]
     L.svip_verify_tree.restype = i32
     L.svip_verify_tree.argtypes = [vp, vp, vp, vp, lng, vp, vp, lng, i32, i32, i32, i32, f32, vp, vp, vp, vp, vp]
     L.svip_selftest_wait_timeout.restype = i32
@@ -297,6 +299,13 @@ class Context:
                                           _ptr(q_stats), _ptr(target_logits), int(t_row_stride), int(dtype), int(B),
                                           int(N), int(V), float(T), _ptr(uniforms), _ptr(n_accepted), _ptr(path),
                                           _ptr(next_token), _stream(stream)), self._h)
+
+    def pair_stats_given(self, q_logits, q_row_stride, q_stats, target_logits, t_row_stride, p_stats, dtype, n_pairs, V, T,
+                         c_bound, out, stream=None):
+        _check(library().svip_pair_stats_given(self._h, _ptr(q_logits), int(q_row_stride), _ptr(q_stats),
+                                               _ptr(target_logits), int(t_row_stride), _ptr(p_stats), int(dtype),
+                                               int(n_pairs), int(V), float(T), float(c_bound), _ptr(out),
+                                               _stream(stream)), self._h)
 
     def selftest_wait_timeout(self, wait_ns: int, stream=None):
         _check(library().svip_selftest_wait_timeout(self._h, int(wait_ns), _stream(stream)), self._h)

@@ -488,6 +488,25 @@ def test_pair_stats_inequalities_and_gamma_condition(oracle):
     assert np.allclose(same[:, 4], 1.0, atol=1e-12)
 
 
+def test_gamma_of_a_one_hot_draft_row(oracle):
+    """gamma = H_qp / H_q = 1 + KL / H_q (Section 2.2 with Eq. 4).  For a one-hot draft row H_q = 0: with KL = 0
+    (the target puts all its mass on the same token) gamma - 1 = KL / H_q is 0 along every path to that point,
+    so gamma = 1; with KL > 0 the ratio diverges: +inf.  Never NaN."""
+    V = 7
+    q = np.full((1, V), -np.inf, dtype=np.float32); q[0, 3] = 1.5
+    same = q.copy()
+    spread = np.zeros((1, V), dtype=np.float32)
+    out = oracle.pair_stats(np.concatenate([same, spread]), np.concatenate([q, q]), 1.0, 0.18)
+    assert out[0, 1] == 0.0 and out[0, 3] == 0.0 and out[0, 4] == 1.0 and out[0, 0] == 1.0
+    assert out[1, 1] == 0.0 and abs(out[1, 3] - math.log(V)) < 1e-12 and out[1, 4] == np.inf
+    assert not np.isnan(out).any()
+    # approaching the one-hot row: gamma stays finite and tends to 1 when p follows q
+    for L in (5.0, 20.0, 40.0):
+        d = np.zeros((1, V), dtype=np.float32); d[0, 3] = L
+        o = oracle.pair_stats(d, d, 1.0, 0.18)
+        assert abs(o[0, 4] - 1.0) < 1e-9
+
+
 # ---------------------------------------------------------------- ragged packing
 
 def test_pack_ragged_is_exclusive_scan(oracle):
