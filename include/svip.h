@@ -69,6 +69,9 @@ typedef enum {
 #define SVIP_STATUS_BAD_TREE 8u      /* svip_verify_tree saw a parent index that is not below its node, or more
                                         rejected candidates at one node than it supports (the rest was ignored) */
 
+#define SVIP_STATUS_DEBUG_OOB 16u    /* bounds-checked build only: a kernel asked for logits outside the buffers
+                                        of its call (the load was not performed) */
+
 /* draft-side layout selector for svip_verify: rows packed sequence after sequence */
 #define SVIP_Q_PACKED (-1L)
 

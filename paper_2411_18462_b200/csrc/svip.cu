@@ -32,6 +32,20 @@
 
 // ==================================================================== host side / C ABI
 
+// -DSVIP_NVTX: a named range around every entry point's host work, for timelines.
+#ifdef SVIP_NVTX
+#include <nvtx3/nvToolsExt.h>
+namespace {
+struct NvtxRange {
+    explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+};
+}  // namespace
+#define SVIP_RANGE(name) NvtxRange svip_nvtx_range_(name)
+#else
+#define SVIP_RANGE(name) do { } while (0)
+#endif
+
 using namespace svip;
 
 struct svip_ctx {
@@ -141,6 +155,36 @@ int pick_cluster(const svip_ctx* ctx, long rows, int V, int dtype) {
     }
     return static_cast<int>(S);
 }
+
+// Bytes from the start of the first row to the end of the last one.
+[[maybe_unused]] size_t rows_extent(long n_rows, long row_stride, int V, size_t esz) {
+    if (n_rows < 1) return 0;
+    return (static_cast<size_t>(n_rows - 1) * static_cast<size_t>(row_stride) + static_cast<size_t>(V)) * esz;
+}
+
+// -DSVIP_DEBUG_BOUNDS: the extents of the (up to two) logits buffers of a call go into constant memory
+// ahead of its kernels, which then refuse loads outside them (see debug_ok).  The vector loads start at the
+// 16-byte boundary below a row and end at the one above it, hence the rounding.
+#ifdef SVIP_DEBUG_BOUNDS
+cudaError_t debug_ranges(const svip_ctx* ctx, cudaStream_t st, const void* p0, size_t bytes0, const void* p1 = nullptr,
+                         size_t bytes1 = 0) {
+    DebugRange r[2];
+    const void* p[2] = {p0, p1};
+    const size_t n[2] = {bytes0, bytes1};
+    for (int i = 0; i < 2; ++i) {
+        const unsigned long long a = reinterpret_cast<unsigned long long>(p[i]);
+        r[i].lo = p[i] ? (a & ~15ull) : 0;
+        r[i].hi = p[i] ? ((a + n[i] + 15ull) & ~15ull) : 0;
+        if (p[i] && n[i] == ~static_cast<size_t>(0)) { r[i].lo = 0; r[i].hi = ~0ull; }   // extent not known
+    }
+    if (ctx->capturing) { r[0].lo = 0; r[0].hi = ~0ull; }   // no copies from host memory into a graph
+    if (ctx->capturing) return cudaSuccess;
+    return cudaMemcpyToSymbolAsync(g_debug_range, r, sizeof r, 0, cudaMemcpyHostToDevice, st);
+}
+#define SVIP_DEBUG_RANGES(...) do { if (debug_ranges(__VA_ARGS__) != cudaSuccess) return SVIP_ERR_CUDA; } while (0)
+#else
+#define SVIP_DEBUG_RANGES(...) do { } while (0)
+#endif
 
 bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
@@ -269,6 +313,13 @@ int svip_read_status(svip_ctx* ctx, unsigned* flags, void* stream) {
     if (e == cudaSuccess) e = cudaMemsetAsync(ctx->status, 0, sizeof v, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
+#ifdef SVIP_DEBUG_BOUNDS
+    unsigned oob = 0, zero = 0;
+    e = cudaMemcpyFromSymbol(&oob, g_debug_oob, sizeof oob);
+    if (e == cudaSuccess) e = cudaMemcpyToSymbol(g_debug_oob, &zero, sizeof zero);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    if (oob) v |= SVIP_STATUS_DEBUG_OOB;
+#endif
     *flags = v;
     return SVIP_OK;
 }
@@ -320,6 +371,9 @@ static int draft_impl(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B
     if (T > 0.f && !uniforms) return SVIP_ERR_INVALID_ARG;
     if (!aligned_to(logits, dtype == SVIP_BF16 ? 2 : 4)) return SVIP_ERR_INVALID_ARG;
     if (B == 0) return SVIP_OK;
+    SVIP_RANGE("svip_draft_step");
+    SVIP_DEBUG_RANGES(ctx, static_cast<cudaStream_t>(stream), logits,
+                      pos ? ~static_cast<size_t>(0) : rows_extent(B, row_stride, V, dtype == SVIP_BF16 ? 2 : 4));
     DraftArgs a;
     a.logits = logits; a.row_stride = row_stride; a.V = V; a.c = scale_for(T); a.thresh = thresh;
     a.greedy = T > 0.f ? 0 : 1; a.uniforms = uniforms; a.token = token; a.entropy = entropy;
@@ -355,6 +409,8 @@ int svip_row_threshold(svip_ctx* ctx, const void* logits, svip_dtype dtype, int 
     if (!(T > 0.f) || std::isinf(T) || !(top_p > 0.f)) return SVIP_ERR_INVALID_ARG;
     if (!aligned_to(logits, dtype == SVIP_BF16 ? 2 : 4)) return SVIP_ERR_INVALID_ARG;
     if (n_rows == 0) return SVIP_OK;
+    SVIP_RANGE("svip_row_threshold");
+    SVIP_DEBUG_RANGES(ctx, static_cast<cudaStream_t>(stream), logits, rows_extent(n_rows, row_stride, V, dtype == SVIP_BF16 ? 2 : 4));
     ThresholdArgs a;
     a.logits = logits; a.row_stride = row_stride; a.V = V; a.c = scale_for(T);
     a.top_k = (top_k >= 1 && top_k < V) ? top_k : 0; a.top_p = top_p; a.thr = thr;
@@ -382,6 +438,8 @@ int svip_draft_step_truncated(svip_ctx* ctx, const void* logits, svip_dtype dtyp
     if (!aligned_to(logits, dtype == SVIP_BF16 ? 2 : 4)) return SVIP_ERR_INVALID_ARG;
     if (row_stats && !aligned_to(row_stats, 8)) return SVIP_ERR_INVALID_ARG;
     if (B == 0) return SVIP_OK;
+    SVIP_RANGE("svip_draft_step_truncated");
+    SVIP_DEBUG_RANGES(ctx, static_cast<cudaStream_t>(stream), logits, rows_extent(B, row_stride, V, dtype == SVIP_BF16 ? 2 : 4));
     ThresholdArgs a;
     a.logits = logits; a.row_stride = row_stride; a.V = V; a.c = scale_for(T);
     a.top_k = (top_k >= 1 && top_k < V) ? top_k : 0; a.top_p = top_p; a.thr = thr;
@@ -439,6 +497,13 @@ static int verify_impl(svip_ctx* ctx, const int32_t* draft_tokens, const void* q
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const float c = scale_for(T);
     cudaError_t e;
+    SVIP_RANGE("svip_verify");
+    {
+        [[maybe_unused]] const long q_rows =
+            q_seq_stride < 0 ? n_target_rows - B : (B - 1) * q_seq_stride + (static_cast<long>(K) - 1) * q_pos_stride + 1;
+        SVIP_DEBUG_RANGES(ctx, st, target_logits, rows_extent(n_target_rows, t_row_stride, V, esz), q_logits,
+                          rows_extent(q_rows, q_row_stride, V, esz));
+    }
 
     StatsArgs s;
     s.logits = target_logits; s.row_stride = t_row_stride; s.V = V; s.c = c; s.draft_rows = 0; s.K = K;
@@ -603,6 +668,9 @@ int svip_verify_tree(svip_ctx* ctx, const int32_t* tokens, const int32_t* parent
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const float c = scale_for(T);
     cudaError_t e;
+    SVIP_RANGE("svip_verify_tree");
+    SVIP_DEBUG_RANGES(ctx, st, target_logits, rows_extent(n_rows, t_row_stride, V, esz), q_logits,
+                      rows_extent(n_rows, q_row_stride, V, esz));
 
     StatsArgs s;
     s.logits = target_logits; s.row_stride = t_row_stride; s.V = V; s.c = c; s.draft_rows = 0; s.K = 1;
@@ -715,6 +783,7 @@ int svip_vp_partial(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, 
     if (!(T >= 0.f) || std::isinf(T)) return SVIP_ERR_INVALID_ARG;
     if (!aligned_to(logits, dtype == SVIP_BF16 ? 2 : 4) || !aligned_to(partial, 16)) return SVIP_ERR_INVALID_ARG;
     if (B == 0) return SVIP_OK;
+    SVIP_DEBUG_RANGES(ctx, static_cast<cudaStream_t>(stream), logits, rows_extent(B, row_stride, V_shard, dtype == SVIP_BF16 ? 2 : 4));
     StatsArgs s;
     s.logits = logits; s.row_stride = row_stride; s.V = V_shard; s.c = scale_for(T); s.draft_rows = 0; s.K = 1;
     s.cu = nullptr; s.q_seq_stride = 0; s.q_pos_stride = 0; s.out_stats = nullptr; s.out_argmax = nullptr;
@@ -757,6 +826,7 @@ int svip_vp_locate(svip_ctx* ctx, const void* logits, svip_dtype dtype, int B, i
     if (!(T > 0.f) || std::isinf(T)) return SVIP_ERR_INVALID_ARG;
     if (!aligned_to(logits, dtype == SVIP_BF16 ? 2 : 4)) return SVIP_ERR_INVALID_ARG;
     if (B == 0) return SVIP_OK;
+    SVIP_DEBUG_RANGES(ctx, static_cast<cudaStream_t>(stream), logits, rows_extent(B, row_stride, V_shard, dtype == SVIP_BF16 ? 2 : 4));
     DraftArgs a;
     a.logits = logits; a.row_stride = row_stride; a.V = V_shard; a.c = scale_for(T); a.thresh = 0.f; a.greedy = 0;
     a.uniforms = nullptr; a.token = token; a.entropy = nullptr; a.stop = nullptr; a.row_stats = nullptr;
@@ -792,6 +862,9 @@ int svip_pair_stats_given(svip_ctx* ctx, const void* q_logits, long q_row_stride
     if (!aligned_to(target_logits, esz) || !aligned_to(q_logits, esz)) return SVIP_ERR_INVALID_ARG;
     if (n_pairs == 0) return SVIP_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    SVIP_RANGE("svip_pair_stats");
+    SVIP_DEBUG_RANGES(ctx, st, target_logits, rows_extent(n_pairs, t_row_stride, V, esz), q_logits,
+                      rows_extent(n_pairs, q_row_stride, V, esz));
     // (Measured: spreading a pair over more blocks so that the second pass finds the rows in L2 costs more
     // in latency than it saves in traffic: 1024 pairs of 152064 bf16 logits 195 us at one block per pair,
     // 290 us at four.)

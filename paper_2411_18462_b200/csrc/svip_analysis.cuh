@@ -88,9 +88,9 @@ __device__ __forceinline__ void stream_pair(const RowGeom& g, const RowGeom& gq,
     seg_range(g, seg, v_lo, v_hi);
     auto masked = [&](int vi) {
         float x[EPV], d[EPV];
-        unpack_masked<DT>(__ldg(g.base + vi), vi, g, x);
+        unpack_masked<DT>(ld_vec(g.base + vi), vi, g, x);
         if (gq.pre == g.pre) {
-            unpack_masked<DT>(__ldg(gq.base + vi), vi, gq, d);
+            unpack_masked<DT>(ld_vec(gq.base + vi), vi, gq, d);
         } else {
 #pragma unroll
             for (int j = 0; j < EPV; ++j) {
@@ -158,9 +158,9 @@ __device__ __noinline__ PairPartial pair_segment_exact(const RowGeom& g, const R
     int v_lo, v_hi;
     seg_range(g, seg, v_lo, v_hi);
     auto load = [&](int vi, float (&x)[EPV], float (&d)[EPV]) {
-        unpack_masked<DT>(__ldg(g.base + vi), vi, g, x);
+        unpack_masked<DT>(ld_vec(g.base + vi), vi, g, x);
         if (gq.pre == g.pre) {
-            unpack_masked<DT>(__ldg(gq.base + vi), vi, gq, d);
+            unpack_masked<DT>(ld_vec(gq.base + vi), vi, gq, d);
         } else {
 #pragma unroll
             for (int j = 0; j < EPV; ++j) {

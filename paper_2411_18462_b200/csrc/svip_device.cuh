@@ -52,6 +52,26 @@ constexpr float kMaxLogit = 1.0e29f;    // rows whose maximum lies outside +-1e2
 
 __device__ __forceinline__ float neg_inf() { return __int_as_float(0xff800000); }
 
+// Bounds-checked build (-DSVIP_DEBUG_BOUNDS): every global load of logits (the ring's cp.async copies, the
+// streaming vector loads, the single-element gathers) is checked against the extents of the logits buffers
+// of the call, which the host puts into constant memory before the launch.  A load outside is not
+// performed (zeros are used) and counted; svip_read_status then reports SVIP_STATUS_DEBUG_OOB.  Stands in
+// for a memory checker where none can be run.
+#ifdef SVIP_DEBUG_BOUNDS
+struct DebugRange { unsigned long long lo, hi; };
+__constant__ DebugRange g_debug_range[2];
+__device__ unsigned g_debug_oob;
+__device__ __forceinline__ bool debug_ok(const void* p, unsigned bytes) {
+    const unsigned long long a = reinterpret_cast<unsigned long long>(p);
+    const bool ok = (a >= g_debug_range[0].lo && a + bytes <= g_debug_range[0].hi) ||
+                    (a >= g_debug_range[1].lo && a + bytes <= g_debug_range[1].hi);
+    if (!ok) atomicAdd(&g_debug_oob, 1u);
+    return ok;
+}
+#else
+__device__ __forceinline__ bool debug_ok(const void*, unsigned) { return true; }
+#endif
+
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -61,10 +81,17 @@ __device__ __forceinline__ float ex2_approx(float x) {
 // 128-bit streaming load: read-only path, no L1 allocation (each byte is used once).
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
     uint4 v;
+    if (!debug_ok(p, 16)) return make_uint4(0, 0, 0, 0);
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                  : "l"(p));
     return v;
+}
+
+// 128-bit load through the read-only path that may be reused (second touches: fine scans, residual rows).
+__device__ __forceinline__ uint4 ld_vec(const uint4* p) {
+    if (!debug_ok(p, 16)) return make_uint4(0, 0, 0, 0);
+    return __ldg(p);
 }
 
 template <int DT> struct ElemTraits;
@@ -76,6 +103,7 @@ template <> struct ElemTraits<kF32> {
         x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
     }
     __device__ static __forceinline__ float load_one(const void* row, int i) {
+        if (!debug_ok(reinterpret_cast<const float*>(row) + i, 4)) return 0.f;
         return __ldg(reinterpret_cast<const float*>(row) + i);
     }
 };
@@ -90,6 +118,7 @@ template <> struct ElemTraits<kBF16> {
         x[6] = __uint_as_float(v.w << 16); x[7] = __uint_as_float(v.w & 0xffff0000u);
     }
     __device__ static __forceinline__ float load_one(const void* row, int i) {
+        if (!debug_ok(reinterpret_cast<const unsigned short*>(row) + i, 2)) return 0.f;
         unsigned short h = __ldg(reinterpret_cast<const unsigned short*>(row) + i);
         return __uint_as_float(static_cast<uint32_t>(h) << 16);
     }
@@ -219,6 +248,7 @@ __device__ __noinline__ Partial reduce_segment_slow(const RowGeom& g, int seg, f
 // Fast path: cp.async ring + packed fp32x2 arithmetic.
 
 __device__ __forceinline__ void cp_async16(uint32_t saddr, const void* gptr) {
+    if (!debug_ok(gptr, 16)) return;
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(saddr), "l"(gptr) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
@@ -612,7 +642,7 @@ __device__ __forceinline__ Partial reduce_segment(const RowGeom& g, int seg, flo
         int iv = warp_min_int(t.rmax == r.m ? t.ivec : kIntMax);
         if (iv != kIntMax) {
             float x[EPV];
-            unpack_masked<DT>(g.base[iv], iv, g, x);
+            unpack_masked<DT>(ld_vec(g.base + iv), iv, g, x);
             int first = -1;
 #pragma unroll
             for (int j = EPV - 1; j >= 0; --j)

@@ -241,7 +241,7 @@ struct SoftmaxWeights {
     float c, M;
     float thr = -INFINITY;   // logits below it carry no weight (truncated distributions)
     typedef uint4 Raw;
-    __device__ __forceinline__ Raw load(int vi) const { return g.base[vi]; }
+    __device__ __forceinline__ Raw load(int vi) const { return ld_vec(g.base + vi); }
     __device__ __forceinline__ void weights(int vi, const Raw& raw, float (&w)[ElemTraits<DT>::kEPV]) const {
         constexpr int EPV = ElemTraits<DT>::kEPV;
         float x[EPV];

@@ -56,8 +56,8 @@ struct TreeWeights {
     }
     __device__ __forceinline__ Raw load(int vi) const {
         Raw r;
-        r.t = __ldg(gt.base + vi);
-        r.q = (nrej > 0 && gq.pre == gt.pre) ? __ldg(gq.base + vi) : make_uint4(0, 0, 0, 0);
+        r.t = ld_vec(gt.base + vi);
+        r.q = (nrej > 0 && gq.pre == gt.pre) ? ld_vec(gq.base + vi) : make_uint4(0, 0, 0, 0);
         return r;
     }
     __device__ __forceinline__ void weights(int vi, const Raw& raw, float (&w)[ElemTraits<DT>::kEPV]) const {

@@ -38,8 +38,8 @@ struct ResidualWeights {
     struct Raw { uint4 t, q; };
     __device__ __forceinline__ Raw load(int vi) const {
         Raw r;
-        r.t = __ldg(gt.base + vi);
-        r.q = (!bonus && gq.pre == gt.pre) ? __ldg(gq.base + vi) : make_uint4(0, 0, 0, 0);
+        r.t = ld_vec(gt.base + vi);
+        r.q = (!bonus && gq.pre == gt.pre) ? ld_vec(gq.base + vi) : make_uint4(0, 0, 0, 0);
         return r;
     }
     __device__ __forceinline__ void operator()(int vi, float (&w)[ElemTraits<DT>::kEPV]) const {
