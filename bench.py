@@ -34,12 +34,13 @@ METRIC = "logits GB/s (% of B200 HBM peak) for draft-step+verify; us/step at B=1
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of row_stats_kernel<bf16> per algorithmic byte, from an
-# ncu capture of a 1056-row launch (332.3 MB moved for 321.2 MB of logits); traffic grows in
-# proportion to the rows, so a full launch is scaled by its bytes
-ROW_STATS_TRAFFIC_PER_ALGORITHMIC_BYTE = 332.34 / 321.16
-# the same for draft_step_kernel<f32, sampling>, from a capture of 128-row launches (132.2 MB read and
-# 7.0 MB written for 131.1 MB of logits)
-DRAFT_F32_TRAFFIC_PER_ALGORITHMIC_BYTE = 139.17 / 131.07
+# ncu capture of a 1056-row launch (321.20 MB read and 10.73 MB written for 321.16 MB of logits); traffic
+# grows in proportion to the rows, so a full launch is scaled by its bytes
+ROW_STATS_TRAFFIC_PER_ALGORITHMIC_BYTE = 331.93 / 321.16
+# the same for draft_step_kernel<f32, sampling> in the launch shape timed on `stress` (clusters of 2,
+# three blocks per SM), from a capture of 160-row launches (166.44 MB read and 9.27 MB written for
+# 163.84 MB of logits)
+DRAFT_F32_TRAFFIC_PER_ALGORITHMIC_BYTE = 175.71 / 163.84
 
 
 def describe(w, B=None):
