@@ -429,6 +429,8 @@ def pair_stats_leg(ctx, torch, rnd, peak, reps=10):
     w, B, V = rnd.w, rnd.B, rnd.V
     if not w.T > 0:
         return None
+    rnd.step()          # the draft rows' normalisers of the plain round (other legs reuse the buffer)
+    torch.cuda.synchronize()
     dev = rnd.d_q.device
     cu = np.concatenate([[0], np.cumsum(rnd.lens.astype(np.int64) + 1)])
     q_idx = np.concatenate([np.arange(rnd.lens[k]) * B + k for k in range(B)])
@@ -465,6 +467,82 @@ def pair_stats_leg(ctx, torch, rnd, peak, reps=10):
                      "mean_beta": float(o[:, 0].mean()), "mean_H_q": float(o[:, 1].mean()),
                      "nan_outputs": int(np.isnan(o).sum())}
     return res
+
+
+def tree_leg(ctx, torch, reps=20):
+    """svip_verify_tree on synthetic candidate trees: 64 sequences, binary trees of depth 3 (14 candidate
+    nodes: the two most likely tokens of every node's draft row), V = 32000 bf16, target = draft + N(0, 0.5^2)."""
+    B, V, T = 64, 32000, 1.0
+    parent = [-1, -1] + [i // 2 - 1 for i in range(4, 16)]       # nodes 2k, 2k+1 are the children of node k-1
+    N = len(parent)
+    g = torch.Generator(device="cuda").manual_seed(20241118)
+    q = torch.randn(B * (N + 1), V, device="cuda", generator=g) * 2.0
+    t = q + torch.randn(B * (N + 1), V, device="cuda", generator=g) * 0.5
+    top2 = q.view(B, N + 1, V).topk(2, dim=2).indices                 # [B, N+1, 2]
+    par = torch.tensor(parent, device="cuda")
+    tokens = torch.stack([top2[:, parent[i] + 1, i % 2] for i in range(N)], dim=1).to(torch.int32).contiguous()
+    parent_t = par.to(torch.int32).repeat(B, 1).contiguous()
+    qb = q.to(torch.bfloat16).view(torch.int16); tb = t.to(torch.bfloat16).view(torch.int16)
+    u = torch.rand(B, N + 1, device="cuda", generator=g)
+    n_acc = torch.zeros(B, dtype=torch.int32, device="cuda"); path = torch.zeros(B, N, dtype=torch.int32, device="cuda")
+    nxt = torch.zeros(B, dtype=torch.int32, device="cuda")
+    st = torch.cuda.current_stream().cuda_stream
+    call = ctx.bind("verify_tree", tokens, parent_t, qb, V, None, tb, V, 1, B, N, V, T, u, n_acc, path, nxt, st)
+    before = ctx.launch_count()
+    call()
+    kernels = ctx.launch_count() - before
+    torch.cuda.synchronize()
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    us = 1000.0 * e0.elapsed_time(e1) / reps
+    rows_bytes = 2 * B * (N + 1) * V * 2
+    return {"sequences": B, "nodes": N, "V": V, "dtype": "bf16", "us_per_call": us, "kernels": kernels,
+            "mean_accepted": float(n_acc.float().mean()), "normaliser_passes_GBps": rows_bytes / (us * 1e-6) / 1e9,
+            "note": "two passes of row statistics over all 2 x B x (N+1) rows, then the walk (a chain of passes over "
+                    "single row pairs: latency-bound)"}
+
+
+def vocab_parallel_leg(ctx, torch, rnd, peak, G=8, reps=20):
+    """One rank's share of a vocabulary-parallel draft step over the first draft launch of the round: the rows'
+    columns cut into G shards, this rank holding shard 0 (svip_vp_partial on the shard, svip_vp_combine on the G
+    partials, svip_vp_locate on the shard).  The two small collectives between them need G GPUs and are not timed."""
+    from paper_2411_18462_b200 import vocab_parallel as VP
+    w, V = rnd.w, rnd.V
+    B = int(rnd.active[0])
+    dev = rnd.d_q.device
+    sp = rnd.stream
+    partials = torch.zeros(G, B, 4, device=dev)
+    for r in range(G):
+        lo, hi = VP.shard_bounds(V, G, r)
+        ctx.vp_partial(rnd.d_q.data_ptr() + lo * rnd.esz, rnd.dt, B, hi - lo, V, w.T, lo, partials[r], sp)
+    lo, hi = VP.shard_bounds(V, G, 0)
+    ent = torch.zeros(B, device=dev); stop = torch.zeros(B, dtype=torch.uint8, device=dev)
+    tok = torch.zeros(B, dtype=torch.int32, device=dev); owner = torch.zeros(B, dtype=torch.int32, device=dev)
+    tgt = torch.zeros(B, device=dev); act = torch.zeros(B, dtype=torch.uint8, device=dev)
+    calls = [ctx.bind("vp_partial", rnd.d_q, rnd.dt, B, hi - lo, V, w.T, lo, partials[0], sp),
+             ctx.bind("vp_combine", partials, G, 0, B, w.T, w.h, rnd.d_ud, ent, stop, tok, owner, tgt, act, sp)]
+    if w.T > 0:
+        calls.append(ctx.bind("vp_locate", rnd.d_q, rnd.dt, B, hi - lo, V, w.T, tgt, act, lo, tok, sp))
+    for c in calls:
+        c()
+    torch.cuda.synchronize()
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        for c in calls:
+            c()
+    e1.record()
+    torch.cuda.synchronize()
+    us = 1000.0 * e0.elapsed_time(e1) / reps
+    owned = int(act.sum().item())
+    nbytes = (B + owned) * (hi - lo) * rnd.esz          # the shard once, the owned rows' shard once more
+    return {"ranks_emulated": G, "rows": B, "shard_columns": hi - lo, "rows_owned_by_this_rank": owned,
+            "us_per_step_on_one_rank": us, "shard_GBps": nbytes / (us * 1e-6) / 1e9,
+            "frac_of_measured_peak": nbytes / (us * 1e-6) / 1e9 / peak, "kernels": len(calls)}
 
 
 CDF_TOL = 1e-5        # a sampled token may differ from the oracle's only across a CDF boundary closer than this
@@ -772,10 +850,13 @@ def run_ours(args):
             line["truncated"] = truncated_round(ctx, torch, rnd)
         except Exception as exc:
             line["truncated"] = {"error": repr(exc)}
-        try:
-            line["pair_stats"] = pair_stats_leg(ctx, torch, rnd, peak)
-        except Exception as exc:
-            line["pair_stats"] = {"error": repr(exc)}
+        for key, leg in (("pair_stats", lambda: pair_stats_leg(ctx, torch, rnd, peak)),
+                         ("vocab_parallel", lambda: vocab_parallel_leg(ctx, torch, rnd, peak)),
+                         ("tree", lambda: tree_leg(ctx, torch))):
+            try:
+                line[key] = leg()
+            except Exception as exc:
+                line[key] = {"error": repr(exc)}
     if not args.no_cpu_baseline and not args.skip_extras:
         line["cpu_baseline"], line["checks"] = cpu_baseline(w, gpu_results)
     if not args.skip_extras and world == 1 and args.batch is None:
