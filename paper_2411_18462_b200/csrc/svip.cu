@@ -189,6 +189,15 @@ cudaError_t debug_ranges(const svip_ctx* ctx, cudaStream_t st, const void* p0, s
 #define SVIP_DEBUG_RANGES(...) do { } while (0)
 #endif
 
+// The candidate path of the threshold kernel reads every row twice.  A launch that fits in L2 finds its rows
+// there the second time; a larger one takes its first bound from the first half of every warp segment instead
+// of all of it (measured on 256 x 256000 fp32 rows, top-k 50: a half or a third 86 us per launch, all 97, a
+// quarter 102 and an eighth 144, because the looser bound lets more candidates in than the counting finish holds).
+int threshold_sample_den(long rows, int V, int dtype) {
+    const long bytes = rows * static_cast<long>(V) * (dtype == SVIP_BF16 ? 2 : 4);
+    return bytes > (48L << 20) ? 2 : 1;
+}
+
 bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 float scale_for(float T) { return static_cast<float>(1.4426950408889634 / (T > 0.f ? static_cast<double>(T) : 1.0)); }
@@ -421,6 +430,7 @@ int svip_row_threshold(svip_ctx* ctx, const void* logits, svip_dtype dtype, int 
     if (stats && !aligned_to(stats, 8)) return SVIP_ERR_INVALID_ARG;
     a.uniforms = nullptr; a.active = nullptr; a.thresh = 0.f; a.token = nullptr; a.entropy = nullptr;
     a.stop = nullptr; a.status = ctx->status;
+    a.sample_den = threshold_sample_den(n_rows, V, dtype);
     const int S = pick_cluster(ctx, n_rows, V, dtype);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = dtype == SVIP_BF16 ? launch_clustered(row_threshold_kernel<kBF16>, n_rows, S, a, st, kRingBytes)
@@ -449,6 +459,7 @@ int svip_draft_step_truncated(svip_ctx* ctx, const void* logits, svip_dtype dtyp
     a.stats = reinterpret_cast<float2*>(row_stats);
     a.uniforms = uniforms; a.active = active; a.thresh = thresh; a.token = token; a.entropy = entropy;
     a.stop = stop; a.status = ctx->status;
+    a.sample_den = threshold_sample_den(B, V, dtype);
     const int S = pick_cluster(ctx, B, V, dtype);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = dtype == SVIP_BF16

@@ -47,6 +47,7 @@ struct ThresholdArgs {
     float* entropy;          // [rows] out
     uint8_t* stop;           // [rows] out
     unsigned* status;        // device status word
+    int sample_den;          // candidate path: the first bound comes from 1/sample_den of every warp segment (1: all)
 };
 
 // Monotone image of a float: a < b  <=>  key(a) < key(b).  NaN counts as -inf.
@@ -62,13 +63,14 @@ __device__ __forceinline__ float key_value(uint32_t key) {
 }
 
 // Streams segment `seg` of the row with the calling warp and hands every vector to f(x, vi), with
-// the elements outside the row set to -inf.
+// the elements outside the row set to -inf.  den > 1: only the first 1/den of the segment (rounded up).
 template <int DT, class F>
-__device__ __forceinline__ void stream_segment(const RowGeom& g, int seg, int lane, uint32_t slot0, F&& f) {
+__device__ __forceinline__ void stream_segment(const RowGeom& g, int seg, int lane, uint32_t slot0, F&& f, int den = 1) {
     constexpr int EPV = ElemTraits<DT>::kEPV;
     constexpr uint32_t kSlotStride = kThreads * 16;
     int v_lo, v_hi;
     seg_range(g, seg, v_lo, v_hi);
+    if (den > 1) v_hi = min(v_hi, v_lo + (v_hi - v_lo + den - 1) / den);
     const int vi0 = v_lo + lane;
     const int n = v_hi > vi0 ? (v_hi - vi0 + 31) >> 5 : 0;
     const uint4* src = g.base + vi0;
@@ -537,10 +539,16 @@ __device__ __forceinline__ bool draft_from_candidates(SelectShared& sh, const ui
 // been written then and the caller takes the radix descent over the full row.
 // kDraft also keeps the positions of the candidates and lets block 0 finish the whole draft step from
 // them (`drafted`, the same in every block); `scratch` is the streaming ring, free by then.
+// sample_den > 1: pass 1 reads only the first 1/sample_den of every warp segment.  The k-th largest of the
+// thread maxima of that part is still k distinct elements of the row, hence still a lower bound of tau_k,
+// only a looser one (about sample_den * k candidates instead of k); pass 2 then finds that part in L2, so the
+// row crosses HBM 1 + 1 / sample_den times instead of twice.  *overflow tells a set that did not fit from a set
+// that is too small.
 template <int DT, bool kDraft>
 __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const RowGeom& g, int S, int rank, int tid,
                                                uint32_t slot0, const ThresholdArgs& a, bool use_p, SelectShared& sh,
-                                               uint32_t& key_out, void* scratch, bool& drafted) {
+                                               uint32_t& key_out, void* scratch, bool& drafted, int sample_den,
+                                               bool* overflow) {
     constexpr int EPV = ElemTraits<DT>::kEPV;
     constexpr int kLevels = DT == kBF16 ? 2 : 4;
     constexpr int kCap = kDraft ? kPoolCapDraft : kPoolCap;
@@ -556,7 +564,7 @@ __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const
         any = true;
 #pragma unroll
         for (int j = 0; j < EPV; ++j) best = fmaxf(best, x[j]);
-    });
+    }, sample_den);
     sh.lane_key[tid] = any ? order_key(best) : 0u;
     if (tid == 0) sh.cand_n = 0;
     cluster.sync();
@@ -604,6 +612,7 @@ __device__ __forceinline__ bool candidate_path(cg::cluster_group& cluster, const
         }
     }
     cluster.sync();     // the peers have read this block's candidates
+    *overflow = !fits;
     if (!fits || total < a.top_k) return false;
     const int row = static_cast<int>(blockIdx.x / S);
     if (total <= kSmallPool) {
@@ -709,8 +718,14 @@ __global__ void __launch_bounds__(kThreads, 2) row_threshold_kernel(ThresholdArg
     // a small k against the number of threads of the cluster: two passes and a handful of candidates
     if (use_k && a.top_k <= (S * kThreads) / 4) {
         uint32_t key_t = 0;
-        bool drafted = false;
-        if (candidate_path<DT, kDraft>(cluster, g, S, rank, tid, slot0, a, use_p, sh, key_t, ring, drafted)) {
+        bool drafted = false, overflow = false;
+        // the bound from a part of the row first (large launches); if that lets too many candidates in, from all of it
+        bool done = candidate_path<DT, kDraft>(cluster, g, S, rank, tid, slot0, a, use_p, sh, key_t, ring, drafted,
+                                               a.sample_den, &overflow);
+        if (!done && overflow && a.sample_den > 1)
+            done = candidate_path<DT, kDraft>(cluster, g, S, rank, tid, slot0, a, use_p, sh, key_t, ring, drafted, 1,
+                                              &overflow);
+        if (done) {
             const float thr = key_t ? key_value(key_t) : neg_inf();
             if (rank == 0 && tid == 0) a.thr[row] = thr;
             if (kDraft && !drafted) draft_at_threshold<DT>(a, cluster, S, rank, row, tid, g, slot0, thr);
