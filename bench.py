@@ -469,6 +469,52 @@ def pair_stats_leg(ctx, torch, rnd, peak, reps=10):
     return res
 
 
+def graph_loop_round(ctx, torch, rnd, reps=20):
+    """The same round as one CUDA graph whose drafting phase is a loop on the device (Algorithm 1's do-while):
+    every iteration is one svip_draft_step_at over all sequences at their own positions (finished ones masked)
+    and the entropy policy, which also decides the loop; then packing from the device-side draft lengths and
+    svip_verify.  No host round trip and no host launch per draft position."""
+    w, B, V, K = rnd.w, rnd.B, rnd.V, rnd.K
+    if not w.T > 0:
+        return None
+    dev = rnd.d_q.device
+    st = torch.cuda.Stream()
+    dlen = torch.zeros(B, dtype=torch.int32, device=dev); act = torch.ones(B, dtype=torch.uint8, device=dev)
+    nact = torch.zeros(1, dtype=torch.int32, device=dev); stop1 = torch.zeros(B, dtype=torch.uint8, device=dev)
+    ENTROPY = 0
+    rnd.step()
+    torch.cuda.synchronize()
+    want_nacc = rnd.d_nacc.clone(); want_next = rnd.d_next.clone()
+    with torch.cuda.stream(st):
+        ctx.graph_begin(st)
+        ctx.policy_update(ENTROPY, None, dlen, None, act, B, w.K_max, st)
+        body = ctx.graph_loop_begin(st, nact, w.K_max)
+        ctx.draft_step_at(rnd.d_q, rnd.dt, B, V, V, B * V, dlen, B, w.T, w.h, rnd.d_ud, act, rnd.d_tok, rnd.d_ent,
+                          stop1, rnd.d_stats, body)
+        ctx.policy_advance(ENTROPY, stop1, None, dlen, act, B, w.K_max, nact, body)
+        ctx.graph_loop_end()
+        ctx.pack_ragged(dlen, B, w.K_max, rnd.d_cu, None, None, st)
+        ctx.verify(rnd.d_tok, rnd.d_q, V, rnd.d_stats, 1, B, rnd.d_t, V, rnd.dt, rnd.d_cu, B, w.K_max, rnd.Rp, V, w.T,
+                   rnd.d_uv, rnd.d_nacc, rnd.d_next, st)
+        g = ctx.graph_end(st)
+        for _ in range(3):
+            g.launch(st)
+        st.synchronize()
+        same = bool(torch.equal(dlen.cpu(), torch.from_numpy(rnd.lens)) and torch.equal(rnd.d_nacc, want_nacc)
+                    and torch.equal(rnd.d_next, want_next))
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(st)
+        for _ in range(reps):
+            g.launch(st)
+        e1.record(st)
+        st.synchronize()
+        us = 1000.0 * e0.elapsed_time(e1) / reps
+        g.destroy()
+    nbytes, _ = rnd.logits_bytes()
+    return {"us_per_round": us, "logits_GBps": nbytes / (us * 1e-6) / 1e9, "loop_iterations": int(rnd.lens.max()),
+            "same_results_as_host_driven_round": same}
+
+
 def tree_leg(ctx, torch, reps=20):
     """svip_verify_tree on synthetic candidate trees: 64 sequences, binary trees of depth 3 (14 candidate
     nodes: the two most likely tokens of every node's draft row), V = 32000 bf16, target = draft + N(0, 0.5^2)."""
@@ -761,6 +807,11 @@ def other_workload(ctx, torch, name, rank, peak, peak_kind, steps):
            "stop_flags_match_draft_lengths": bool(m["stops_ok"]) if name == "ragged" else None,
            "status_word": m["status"],
            "roofline": {k: first[k] for k in keep}, "roofline_other": {k: second[k] for k in keep}}
+    if name == "ragged":
+        try:
+            out["device_loop_graph"] = graph_loop_round(ctx, torch, rnd)
+        except Exception as exc:
+            out["device_loop_graph"] = {"error": repr(exc)}
     del rnd
     torch.cuda.empty_cache()
     return out
