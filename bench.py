@@ -849,7 +849,7 @@ def run_ours(args):
     total_ms, total_bytes = sharding.aggregate(m["local_ms"], step_bytes * args.steps, device=torch.device("cuda", dev))
 
     # end to end: host buffers in, results out, every step
-    e2e_steps = 0 if args.skip_extras else max(1, min(args.steps, 5))
+    e2e_steps = 0 if (args.skip_extras or args.only_leg) else max(1, min(args.steps, 5))
     h2d = d2h = 0
     torch.cuda.synchronize()
     if world > 1:
@@ -892,6 +892,14 @@ def run_ours(args):
         "gpu_launches": m["launches"], "clocks": clocks,
     }
     gpu_results = rnd.results_by_sequence()
+    if args.only_leg:       # for profiling one of the extra legs without the others' launches
+        legs = {"pair_stats": lambda: pair_stats_leg(ctx, torch, rnd, peak, reps=2),
+                "vocab_parallel": lambda: vocab_parallel_leg(ctx, torch, rnd, peak, reps=2),
+                "tree": lambda: tree_leg(ctx, torch, reps=2),
+                "truncated": lambda: truncated_round(ctx, torch, rnd, reps=2)}
+        line[args.only_leg] = legs[args.only_leg]()
+        print(json.dumps(line))
+        return
     if not args.skip_extras:
         try:
             line["b1"] = b1_latency(ctx, torch)
@@ -985,6 +993,8 @@ def main():
                     help="sequences per GPU instead of the published batch size (smaller cases for profiling)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only-leg", default=None, choices=["pair_stats", "vocab_parallel", "tree", "truncated"],
+                    help="after the timed region run just this extra leg, briefly (for profiling it)")
     ap.add_argument("--skip-extras", action="store_true",
                     help="only the timed region: no end-to-end leg, no B=1 latency, no CPU baseline (for profiling)")
     args = ap.parse_args()
