@@ -329,6 +329,29 @@ int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits
                 const float* uniforms, int32_t* n_accepted, int32_t* next_token, void* stream);
 
 /*
+ * svip_verify with the same arguments, results and error behaviour, reading
+ * less: the accept tests of a sequence end at its first rejection (Algorithm 1,
+ * verify loop), so the target rows after it are never needed.  One group of
+ * thread blocks per sequence reads the sequence's target rows in order and
+ * stops at the first rejection (or after the bonus row); rows after it are not
+ * read.  The rows of one sequence are read one after another, so this pays off
+ * where the batch is large enough to fill the GPU with sequences (B of a few
+ * dozen and more) and rejections come early; for a few sequences with long
+ * accepted runs svip_verify, which reads all rows at once, is faster.
+ * Same arithmetic as svip_verify; the rows are cut over another number of
+ * thread blocks, so the fp32 normalisers can differ from svip_verify's in
+ * their last bits (a result can differ only where a draw lies within fp32
+ * rounding of a boundary).  q_stats == NULL costs one more pass over all draft
+ * rows first.
+ */
+int svip_verify_early_exit(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits,
+                           long q_row_stride, const float* q_stats, long q_seq_stride,
+                           long q_pos_stride, const void* target_logits, long t_row_stride,
+                           svip_dtype dtype, const int32_t* cu_rows, int B, int K,
+                           int n_target_rows, int V, float T, const float* uniforms,
+                           int32_t* n_accepted, int32_t* next_token, void* stream);
+
+/*
  * Vocabulary-parallel draft step: the V logits of every row are sharded over G
  * ranks (a tensor-parallel LM head), rank g holding the V_shard columns that
  * start at vocab_offset.  The paper's draft step (Algorithm 1 inner loop, Eq. 7)

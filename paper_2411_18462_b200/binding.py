@@ -69,6 +69,9 @@ def library():
     L.svip_verify.restype = i32
     L.svip_verify.argtypes = [vp, vp, vp, lng, vp, lng, lng, vp, lng, i32, vp, i32, i32, i32, i32, f32,
                               vp, vp, vp, vp]
+    L.svip_verify_early_exit.restype = i32
+    L.svip_verify_early_exit.argtypes = [vp, vp, vp, lng, vp, lng, lng, vp, lng, i32, vp, i32, i32, i32, i32, f32,
+                              vp, vp, vp, vp]
     L.svip_profile_enable.restype = i32
     L.svip_profile_enable.argtypes = [vp, i32]
     L.svip_profile_read.restype = i32
@@ -270,6 +273,16 @@ class Context:
                                      _ptr(target_logits), int(t_row_stride), int(dtype), _ptr(cu_rows),
                                      int(B), int(K), int(n_target_rows), int(V), float(T), _ptr(uniforms),
                                      _ptr(n_accepted), _ptr(next_token), _stream(stream)), self._h)
+
+    def verify_early_exit(self, draft_tokens, q_logits, q_row_stride, q_stats, q_seq_stride, q_pos_stride,
+                          target_logits, t_row_stride, dtype, cu_rows, B, K, n_target_rows, V, T, uniforms,
+                          n_accepted, next_token, stream=None):
+        _check(library().svip_verify_early_exit(self._h, _ptr(draft_tokens), _ptr(q_logits), int(q_row_stride),
+                                                _ptr(q_stats), int(q_seq_stride), int(q_pos_stride),
+                                                _ptr(target_logits), int(t_row_stride), int(dtype), _ptr(cu_rows),
+                                                int(B), int(K), int(n_target_rows), int(V), float(T),
+                                                _ptr(uniforms), _ptr(n_accepted), _ptr(next_token),
+                                                _stream(stream)), self._h)
 
     def vp_partial(self, logits, dtype, B, V_shard, row_stride, T, vocab_offset, partial, stream=None):
         _check(library().svip_vp_partial(self._h, _ptr(logits), int(dtype), int(B), int(V_shard), int(row_stride),

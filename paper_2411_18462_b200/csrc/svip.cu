@@ -257,7 +257,9 @@ int svip_create(svip_ctx** out, int device, int max_rows) {
             (const void*)row_stats_kernel<kBF16, 1, true>, (const void*)row_stats_kernel<kF32, 1, true>,
             (const void*)verify_finish_kernel<kBF16, true>, (const void*)verify_finish_kernel<kF32, true>,
             (const void*)pair_stats_kernel<kBF16>, (const void*)pair_stats_kernel<kF32>,
-            (const void*)pair_stats_kernel<kBF16, true>, (const void*)pair_stats_kernel<kF32, true>};
+            (const void*)pair_stats_kernel<kBF16, true>, (const void*)pair_stats_kernel<kF32, true>,
+            (const void*)verify_scan_kernel<kBF16, false>, (const void*)verify_scan_kernel<kF32, false>,
+            (const void*)verify_scan_kernel<kBF16, true>, (const void*)verify_scan_kernel<kF32, true>};
         for (const void* k : ringed)
             if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes) != cudaSuccess)
                 rc = SVIP_ERR_CUDA;
@@ -490,7 +492,7 @@ static int verify_impl(svip_ctx* ctx, const int32_t* draft_tokens, const void* q
                        long t_row_stride, svip_dtype dtype, const int32_t* cu_rows, int B, int K,
                        int n_target_rows, int V, float T, const float* uniforms, int32_t* n_accepted,
                        int32_t* next_token, void* stream, const float* q_thr, const float* p_thr,
-                       const float* p_stats_user) {
+                       const float* p_stats_user, bool early_exit = false) {
     if (!ctx || !draft_tokens || !target_logits || !n_accepted || !next_token) return SVIP_ERR_INVALID_ARG;
     const bool truncated = q_thr != nullptr;
     if (dtype != SVIP_F32 && dtype != SVIP_BF16) return SVIP_ERR_UNSUPPORTED;
@@ -526,6 +528,45 @@ static int verify_impl(svip_ctx* ctx, const int32_t* draft_tokens, const void* q
     s.out_partial = nullptr; s.idx_offset = 0; s.thr = p_thr;
     int S = pick_cluster(ctx, n_target_rows, V, dtype);
     const bool timed = ctx->profiling && !ctx->capturing && ctx->prof_used < kProfilePairs;
+    if (early_exit) {
+        // the draft rows' normalisers first (the accept test of a position needs them), then one cluster
+        // per sequence walks the target rows up to the first rejection
+        if (sampling && !q_stats) {
+            StatsArgs d = s;
+            d.logits = q_logits; d.row_stride = q_row_stride; d.draft_rows = 1;
+            d.out_stats = ctx->q_stats; d.out_argmax = nullptr; d.thr = nullptr;
+            const int Sd = pick_cluster(ctx, n_target_rows - B, V, dtype);
+            e = dtype == SVIP_BF16 ? launch_clustered(row_stats_kernel<kBF16, 1>, static_cast<long>(B) * K, Sd, d, st, kRingBytes)
+                                   : launch_clustered(row_stats_kernel<kF32, 1>, static_cast<long>(B) * K, Sd, d, st, kRingBytes);
+            if (e != cudaSuccess) return cuda_fail(ctx, e);
+            ctx->launches += 1;
+        }
+        ScanArgs w;
+        w.draft_tokens = draft_tokens; w.q_logits = q_logits; w.q_row_stride = q_row_stride;
+        w.q_stats_user = reinterpret_cast<const float2*>(q_stats); w.q_stats_ws = ctx->q_stats;
+        w.q_seq_stride = q_seq_stride; w.q_pos_stride = q_pos_stride; w.t_logits = target_logits;
+        w.t_row_stride = t_row_stride; w.p_stats = ctx->p_stats; w.cu = cu_rows; w.K = K; w.V = V; w.c = c;
+        w.uniforms = uniforms; w.n_accepted = n_accepted; w.next_token = next_token; w.status = ctx->status;
+        // the rows of a sequence are read one after another: a row is cut over enough blocks that the chain
+        // of the longest accepted run stays short (each block at most 128 KB of a row)
+        int Sw = pick_cluster(ctx, B, V, dtype);
+        if (ctx->cluster_override == 0) {
+            const long row_bytes = static_cast<long>(V) * static_cast<long>(esz);
+            while (Sw < kMaxCluster && row_bytes / Sw > (128L << 10)) Sw *= 2;
+            if (Sw > kMaxCluster) Sw = kMaxCluster;
+        }
+        if (timed) cudaEventRecord(ctx->prof_start[ctx->prof_used], st);
+        if (sampling)
+            e = dtype == SVIP_BF16 ? launch_clustered(verify_scan_kernel<kBF16, false>, B, Sw, w, st, kRingBytes)
+                                   : launch_clustered(verify_scan_kernel<kF32, false>, B, Sw, w, st, kRingBytes);
+        else
+            e = dtype == SVIP_BF16 ? launch_clustered(verify_scan_kernel<kBF16, true>, B, Sw, w, st, kRingBytes)
+                                   : launch_clustered(verify_scan_kernel<kF32, true>, B, Sw, w, st, kRingBytes);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        ctx->launches += 1;
+        if (timed) cudaEventRecord(ctx->prof_stop[ctx->prof_used++], st);
+        if (!sampling) return SVIP_OK;
+    } else {
     if (timed) cudaEventRecord(ctx->prof_start[ctx->prof_used], st);
     if (p_stats_user)
         e = cudaSuccess;   // the caller already holds (m, Z) of every target row
@@ -542,6 +583,7 @@ static int verify_impl(svip_ctx* ctx, const int32_t* draft_tokens, const void* q
     if (!p_stats_user) ctx->launches += 1;
     if (timed) cudaEventRecord(ctx->prof_stop[ctx->prof_used++], st);
 
+    }
     if (!sampling) {
         GreedyArgs g;
         g.draft_tokens = draft_tokens; g.p_argmax = ctx->p_argmax; g.cu = cu_rows;
@@ -553,7 +595,7 @@ static int verify_impl(svip_ctx* ctx, const int32_t* draft_tokens, const void* q
         return SVIP_OK;
     }
 
-    if (!q_stats) {
+    if (!q_stats && !early_exit) {
         StatsArgs d = s;
         d.logits = q_logits; d.row_stride = q_row_stride; d.draft_rows = 1;
         d.out_stats = ctx->q_stats; d.out_argmax = nullptr; d.thr = q_thr;
@@ -578,6 +620,7 @@ static int verify_impl(svip_ctx* ctx, const int32_t* draft_tokens, const void* q
     f.cu = cu_rows; f.K = K; f.V = V; f.c = c;
     f.uniforms = uniforms; f.n_accepted = n_accepted; f.next_token = next_token; f.status = ctx->status;
     f.p_thr = p_thr; f.q_thr = q_thr;
+    f.n_acc_in = early_exit ? n_accepted : nullptr;
     // up to two rows per sequence are streamed: long rows are cut finer than the one-wave policy
     // asks for (this kernel runs for many microseconds, so several waves are fine)
     int Sf = pick_cluster(ctx, B, V, dtype);
@@ -605,6 +648,16 @@ int svip_verify(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits
     return verify_impl(ctx, draft_tokens, q_logits, q_row_stride, q_stats, q_seq_stride, q_pos_stride,
                        target_logits, t_row_stride, dtype, cu_rows, B, K, n_target_rows, V, T, uniforms,
                        n_accepted, next_token, stream, nullptr, nullptr, nullptr);
+}
+
+int svip_verify_early_exit(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits, long q_row_stride,
+                           const float* q_stats, long q_seq_stride, long q_pos_stride, const void* target_logits,
+                           long t_row_stride, svip_dtype dtype, const int32_t* cu_rows, int B, int K,
+                           int n_target_rows, int V, float T, const float* uniforms, int32_t* n_accepted,
+                           int32_t* next_token, void* stream) {
+    return verify_impl(ctx, draft_tokens, q_logits, q_row_stride, q_stats, q_seq_stride, q_pos_stride,
+                       target_logits, t_row_stride, dtype, cu_rows, B, K, n_target_rows, V, T, uniforms,
+                       n_accepted, next_token, stream, nullptr, nullptr, nullptr, true);
 }
 
 int svip_verify_filtered(svip_ctx* ctx, const int32_t* draft_tokens, const void* q_logits, long q_row_stride,

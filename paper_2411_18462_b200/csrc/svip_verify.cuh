@@ -25,6 +25,7 @@ struct FinishArgs {
     unsigned* status;
     const float* p_thr;           // kThr: truncation threshold of every target row
     const float* q_thr;           // kThr: ... of every draft row (indexed like the draft tokens)
+    const int32_t* n_acc_in;      // not NULL: the first rejection of every sequence is already known
 };
 
 // Weights max(0, p - q) of Algorithm 4 (or p alone for the bonus token) for one vector.
@@ -183,6 +184,22 @@ __device__ __forceinline__ float residual_segment_sum(const ResidualWeights<DT>&
     return acc;
 }
 
+// Algorithm 2 for one position: r < min(1, p(x)/q(x)), from the two logits of the drafted token and the
+// (max, Z) of the two rows.  p(x)/q(x) = 2^(ap - aq) * Zq / Zp, from the difference of the two log2
+// arguments, so that a token however unlikely under both models keeps its ratio (no underflow).  No
+// division: a ratio >= 1 accepts every r in [0,1); p(x) == 0 accepts none; q(x) == 0 < p(x) is a ratio of
+// +inf.  `p_out` / `q_out`: the token lies outside the truncated support of that side.
+__device__ __forceinline__ bool accept_test(float tv, float dv, float2 ps, float2 qs, float c, float r,
+                                            bool p_out, bool q_out) {
+    const float ap = __fmaf_rn(tv, c, -__fmul_rn(ps.x, c));
+    const float aq = __fmaf_rn(dv, c, -__fmul_rn(qs.x, c));
+    const bool p_zero = p_out || !(tv > neg_inf());   // NaN counts as -inf
+    const bool q_zero = q_out || !(dv > neg_inf());
+    const float d = fminf(fmaxf(ap - aq, -126.f), 126.f);
+    const float num = __fmul_rn(exp2f(d), qs.y);
+    return !p_zero && (q_zero || num >= ps.y || __fmul_rn(r, ps.y) < num);
+}
+
 struct FinishShared {
     int n_acc;
     SegPick pick;
@@ -213,7 +230,9 @@ __global__ void __launch_bounds__(kThreads, 2) verify_finish_kernel(FinishArgs a
     const char* ql = static_cast<const char*>(a.q_logits);
 
     // Algorithm 2 at every position at once; the first rejection is the lowest set bit.
-    if (warp == 0) {
+    if (a.n_acc_in) {
+        if (tid == 0) fs.n_acc = min(max(a.n_acc_in[i], 0), Ki);
+    } else if (warp == 0) {
         int n_acc = Ki;
         for (int j0 = 0; j0 < Ki; j0 += 32) {
             int j = j0 + lane;
@@ -227,21 +246,12 @@ __global__ void __launch_bounds__(kThreads, 2) verify_finish_kernel(FinishArgs a
                     float dv = E::load_one(ql + static_cast<size_t>(dr) * a.q_row_stride * E::kBytes, x);
                     float2 ps = a.p_stats[row0 + j];
                     float2 qs = a.q_stats_user ? a.q_stats_user[dr] : a.q_stats_ws[row0 + j];
-                    // p(x)/q(x) = 2^(ap - aq) * Zq / Zp, from the difference of the two log2 arguments, so
-                    // that a token however unlikely under both models keeps its ratio (no underflow)
-                    const float ap = __fmaf_rn(tv, a.c, -__fmul_rn(ps.x, a.c));
-                    const float aq = __fmaf_rn(dv, a.c, -__fmul_rn(qs.x, a.c));
-                    bool p_zero = !(tv > neg_inf()), q_zero = !(dv > neg_inf());   // NaN counts as -inf
+                    bool p_out = false, q_out = false;
                     if (kThr) {   // tokens that the truncation dropped have probability zero
-                        p_zero = p_zero || !(tv >= a.p_thr[row0 + j]);
-                        q_zero = q_zero || !(dv >= a.q_thr[dr]);
+                        p_out = !(tv >= a.p_thr[row0 + j]);
+                        q_out = !(dv >= a.q_thr[dr]);
                     }
-                    // r < min(1, ratio) without the division: a ratio >= 1 accepts every r in [0,1);
-                    // p(x) == 0 accepts none; q(x) == 0 < p(x) is a ratio of +inf
-                    const float r = a.uniforms[row0 + j];
-                    const float d = fminf(fmaxf(ap - aq, -126.f), 126.f);
-                    const float num = __fmul_rn(exp2f(d), qs.y);
-                    acc = !p_zero && (q_zero || num >= ps.y || __fmul_rn(r, ps.y) < num);
+                    acc = accept_test(tv, dv, ps, qs, a.c, a.uniforms[row0 + j], p_out, q_out);
                 }
                 rej = !acc;
             }
@@ -355,6 +365,120 @@ __global__ void __launch_bounds__(kThreads) verify_greedy_kernel(GreedyArgs a) {
         a.n_accepted[i] = n_acc;
         a.next_token[i] = a.p_argmax[row0 + n_acc];
     }
+}
+
+// ------------------------------------------------------------------ verify with early exit, phase 1
+
+// The accept tests of a sequence stop at its first rejection (Algorithm 1, verify loop), so the target rows
+// after it are never needed.  One cluster per sequence reads the target rows in order: statistics of row j,
+// accept test of position j, next row only if accepted.  Writes the (max, Z) of every row it read (the row
+// of the first rejection, or the bonus row, is the last) and the number of accepted tokens; greedy: also
+// the next token.
+struct ScanArgs {
+    const int32_t* draft_tokens;
+    const void* q_logits;
+    long q_row_stride;
+    const float2* q_stats_user;   // indexed by draft row, or NULL
+    const float2* q_stats_ws;     // indexed by target row (used when q_stats_user is NULL)
+    long q_seq_stride, q_pos_stride;
+    const void* t_logits;
+    long t_row_stride;
+    float2* p_stats;              // out, indexed by target row
+    const int32_t* cu;
+    int K, V;
+    float c;
+    const float* uniforms;
+    int32_t* n_accepted;
+    int32_t* next_token;          // greedy only
+    unsigned* status;
+};
+
+struct ScanShared2 {
+    // what the accept test of positions j0 .. j0+31 needs besides the target row's statistics
+    float tv[32], dv[32], r[32];
+    float2 qs[32];
+    int x[32];
+    int go;                       // decision of the current row: 1 = accepted, read the next row
+};
+
+template <int DT, bool kGreedy>
+__global__ void __launch_bounds__(kThreads) verify_scan_kernel(ScanArgs a) {
+    using E = ElemTraits<DT>;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int S = cluster.dim_blocks().x;
+    const int rank = cluster.block_rank();
+    const int i = blockIdx.x / S;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __shared__ SegEntry seg[2][kWarps];   // by row parity: a peer may still read row j while row j+1 is reduced
+    __shared__ ScanShared2 sh;
+    extern __shared__ uint4 ring[];
+    const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
+
+    pdl_launch_dependents();
+    pdl_wait();
+    const int row0 = a.cu ? a.cu[i] : i * (a.K + 1);
+    const int Ki = a.cu ? a.cu[i + 1] - row0 - 1 : a.K;
+    const long dbase = a.q_seq_stride < 0 ? static_cast<long>(row0 - i) : i * a.q_seq_stride;
+    const long dstep = a.q_seq_stride < 0 ? 1 : a.q_pos_stride;
+    const char* tl = static_cast<const char*>(a.t_logits);
+    const char* ql = static_cast<const char*>(a.q_logits);
+
+    int n_acc = Ki;
+    int last_idx = 0;
+    for (int j = 0; j <= Ki; ++j) {
+        if ((j & 31) == 0 && j < Ki) {
+            // the drafted tokens of the next 32 positions, their two logits, the draft rows' statistics
+            __syncthreads();
+            if (warp == 0 && j + lane < Ki) {
+                const int jj = j + lane;
+                const long dr = dbase + jj * dstep;
+                const int x = a.draft_tokens[dr];
+                sh.x[lane] = x;
+                if (!kGreedy) {
+                    const bool in = x >= 0 && x < a.V;
+                    sh.tv[lane] = in ? E::load_one(tl + static_cast<size_t>(row0 + jj) * a.t_row_stride * E::kBytes, x) : 0.f;
+                    sh.dv[lane] = in ? E::load_one(ql + static_cast<size_t>(dr) * a.q_row_stride * E::kBytes, x) : 0.f;
+                    sh.qs[lane] = a.q_stats_user ? a.q_stats_user[dr] : a.q_stats_ws[row0 + jj];
+                    sh.r[lane] = a.uniforms[row0 + jj];
+                }
+            }
+        }
+        const char* trow = tl + static_cast<size_t>(row0 + j) * a.t_row_stride * E::kBytes;
+        const RowGeom g = make_geom<DT>(trow, a.V, S * kWarps);
+        SegEntry* mine = seg[j & 1];
+        Partial t = reduce_segment<DT, kGreedy ? 0 : 1, kGreedy, false>(g, rank * kWarps + warp, a.c, lane, slot0, neg_inf());
+        if (lane == 0) { mine[warp].m = t.m; mine[warp].idx = t.idx; mine[warp].Z = t.Z; mine[warp].A = t.A; }
+        cluster.sync();
+        if (warp == 0) {
+            Partial r; SegPick p;
+            combine_segments<kGreedy ? 0 : 1>(cluster, mine, S, a.c, 0.f, lane, r, p);
+            const bool ok = fabsf(r.m) <= kMaxLogit && (kGreedy || r.Z > 0.f);
+            const int idx = (r.idx >= 0 && r.idx < a.V) ? r.idx : 0;
+            int go = 0;
+            if (j < Ki) {
+                const int k = j & 31;
+                const int x = sh.x[k];
+                if (kGreedy) go = x == idx;
+                else if (x >= 0 && x < a.V)
+                    go = accept_test(sh.tv[k], sh.dv[k], make_float2(r.m, r.Z), sh.qs[k], a.c, sh.r[k], false, false);
+            }
+            if (lane == 0) {
+                sh.go = go;
+                if (rank == 0) {
+                    if (!ok) atomicOr(a.status, SVIP_STATUS_NONFINITE_ROW);
+                    if (!kGreedy) a.p_stats[row0 + j] = make_float2(r.m, r.Z);
+                }
+            }
+            last_idx = idx;
+        }
+        __syncthreads();
+        if (!sh.go) { n_acc = j; break; }
+    }
+    if (rank == 0 && tid == 0) {
+        a.n_accepted[i] = n_acc;
+        if (kGreedy) a.next_token[i] = last_idx;
+    }
+    cluster.sync();   // no block leaves while a peer may still read its segment entries
 }
 
 }  // namespace svip

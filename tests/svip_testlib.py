@@ -67,7 +67,8 @@ def gpu_draft_step(ctx, logits: np.ndarray, T, h, uniforms, want_stats=True, pad
 
 
 def gpu_verify(ctx, draft_tokens, q_logits, target_logits, cu_rows, K, T, uniforms, q_stats=None,
-               fixed_K=False, layout="packed", q_seq_stride=None, q_pos_stride=None):
+               fixed_K=False, layout="packed", q_seq_stride=None, q_pos_stride=None, early_exit=False):
+    """svip_verify; with early_exit also svip_verify_early_exit on the same buffers: returns (plain, early)."""
     torch = torch_mod()
     B = len(cu_rows) - 1
     Rp, V = target_logits.shape
@@ -86,7 +87,15 @@ def gpu_verify(ctx, draft_tokens, q_logits, target_logits, cu_rows, K, T, unifor
     ctx.verify(d_tok, d_q, V, d_qs, qs, qp, d_t, V, dtype_code(target_logits), d_cu, B, K, Rp, V, T, d_u,
                n_acc, nxt, None)
     torch.cuda.synchronize()
-    return n_acc.cpu().numpy(), nxt.cpu().numpy()
+    got = n_acc.cpu().numpy(), nxt.cpu().numpy()
+    if not early_exit:
+        return got
+    # the early-exit entry point on the same buffers
+    n_acc.fill_(-7); nxt.fill_(-7)
+    ctx.verify_early_exit(d_tok, d_q, V, d_qs, qs, qp, d_t, V, dtype_code(target_logits), d_cu, B, K, Rp, V, T, d_u,
+                          n_acc, nxt, None)
+    torch.cuda.synchronize()
+    return got, (n_acc.cpu().numpy(), nxt.cpu().numpy())
 
 
 # ---------------------------------------------------------------- oracle-side guard bands / predicates

@@ -86,9 +86,10 @@ def test_long_draft_of_200_tokens(ctx, oracle):
     tok, _, _ = oracle.draft_step(q, 1.0, 0.3, rng.random(K))
     tok = tok.astype(np.int32)
     uv, _ = tl.guard_accept_uniforms(oracle, tok, q, tgt, cu, 1.0, rng.random(K + 1).astype(np.float32))
-    got = tl.gpu_verify(ctx, tok, q, tgt, cu, K, 1.0, uv, fixed_K=True)
+    got, early = tl.gpu_verify(ctx, tok, q, tgt, cu, K, 1.0, uv, fixed_K=True, early_exit=True)
     c = tl.check_verify_against_oracle(oracle, tok, q, tgt, cu, 1.0, uv, got, "K=200")
     assert c["mean_accepted"] >= 150     # the first rejection lies beyond four ballots of 32
+    tl.check_verify_against_oracle(oracle, tok, q, tgt, cu, 1.0, uv, early, "K=200 (early exit)")
 
 
 def test_masked_draft_step_leaves_skipped_rows_alone(ctx, oracle):

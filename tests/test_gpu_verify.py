@@ -39,7 +39,9 @@ def run_case(ctx, oracle, lens, cu, q, tgt, ud, uv, T, K_max, label, with_stats=
     stats = None
     if with_stats and T > 0:
         stats = tl.gpu_draft_step(ctx, q, T, 0.3, ud)[3]
-    got = tl.gpu_verify(ctx, tok, q, tgt, cu, K_max, T, uv if T > 0 else None, q_stats=stats, fixed_K=fixed)
+    got, early = tl.gpu_verify(ctx, tok, q, tgt, cu, K_max, T, uv if T > 0 else None, q_stats=stats, fixed_K=fixed,
+                               early_exit=True)
+    tl.check_verify_against_oracle(oracle, tok, q, tgt, cu, T, uv, early, label + " (early exit)")
     return tl.check_verify_against_oracle(oracle, tok, q, tgt, cu, T, uv, got, label)
 
 
@@ -99,8 +101,10 @@ def test_position_major_draft_layout(ctx, oracle):
         for j in range(lens[i]):
             q_pm[j * B + i] = q[cu[i] - i + j]; tok_pm[j * B + i] = tok[cu[i] - i + j]
     uv, _ = tl.guard_accept_uniforms(oracle, tok.astype(np.int32), q, tgt, cu, 1.0, uv)
-    got = tl.gpu_verify(ctx, tok_pm, q_pm, tgt, cu, K, 1.0, uv, layout="strided", q_seq_stride=1, q_pos_stride=B)
+    got, early = tl.gpu_verify(ctx, tok_pm, q_pm, tgt, cu, K, 1.0, uv, layout="strided", q_seq_stride=1, q_pos_stride=B,
+                               early_exit=True)
     tl.check_verify_against_oracle(oracle, tok.astype(np.int32), q, tgt, cu, 1.0, uv, got, "position-major")
+    tl.check_verify_against_oracle(oracle, tok.astype(np.int32), q, tgt, cu, 1.0, uv, early, "position-major (early exit)")
 
 
 def test_pack_ragged(ctx, oracle):
@@ -191,11 +195,18 @@ def test_published_configs(ctx, oracle, name):
         uv, moved = tl.guard_accept_uniforms(oracle, tok, w.q_logits, w.target_logits, w.cu_rows, T,
                                              w.verify_uniforms, threads=16)
         stats = tl.gpu_draft_step(ctx, w.q_logits, T, w.h, w.draft_uniforms)[3] if T > 0 else None
-        got = tl.gpu_verify(ctx, tok, w.q_logits, w.target_logits, w.cu_rows, w.K_max, T,
-                            uv if T > 0 else None, q_stats=stats, fixed_K=fixed)
+        got, early = tl.gpu_verify(ctx, tok, w.q_logits, w.target_logits, w.cu_rows, w.K_max, T,
+                                   uv if T > 0 else None, q_stats=stats, fixed_K=fixed, early_exit=True)
         c = tl.check_verify_against_oracle(oracle, tok, w.q_logits, w.target_logits, w.cu_rows, T, uv, got,
                                            "%s T=%g" % (name, T), threads=16)
-        print("verify parity", name, "T=%g" % T, c, "uniforms moved off the accept boundary:", moved)
+        ce = tl.check_verify_against_oracle(oracle, tok, w.q_logits, w.target_logits, w.cu_rows, T, uv, early,
+                                            "%s T=%g (early exit)" % (name, T), threads=16)
+        # the two entry points cut the rows over different numbers of blocks, so the fp32 normalisers differ in
+        # their last bits: the accepted counts must agree (the accept draws are off the boundary), the next
+        # token may fall on the other side of a CDF boundary within the tolerance
+        assert np.array_equal(got[0], early[0])
+        print("verify parity", name, "T=%g" % T, c, "early exit:", ce, "same next token in",
+              int((got[1] == early[1]).sum()), "of", len(got[1]), "uniforms moved off the accept boundary:", moved)
     if name == "tiny":   # target := draft everywhere: all K accepted, bonus token from row K
         t2 = w.target_logits.copy(); t2[:w.K_max] = w.q_logits
         tok, _, _ = oracle.draft_step(w.q_logits, 1.0, w.h, w.draft_uniforms)
@@ -330,3 +341,46 @@ def test_rejection_with_a_residual_below_fp32_resolution(ctx, oracle):
         n_b_zero64 += int(S64 == 0.0)
     assert n_a >= 9 and n_b_zero64 <= 5      # both families occurred
     assert ctx.read_status() == 0
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("T", [1.0, 0.0])
+def test_early_exit_never_reads_rows_after_the_first_rejection(ctx, oracle, bf16, T):
+    """The target rows after a sequence's first rejection are overwritten with NaN: svip_verify_early_exit
+    must still give the oracle's result on the clean rows and raise no status bit (a NaN row that is read
+    raises the non-finite bit, as the plain entry point shows on the same buffers)."""
+    import torch
+    rng = np.random.default_rng(77 + int(bf16) + int(T * 10))
+    lens, cu, q, tgt, ud, uv = small_case(rng, 24, 3000, 7, bf16, noise=0.8)
+    tok, _, _ = oracle.draft_step(q, T if T > 0 else 1.0, 0.3, ud, threads=8)
+    tok = tok.astype(np.int32)
+    uv, _ = tl.guard_accept_uniforms(oracle, tok, q, tgt, cu, T, uv)
+    n_ref, nx_ref, _ = oracle.verify(tok, q, tgt, cu, T, uv)
+    assert (n_ref < lens).sum() >= 8, "the case needs early rejections"
+    dirty = tgt.copy()
+    nan = np.uint16(0x7FC0) if bf16 else np.float32(np.nan)
+    poisoned = 0
+    for i in range(len(lens)):
+        lo, hi = cu[i] + n_ref[i] + 1, cu[i + 1]
+        dirty[lo:hi] = nan
+        poisoned += hi - lo
+    assert poisoned > 20
+    B, K = len(lens), 7
+    Rp, V = tgt.shape
+    dt = tl.dtype_code(tgt)
+    d_tok, d_q, d_t = tl.to_device(tok), tl.to_device(q), tl.to_device(dirty)
+    d_cu, d_u = tl.to_device(cu.astype(np.int32)), tl.to_device(uv.astype(np.float32))
+    n_acc = torch.full((B,), -7, dtype=torch.int32, device="cuda"); nxt = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+    for S in (0, 1, 2, 3, 8):
+        ctx.set_cluster_size(S)
+        assert ctx.read_status() == 0
+        n_acc.fill_(-7); nxt.fill_(-7)
+        ctx.verify_early_exit(d_tok, d_q, V, None, -1, 0, d_t, V, dt, d_cu, B, K, Rp, V, T, d_u if T > 0 else None, n_acc, nxt)
+        torch.cuda.synchronize()
+        assert ctx.read_status() == 0, "a row after the first rejection was read (S=%d)" % S
+        tl.check_verify_against_oracle(oracle, tok, q, tgt, cu, T, uv, (n_acc.cpu().numpy(), nxt.cpu().numpy()),
+                                       "early exit, poisoned tail, S=%d" % S)
+    ctx.set_cluster_size(0)
+    ctx.verify(d_tok, d_q, V, None, -1, 0, d_t, V, dt, d_cu, B, K, Rp, V, T, d_u if T > 0 else None, n_acc, nxt)
+    torch.cuda.synchronize()
+    assert ctx.read_status() & 1, "the plain entry point reads every row, the NaN ones too"
