@@ -541,19 +541,20 @@ static int verify_impl(svip_ctx* ctx, const int32_t* draft_tokens, const void* q
             if (e != cudaSuccess) return cuda_fail(ctx, e);
             ctx->launches += 1;
         }
-        ScanArgs w;
+        FinishArgs w;
         w.draft_tokens = draft_tokens; w.q_logits = q_logits; w.q_row_stride = q_row_stride;
         w.q_stats_user = reinterpret_cast<const float2*>(q_stats); w.q_stats_ws = ctx->q_stats;
         w.q_seq_stride = q_seq_stride; w.q_pos_stride = q_pos_stride; w.t_logits = target_logits;
-        w.t_row_stride = t_row_stride; w.p_stats = ctx->p_stats; w.cu = cu_rows; w.K = K; w.V = V; w.c = c;
+        w.t_row_stride = t_row_stride; w.p_stats = ctx->p_stats; w.p_stats_out = ctx->p_stats;
+        w.cu = cu_rows; w.K = K; w.V = V; w.c = c;
         w.uniforms = uniforms; w.n_accepted = n_accepted; w.next_token = next_token; w.status = ctx->status;
-        // the rows of a sequence are read one after another: a row is cut over enough blocks that the chain
-        // of the longest accepted run stays short (each block at most 128 KB of a row)
+        w.p_thr = nullptr; w.q_thr = nullptr; w.n_acc_in = nullptr;
+        // one cluster per sequence, cut as for the finish kernel (measured on 256 sequences of 1 MB rows: 2 or 4
+        // blocks per sequence are equally fast, 8 are slower; on 32 sequences of 304 KB rows 8 are fastest)
         int Sw = pick_cluster(ctx, B, V, dtype);
         if (ctx->cluster_override == 0) {
             const long row_bytes = static_cast<long>(V) * static_cast<long>(esz);
-            while (Sw < kMaxCluster && row_bytes / Sw > (128L << 10)) Sw *= 2;
-            if (Sw > kMaxCluster) Sw = kMaxCluster;
+            while (Sw < 4 && 2 * row_bytes / Sw > (512L << 10)) Sw *= 2;
         }
         if (timed) cudaEventRecord(ctx->prof_start[ctx->prof_used], st);
         if (sampling)
@@ -565,7 +566,7 @@ static int verify_impl(svip_ctx* ctx, const int32_t* draft_tokens, const void* q
         if (e != cudaSuccess) return cuda_fail(ctx, e);
         ctx->launches += 1;
         if (timed) cudaEventRecord(ctx->prof_stop[ctx->prof_used++], st);
-        if (!sampling) return SVIP_OK;
+        return SVIP_OK;
     } else {
     if (timed) cudaEventRecord(ctx->prof_start[ctx->prof_used], st);
     if (p_stats_user)
@@ -595,7 +596,7 @@ static int verify_impl(svip_ctx* ctx, const int32_t* draft_tokens, const void* q
         return SVIP_OK;
     }
 
-    if (!q_stats && !early_exit) {
+    if (!q_stats) {
         StatsArgs d = s;
         d.logits = q_logits; d.row_stride = q_row_stride; d.draft_rows = 1;
         d.out_stats = ctx->q_stats; d.out_argmax = nullptr; d.thr = q_thr;
@@ -620,7 +621,7 @@ static int verify_impl(svip_ctx* ctx, const int32_t* draft_tokens, const void* q
     f.cu = cu_rows; f.K = K; f.V = V; f.c = c;
     f.uniforms = uniforms; f.n_accepted = n_accepted; f.next_token = next_token; f.status = ctx->status;
     f.p_thr = p_thr; f.q_thr = q_thr;
-    f.n_acc_in = early_exit ? n_accepted : nullptr;
+    f.n_acc_in = nullptr; f.p_stats_out = nullptr;
     // up to two rows per sequence are streamed: long rows are cut finer than the one-wave policy
     // asks for (this kernel runs for many microseconds, so several waves are fine)
     int Sf = pick_cluster(ctx, B, V, dtype);

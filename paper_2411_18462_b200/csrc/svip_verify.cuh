@@ -26,6 +26,7 @@ struct FinishArgs {
     const float* p_thr;           // kThr: truncation threshold of every target row
     const float* q_thr;           // kThr: ... of every draft row (indexed like the draft tokens)
     const int32_t* n_acc_in;      // not NULL: the first rejection of every sequence is already known
+    float2* p_stats_out;          // verify_scan_kernel: (max, Z) of every target row it read, by target row
 };
 
 // Weights max(0, p - q) of Algorithm 4 (or p alone for the bonus token) for one vector.
@@ -205,75 +206,28 @@ struct FinishShared {
     SegPick pick;
 };
 
-template <int DT, bool kThr = false>
-__global__ void __launch_bounds__(kThreads, 2) verify_finish_kernel(FinishArgs a) {
+// Correction token from max(0, p - q) of the first rejected position, or bonus token from p of the row after
+// the last draft token (Algorithms 4 and 5), for sequence i whose number of accepted tokens is known.  Run by
+// every thread of the sequence's cluster; writes n_accepted[i] and next_token[i].
+template <int DT, bool kThr>
+__device__ __forceinline__ void finish_sequence(const FinishArgs& a, cg::cluster_group& cluster, int S, int rank,
+                                                int i, int row0, int Ki, long dbase, long dstep, int n_acc,
+                                                float2 ps, SegEntry* seg, ScanShared& scan, FinishShared& fs,
+                                                uint32_t slot0) {
     using E = ElemTraits<DT>;
     constexpr int EPV = E::kEPV;
-    cg::cluster_group cluster = cg::this_cluster();
-    const int S = cluster.dim_blocks().x;
-    const int rank = cluster.block_rank();
-    const int i = blockIdx.x / S;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    __shared__ SegEntry seg[kWarps];
-    __shared__ ScanShared scan;
-    __shared__ FinishShared fs;
-    extern __shared__ uint4 ring[];
-    const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
-
-    pdl_launch_dependents();
-    pdl_wait();
-    const int row0 = a.cu ? a.cu[i] : i * (a.K + 1);
-    const int Ki = a.cu ? a.cu[i + 1] - row0 - 1 : a.K;
-    const long dbase = a.q_seq_stride < 0 ? static_cast<long>(row0 - i) : i * a.q_seq_stride;
-    const long dstep = a.q_seq_stride < 0 ? 1 : a.q_pos_stride;
     const char* tl = static_cast<const char*>(a.t_logits);
     const char* ql = static_cast<const char*>(a.q_logits);
-
-    // Algorithm 2 at every position at once; the first rejection is the lowest set bit.
-    if (a.n_acc_in) {
-        if (tid == 0) fs.n_acc = min(max(a.n_acc_in[i], 0), Ki);
-    } else if (warp == 0) {
-        int n_acc = Ki;
-        for (int j0 = 0; j0 < Ki; j0 += 32) {
-            int j = j0 + lane;
-            bool rej = false;
-            if (j < Ki) {
-                long dr = dbase + j * dstep;
-                int x = a.draft_tokens[dr];
-                bool acc = false;
-                if (x >= 0 && x < a.V) {
-                    float tv = E::load_one(tl + static_cast<size_t>(row0 + j) * a.t_row_stride * E::kBytes, x);
-                    float dv = E::load_one(ql + static_cast<size_t>(dr) * a.q_row_stride * E::kBytes, x);
-                    float2 ps = a.p_stats[row0 + j];
-                    float2 qs = a.q_stats_user ? a.q_stats_user[dr] : a.q_stats_ws[row0 + j];
-                    bool p_out = false, q_out = false;
-                    if (kThr) {   // tokens that the truncation dropped have probability zero
-                        p_out = !(tv >= a.p_thr[row0 + j]);
-                        q_out = !(dv >= a.q_thr[dr]);
-                    }
-                    acc = accept_test(tv, dv, ps, qs, a.c, a.uniforms[row0 + j], p_out, q_out);
-                }
-                rej = !acc;
-            }
-            unsigned mask = __ballot_sync(0xffffffffu, rej);
-            if (mask) { n_acc = j0 + __ffs(mask) - 1; break; }
-        }
-        if (lane == 0) fs.n_acc = n_acc;
-    }
-    __syncthreads();
-    const int n_acc = fs.n_acc;
     const float u = a.uniforms[row0 + Ki];
 
     ResidualWeights<DT> wf;
     const char* trow = tl + static_cast<size_t>(row0 + n_acc) * a.t_row_stride * E::kBytes;
     wf.gt = make_geom<DT>(trow, a.V, S * kWarps);
     wf.c = a.c;
-    {
-        float2 ps = a.p_stats[row0 + n_acc];
-        wf.Mp = __fmul_rn(ps.x, a.c);
-        wf.rZp = 1.0f / ps.y;
-        if (kThr) wf.thr_p = a.p_thr[row0 + n_acc];
-    }
+    wf.Mp = __fmul_rn(ps.x, a.c);
+    wf.rZp = 1.0f / ps.y;
+    if (kThr) wf.thr_p = a.p_thr[row0 + n_acc];
     wf.bonus = n_acc >= Ki;
     wf.qrow = nullptr; wf.gq = wf.gt; wf.Mq = 0.f; wf.rZq = 0.f;
     if (!wf.bonus) {
@@ -331,6 +285,66 @@ __global__ void __launch_bounds__(kThreads, 2) verify_finish_kernel(FinishArgs a
     }
 }
 
+template <int DT, bool kThr = false>
+__global__ void __launch_bounds__(kThreads, 2) verify_finish_kernel(FinishArgs a) {
+    using E = ElemTraits<DT>;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int S = cluster.dim_blocks().x;
+    const int rank = cluster.block_rank();
+    const int i = blockIdx.x / S;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __shared__ SegEntry seg[kWarps];
+    __shared__ ScanShared scan;
+    __shared__ FinishShared fs;
+    extern __shared__ uint4 ring[];
+    const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
+
+    pdl_launch_dependents();
+    pdl_wait();
+    const int row0 = a.cu ? a.cu[i] : i * (a.K + 1);
+    const int Ki = a.cu ? a.cu[i + 1] - row0 - 1 : a.K;
+    const long dbase = a.q_seq_stride < 0 ? static_cast<long>(row0 - i) : i * a.q_seq_stride;
+    const long dstep = a.q_seq_stride < 0 ? 1 : a.q_pos_stride;
+    const char* tl = static_cast<const char*>(a.t_logits);
+    const char* ql = static_cast<const char*>(a.q_logits);
+
+    // Algorithm 2 at every position at once; the first rejection is the lowest set bit.
+    if (a.n_acc_in) {
+        if (tid == 0) fs.n_acc = min(max(a.n_acc_in[i], 0), Ki);
+    } else if (warp == 0) {
+        int n_acc = Ki;
+        for (int j0 = 0; j0 < Ki; j0 += 32) {
+            int j = j0 + lane;
+            bool rej = false;
+            if (j < Ki) {
+                long dr = dbase + j * dstep;
+                int x = a.draft_tokens[dr];
+                bool acc = false;
+                if (x >= 0 && x < a.V) {
+                    float tv = E::load_one(tl + static_cast<size_t>(row0 + j) * a.t_row_stride * E::kBytes, x);
+                    float dv = E::load_one(ql + static_cast<size_t>(dr) * a.q_row_stride * E::kBytes, x);
+                    float2 ps = a.p_stats[row0 + j];
+                    float2 qs = a.q_stats_user ? a.q_stats_user[dr] : a.q_stats_ws[row0 + j];
+                    bool p_out = false, q_out = false;
+                    if (kThr) {   // tokens that the truncation dropped have probability zero
+                        p_out = !(tv >= a.p_thr[row0 + j]);
+                        q_out = !(dv >= a.q_thr[dr]);
+                    }
+                    acc = accept_test(tv, dv, ps, qs, a.c, a.uniforms[row0 + j], p_out, q_out);
+                }
+                rej = !acc;
+            }
+            unsigned mask = __ballot_sync(0xffffffffu, rej);
+            if (mask) { n_acc = j0 + __ffs(mask) - 1; break; }
+        }
+        if (lane == 0) fs.n_acc = n_acc;
+    }
+    __syncthreads();
+    const int n_acc = fs.n_acc;
+    finish_sequence<DT, kThr>(a, cluster, S, rank, i, row0, Ki, dbase, dstep, n_acc, a.p_stats[row0 + n_acc], seg,
+                              scan, fs, slot0);
+}
+
 // ------------------------------------------------------------------ verify, phase 2 (greedy)
 
 struct GreedyArgs {
@@ -367,42 +381,23 @@ __global__ void __launch_bounds__(kThreads) verify_greedy_kernel(GreedyArgs a) {
     }
 }
 
-// ------------------------------------------------------------------ verify with early exit, phase 1
+// ------------------------------------------------------------------ verify with early exit
 
-// The accept tests of a sequence stop at its first rejection (Algorithm 1, verify loop), so the target rows
-// after it are never needed.  One cluster per sequence reads the target rows in order: statistics of row j,
-// accept test of position j, next row only if accepted.  Writes the (max, Z) of every row it read (the row
-// of the first rejection, or the bonus row, is the last) and the number of accepted tokens; greedy: also
-// the next token.
-struct ScanArgs {
-    const int32_t* draft_tokens;
-    const void* q_logits;
-    long q_row_stride;
-    const float2* q_stats_user;   // indexed by draft row, or NULL
-    const float2* q_stats_ws;     // indexed by target row (used when q_stats_user is NULL)
-    long q_seq_stride, q_pos_stride;
-    const void* t_logits;
-    long t_row_stride;
-    float2* p_stats;              // out, indexed by target row
-    const int32_t* cu;
-    int K, V;
-    float c;
-    const float* uniforms;
-    int32_t* n_accepted;
-    int32_t* next_token;          // greedy only
-    unsigned* status;
-};
-
-struct ScanShared2 {
+struct WalkShared {
     // what the accept test of positions j0 .. j0+31 needs besides the target row's statistics
     float tv[32], dv[32], r[32];
     float2 qs[32];
     int x[32];
     int go;                       // decision of the current row: 1 = accepted, read the next row
+    float2 ps;                    // (max, Z) of the current row
 };
 
+// The accept tests of a sequence stop at its first rejection (Algorithm 1, verify loop), so the target rows
+// after it are never needed.  One cluster per sequence reads the target rows in order: statistics of row j,
+// accept test of position j (Algorithm 2 / 3), next row only if accepted; then the correction or bonus token
+// from the row it stopped at (Algorithms 4 and 5).  Also writes the (max, Z) of every row it read.
 template <int DT, bool kGreedy>
-__global__ void __launch_bounds__(kThreads) verify_scan_kernel(ScanArgs a) {
+__global__ void __launch_bounds__(kThreads, 2) verify_scan_kernel(FinishArgs a) {
     using E = ElemTraits<DT>;
     cg::cluster_group cluster = cg::this_cluster();
     const int S = cluster.dim_blocks().x;
@@ -410,7 +405,9 @@ __global__ void __launch_bounds__(kThreads) verify_scan_kernel(ScanArgs a) {
     const int i = blockIdx.x / S;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     __shared__ SegEntry seg[2][kWarps];   // by row parity: a peer may still read row j while row j+1 is reduced
-    __shared__ ScanShared2 sh;
+    __shared__ WalkShared sh;
+    __shared__ ScanShared scan;
+    __shared__ FinishShared fs;
     extern __shared__ uint4 ring[];
     const uint32_t slot0 = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + tid * 16;
 
@@ -464,9 +461,10 @@ __global__ void __launch_bounds__(kThreads) verify_scan_kernel(ScanArgs a) {
             }
             if (lane == 0) {
                 sh.go = go;
+                sh.ps = make_float2(r.m, r.Z);
                 if (rank == 0) {
                     if (!ok) atomicOr(a.status, SVIP_STATUS_NONFINITE_ROW);
-                    if (!kGreedy) a.p_stats[row0 + j] = make_float2(r.m, r.Z);
+                    if (!kGreedy) a.p_stats_out[row0 + j] = make_float2(r.m, r.Z);
                 }
             }
             last_idx = idx;
@@ -474,11 +472,14 @@ __global__ void __launch_bounds__(kThreads) verify_scan_kernel(ScanArgs a) {
         __syncthreads();
         if (!sh.go) { n_acc = j; break; }
     }
-    if (rank == 0 && tid == 0) {
-        a.n_accepted[i] = n_acc;
-        if (kGreedy) a.next_token[i] = last_idx;
+    if (kGreedy) {
+        if (rank == 0 && tid == 0) { a.n_accepted[i] = n_acc; a.next_token[i] = last_idx; }
+        cluster.sync();   // no block leaves while a peer may still read its segment entries
+    } else {
+        // the entries of row n_acc - 1 have been read by every peer (they passed the barrier of row n_acc)
+        finish_sequence<DT, false>(a, cluster, S, rank, i, row0, Ki, dbase, dstep, n_acc, sh.ps, seg[(n_acc + 1) & 1],
+                                   scan, fs, slot0);
     }
-    cluster.sync();   // no block leaves while a peer may still read its segment entries
 }
 
 }  // namespace svip
