@@ -515,6 +515,45 @@ def graph_loop_round(ctx, torch, rnd, reps=20):
             "same_results_as_host_driven_round": same}
 
 
+def early_exit_leg(ctx, torch, rnd, reps=10):
+    """The round with svip_verify_early_exit in place of svip_verify: the target rows of a sequence are read in order
+    up to its first rejection.  Times the verify call alone in both forms and the whole round in both forms; counts
+    the target rows the early-exit form needs (n_accepted + 1 per sequence)."""
+    w, B, V = rnd.w, rnd.B, rnd.V
+    rnd.step()
+    torch.cuda.synchronize()
+    plain = (rnd.d_nacc.clone(), rnd.d_next.clone())
+    early = ctx.bind("verify_early_exit", rnd.d_tok, rnd.d_q, V, rnd.d_stats, 1, B, rnd.d_t, V, rnd.dt, rnd.d_cu, B,
+                     w.K_max, rnd.Rp, V, w.T, rnd.d_uv, rnd.d_nacc, rnd.d_next, rnd.stream)
+
+    def timed(calls):
+        for c in calls:
+            c()
+        torch.cuda.synchronize()
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            for c in calls:
+                c()
+        e1.record()
+        torch.cuda.synchronize()
+        return 1000.0 * e0.elapsed_time(e1) / reps
+
+    res = {"verify_us": timed(rnd.calls[-1:]), "verify_early_exit_us": timed([early]),
+           "round_us": timed(rnd.calls), "round_early_exit_us": timed(rnd.calls[:-1] + [early])}
+    nacc = rnd.d_nacc.cpu().numpy()
+    res["target_rows"] = rnd.Rp
+    res["target_rows_needed"] = int((nacc + 1).sum())
+    res["same_n_accepted"] = int((rnd.d_nacc == plain[0]).sum())
+    res["same_next_token"] = int((rnd.d_next == plain[1]).sum())
+    res["sequences"] = B
+    res["note"] = ("one kernel, one cluster per sequence; the rows of a sequence are read one after another, so it "
+                   "pays where rejections come early or the batch fills the GPU")
+    rnd.step()      # leave the plain round's results in the buffers
+    torch.cuda.synchronize()
+    return res
+
+
 def tree_leg(ctx, torch, reps=20):
     """svip_verify_tree on synthetic candidate trees: 64 sequences, binary trees of depth 3 (14 candidate
     nodes: the two most likely tokens of every node's draft row), V = 32000 bf16, target = draft + N(0, 0.5^2)."""
@@ -807,6 +846,10 @@ def other_workload(ctx, torch, name, rank, peak, peak_kind, steps):
            "stop_flags_match_draft_lengths": bool(m["stops_ok"]) if name == "ragged" else None,
            "status_word": m["status"],
            "roofline": {k: first[k] for k in keep}, "roofline_other": {k: second[k] for k in keep}}
+    try:
+        out["early_exit"] = early_exit_leg(ctx, torch, rnd, reps=5)
+    except Exception as exc:
+        out["early_exit"] = {"error": repr(exc)}
     if name == "ragged":
         try:
             out["device_loop_graph"] = graph_loop_round(ctx, torch, rnd)
@@ -896,7 +939,8 @@ def run_ours(args):
         legs = {"pair_stats": lambda: pair_stats_leg(ctx, torch, rnd, peak, reps=2),
                 "vocab_parallel": lambda: vocab_parallel_leg(ctx, torch, rnd, peak, reps=2),
                 "tree": lambda: tree_leg(ctx, torch, reps=2),
-                "truncated": lambda: truncated_round(ctx, torch, rnd, reps=2)}
+                "truncated": lambda: truncated_round(ctx, torch, rnd, reps=2),
+                "early_exit": lambda: early_exit_leg(ctx, torch, rnd, reps=2)}
         line[args.only_leg] = legs[args.only_leg]()
         print(json.dumps(line))
         return
@@ -911,6 +955,7 @@ def run_ours(args):
             line["truncated"] = {"error": repr(exc)}
         for key, leg in (("pair_stats", lambda: pair_stats_leg(ctx, torch, rnd, peak)),
                          ("vocab_parallel", lambda: vocab_parallel_leg(ctx, torch, rnd, peak)),
+                         ("early_exit", lambda: early_exit_leg(ctx, torch, rnd)),
                          ("tree", lambda: tree_leg(ctx, torch))):
             try:
                 line[key] = leg()
@@ -993,7 +1038,7 @@ def main():
                     help="sequences per GPU instead of the published batch size (smaller cases for profiling)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--only-leg", default=None, choices=["pair_stats", "vocab_parallel", "tree", "truncated"],
+    ap.add_argument("--only-leg", default=None, choices=["pair_stats", "vocab_parallel", "tree", "truncated", "early_exit"],
                     help="after the timed region run just this extra leg, briefly (for profiling it)")
     ap.add_argument("--skip-extras", action="store_true",
                     help="only the timed region: no end-to-end leg, no B=1 latency, no CPU baseline (for profiling)")
