@@ -146,9 +146,11 @@ def test_workspace_limit_and_bad_arguments():
     c.destroy()
 
 
-def test_graph_replay_matches_direct_calls(ctx, oracle):
+@pytest.mark.parametrize("early_exit", [False, True])
+def test_graph_replay_matches_direct_calls(ctx, oracle, early_exit):
     """B = 1: eight draft steps, packing and the verify round recorded once, replayed on new inputs."""
     import torch
+    verify = ctx.verify_early_exit if early_exit else ctx.verify
     w = W.make_workload("tiny")
     K, V = w.K_max, w.V
     dq = tl.to_device(w.q_logits); dt = tl.to_device(w.target_logits)
@@ -165,7 +167,7 @@ def test_graph_replay_matches_direct_calls(ctx, oracle):
                            tok.data_ptr() + 4 * j, ent.data_ptr() + 4 * j, stop.data_ptr() + j,
                            stats.data_ptr() + 8 * j, st)
         ctx.pack_ragged(lens, 1, K, cu, None, None, st)
-        ctx.verify(tok, dq, V, stats, -1, 0, dt, V, 0, cu, 1, K, K + 1, V, 1.0, uv, nacc, nxt, st)
+        verify(tok, dq, V, stats, -1, 0, dt, V, 0, cu, 1, K, K + 1, V, 1.0, uv, nacc, nxt, st)
 
     enqueue(); st.synchronize()
     direct = (tok.cpu().numpy().copy(), nacc.item(), nxt.item())
