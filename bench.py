@@ -262,22 +262,23 @@ def b1_latency(ctx, torch):
     nacc = torch.zeros(1, dtype=torch.int32, device="cuda"); nxt = torch.zeros(1, dtype=torch.int32, device="cuda")
     torch.cuda.synchronize()
 
-    def enqueue(s):
+    def enqueue(s, verify=None):
         for j in range(K):
             ctx.draft_step(dq.data_ptr() + j * V * 4, 0, 1, V, V, w.T, w.h, ud.data_ptr() + 4 * j,
                            tok.data_ptr() + 4 * j, ent.data_ptr() + 4 * j, stop.data_ptr() + j,
                            stats.data_ptr() + 8 * j, s)
         ctx.pack_ragged(lens, 1, K, cu, None, None, s)
-        ctx.verify(tok, dq, V, stats, -1, 0, dt, V, 0, cu, 1, K, K + 1, V, w.T, uv, nacc, nxt, s)
+        (verify or ctx.verify)(tok, dq, V, stats, -1, 0, dt, V, 0, cu, 1, K, K + 1, V, w.T, uv, nacc, nxt, s)
 
     out = {}
     with torch.cuda.stream(st):
         ctx.graph_begin(st); enqueue(st); g = ctx.graph_end(st)
+        ctx.graph_begin(st); enqueue(st, ctx.verify_early_exit); ge = ctx.graph_end(st)
         one = None
         ctx.graph_begin(st)
         ctx.draft_step(dq, 0, 1, V, V, w.T, w.h, ud, tok, ent, stop, stats, st)
         one = ctx.graph_end(st)
-        for name, graph, reps in (("round_us", g, 200), ("draft_step_us", one, 500)):
+        for name, graph, reps in (("round_us", g, 200), ("round_early_exit_us", ge, 200), ("draft_step_us", one, 500)):
             for _ in range(20):
                 graph.launch(st)
             e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
@@ -294,7 +295,8 @@ def b1_latency(ctx, torch):
                 graph.launch(st)
                 st.synchronize()
             out[name.replace("_us", "_to_host_us")] = 1e6 * (time.perf_counter() - t0) / reps
-        g.destroy(); one.destroy()
+        out["accepted_in_this_round"] = int(nacc.item())
+        g.destroy(); ge.destroy(); one.destroy()
 
         # one truncated draft step (top-k 50, top-p 0.9) at B = 1, by graph replay
         thr1 = torch.zeros(1, device="cuda")
